@@ -1,0 +1,342 @@
+"""Pins for the CPU oracle: it is checked against things other than itself.
+
+Brute force written a different way (numpy, coordinate ranges instead of tile-id
+distances), torch's fp64 scaled_dot_product_attention, the numbers the paper
+prints (tests/golden/paper_pins.json), closed forms and invariants.
+"""
+import json
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+
+GOLD = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "paper_pins.json")))
+
+
+# --------------------------------------------------------------------------- helpers
+def coords(grid):
+    T, H, W = grid
+    t, h, w = np.meshgrid(np.arange(T), np.arange(H), np.arange(W), indexing="ij")
+    return np.stack([t.ravel(), h.ravel(), w.ravel()], axis=1)  # frame-major token order
+
+
+def brute_mask(grid, tile, window):
+    """Token mask from key *coordinate ranges*: the window of (2*half+1) tiles,
+    shifted inward at the borders, turned into [lo, hi) token coordinates."""
+    c = coords(grid)
+    L = c.shape[0]
+    M = np.ones((L, L), dtype=bool)
+    for a in range(3):
+        nt = -(-grid[a] // tile[a])
+        half = window[a] // 2
+        if nt <= 2 * half + 1:
+            continue
+        q = c[:, a] // tile[a]
+        centre = np.clip(q, half, nt - 1 - half)
+        lo = (centre - half) * tile[a]
+        hi = np.minimum((centre + half + 1) * tile[a], grid[a])
+        k = c[:, a]
+        M &= (k[None, :] >= lo[:, None]) & (k[None, :] < hi[:, None])
+    return M
+
+
+def dense_attention(Q, K, V, scale, mask=None):
+    S = scale * (Q @ K.T)
+    if mask is not None:
+        S = np.where(mask, S, -np.inf)
+    S = S - S.max(axis=1, keepdims=True)
+    P = np.exp(S)
+    P /= P.sum(axis=1, keepdims=True)
+    return P @ V, P
+
+
+def brute_select(grid, bucket, r, X):
+    """Bucketed selection written with numpy sorting, bucket by bucket."""
+    T, H, W = grid
+    tok = np.arange(T * H * W).reshape(T, H, W)
+    core, src = [], np.zeros(T * H * W, dtype=np.int64)
+    for bt in range(0, T, bucket[0]):
+        for bh in range(0, H, bucket[1]):
+            for bw in range(0, W, bucket[2]):
+                blk = tok[bt:bt + bucket[0], bh:bh + bucket[1], bw:bw + bucket[2]]
+                e = blk.shape
+                ids = blk.ravel()
+                n = ids.size
+                ci = np.ravel_multi_index((e[0] // 2, e[1] // 2, e[2] // 2), e)
+                xc = X[ids[ci]]
+                others = np.array([l for l in range(n) if l != ci], dtype=np.int64)
+                xo = X[ids[others]]
+                den = np.linalg.norm(xc) * np.linalg.norm(xo, axis=1)
+                cos = np.where(den > 0, (xo @ xc) / np.where(den > 0, den, 1.0), 0.0)
+                keep = max(1, int(np.floor(r * n + 0.5)))
+                k = n - keep
+                order = np.lexsort((others, -cos))  # primary: cos descending; then index
+                pruned = set(others[order[:k]].tolist())
+                seg = len(core)
+                core.append(ids[ci])
+                src[ids[ci]] = seg
+                for l in range(n):
+                    if l == ci:
+                        continue
+                    if l in pruned:
+                        src[ids[l]] = seg
+                    else:
+                        src[ids[l]] = len(core)
+                        core.append(ids[l])
+    return np.array(core, dtype=np.int64), src
+
+
+def rand_qkv(L, d, seed):
+    g = np.random.default_rng(seed)
+    return (g.standard_normal((L, d)), g.standard_normal((L, d)), g.standard_normal((L, d)))
+
+
+GRIDS = [
+    # grid, tile, window (tiles)
+    ((4, 8, 8), (2, 4, 4), (3, 3, 3)),      # window covers the 2x2x2 tile grid
+    ((5, 7, 9), (1, 2, 2), (3, 3, 3)),      # ragged on H and W, real windows on all axes
+    ((8, 6, 10), (2, 2, 2), (3, 1, 5)),     # per-axis windows: 3, 1 (own tile only), 5
+    ((10, 5, 5), (2, 2, 3), (2, 3, 3)),     # even window behaves like the next odd one
+]
+
+
+# --------------------------------------------------------------------------- sliding tile mask
+@pytest.mark.parametrize("grid,tile,window", GRIDS)
+def test_token_mask_matches_coordinate_range_brute_force(grid, tile, window):
+    M = oracle.sta_token_mask(grid, tile, window).astype(bool)
+    assert np.array_equal(M, brute_mask(grid, tile, window))
+
+
+@pytest.mark.parametrize("grid,tile,window", GRIDS)
+def test_block_mask_expands_to_token_mask(grid, tile, window):
+    BM = oracle.sta_block_mask(grid, tile, window)
+    c = coords(grid)
+    nt = [-(-g // t) for g, t in zip(grid, tile)]
+    tid = ((c[:, 0] // tile[0]) * nt[1] + c[:, 1] // tile[1]) * nt[2] + c[:, 2] // tile[2]
+    assert np.array_equal(BM[tid][:, tid].astype(bool), brute_mask(grid, tile, window))
+
+
+@pytest.mark.parametrize("grid,tile,window", GRIDS + [((21, 30, 52), (4, 4, 4), (3, 3, 3))])
+def test_block_mask_row_counts_closed_form(grid, tile, window):
+    BM = oracle.sta_block_mask(grid, tile, window)
+    nt = [-(-g // t) for g, t in zip(grid, tile)]
+    per_row = int(np.prod([min(n, 2 * (w // 2) + 1) for n, w in zip(nt, window)]))
+    assert (BM.sum(axis=1) == per_row).all()
+    assert (np.diag(BM) == 1).all()  # every tile sees itself
+
+
+def test_block_mask_is_not_symmetric_at_the_border():
+    BM = oracle.sta_block_mask((1, 1, 8), (1, 1, 1), (1, 1, 3))
+    # tile 0's window is shifted inward to tiles {0,1,2}; tile 2's window is {1,2,3}
+    assert BM[0].tolist() == [1, 1, 1, 0, 0, 0, 0, 0]
+    assert BM[2].tolist() == [0, 1, 1, 1, 0, 0, 0, 0]
+    assert BM[7].tolist() == [0, 0, 0, 0, 0, 1, 1, 1]
+    assert BM[0, 2] == 1 and BM[2, 0] == 0
+
+
+def test_paper_window_18_27_24_gives_11664_keys():
+    g = GOLD["sliding_window_keys"]
+    grid, tile, win = g["grid"], g["tile"], g["window_tiles"]
+    assert [t * w for t, w in zip(tile, win)] == g["window_tokens"]
+    assert grid[0] * grid[1] * grid[2] == g["tokens"]
+    BM = oracle.sta_block_mask(grid, tile, win)
+    keys = BM.sum(axis=1) * (tile[0] * tile[1] * tile[2])  # the grid divides into whole tiles
+    assert (keys == g["keys_per_query"]).all()
+    assert abs(g["keys_per_query"] / g["tokens"] - 0.108) < 1e-12
+
+
+# --------------------------------------------------------------------------- attention
+@pytest.mark.parametrize("L,d", [(37, 8), (64, 16)])
+def test_full_attention_vs_torch_sdpa_and_numpy(L, d):
+    Q, K, V = rand_qkv(L, d, 1)
+    scale = 1.0 / np.sqrt(d)
+    O, P = oracle.attn_full(Q, K, V, scale, return_probs=True)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(Q)[None], torch.from_numpy(K)[None], torch.from_numpy(V)[None],
+        scale=scale)[0].numpy()
+    assert np.abs(O - ref).max() < 1e-12
+    On, Pn = dense_attention(Q, K, V, scale)
+    assert np.abs(O - On).max() < 1e-12 and np.abs(P - Pn).max() < 1e-13
+    assert np.abs(P.sum(axis=1) - 1).max() < 1e-12 and (P >= 0).all()
+
+
+def test_full_attention_row_subset():
+    Q, K, V = rand_qkv(50, 8, 2)
+    rows = [49, 0, 7, 7, 13]
+    O = oracle.attn_full(Q, K, V, 0.3)
+    assert np.array_equal(oracle.attn_full(Q, K, V, 0.3, q_rows=rows), O[rows])
+
+
+@pytest.mark.parametrize("grid,tile,window", GRIDS[1:])
+def test_sliding_attention_vs_brute_force_and_sdpa(grid, tile, window):
+    L = grid[0] * grid[1] * grid[2]
+    d = 8
+    Q, K, V = rand_qkv(L, d, 3)
+    scale = 1.0 / np.sqrt(d)
+    O, P = oracle.attn_sliding(grid, tile, window, Q, K, V, scale, return_probs=True)
+    M = brute_mask(grid, tile, window)
+    On, Pn = dense_attention(Q, K, V, scale, M)
+    assert np.abs(O - On).max() < 1e-12
+    assert np.abs(P - Pn).max() < 1e-13
+    assert (P[~M] == 0).all()
+    assert np.abs(P.sum(axis=1) - 1).max() < 1e-12
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(Q)[None], torch.from_numpy(K)[None], torch.from_numpy(V)[None],
+        attn_mask=torch.from_numpy(M)[None], scale=scale)[0].numpy()
+    assert np.abs(O - ref).max() < 1e-12
+    # the masked result really differs from full attention
+    assert np.abs(O - oracle.attn_full(Q, K, V, scale)).max() > 1e-3
+
+
+def test_window_covering_the_grid_is_full_attention():
+    grid, tile, window = GRIDS[0]
+    Q, K, V = rand_qkv(256, 16, 4)
+    a = oracle.attn_sliding(grid, tile, window, Q, K, V, 0.25)
+    b = oracle.attn_full(Q, K, V, 0.25)
+    assert np.array_equal(a, b)
+
+
+def test_scaling_v_and_permuting_keys():
+    Q, K, V = rand_qkv(48, 8, 5)
+    O = oracle.attn_full(Q, K, V, 0.35)
+    assert np.abs(oracle.attn_full(Q, K, 3.0 * V, 0.35) - 3.0 * O).max() < 1e-12
+    perm = np.random.default_rng(0).permutation(48)
+    assert np.abs(oracle.attn_full(Q, K[perm], V[perm], 0.35) - O).max() < 1e-12
+    # queries and keys are not interchangeable
+    assert np.abs(oracle.attn_full(K, Q, V, 0.35) - O).max() > 1e-3
+
+
+# --------------------------------------------------------------------------- core-set selection
+def test_keep_count_rounding():
+    # a grid that is one bucket: Lc = keep(n)
+    for n_dims, r, want in [((2, 3, 2), 0.5, 6), ((2, 3, 2), 0.25, 3), ((1, 3, 2), 0.5, 3),
+                            ((1, 3, 2), 0.25, 2), ((2, 2, 2), 0.5, 4), ((2, 2, 2), 0.25, 2),
+                            ((1, 3, 3), 0.5, 5), ((1, 1, 1), 0.25, 1), ((1, 1, 2), 0.1, 1)]:
+        assert oracle.coreset_len(n_dims, (2, 3, 3), r) == want, (n_dims, r)
+
+
+def test_fig2_bucket_centre_and_dropped_count():
+    g = GOLD["bcs_figure"]
+    grid = g["bucket"]
+    X = np.random.default_rng(6).standard_normal((9, 5))
+    core, src = oracle.coreset_select(grid, grid, 0.5, X)
+    assert core[0] == g["centre_local_index_0_based"]
+    assert len(core) == g["kept"] and 9 - len(core) == g["dropped"]
+    assert sorted(core[1:].tolist()) == core[1:].tolist()
+
+
+def test_half_coreset_quarter_cost_and_config_lengths():
+    g = GOLD["coreset_cost"]
+    b = GOLD["bucket_defaults"]["bucket"]
+    for grid in [(4, 6, 4), (8, 9, 10), (30, 45, 80)]:
+        L = grid[0] * grid[1] * grid[2]
+        Lc = oracle.coreset_len(grid, b, g["ratio"])
+        assert 2 * Lc == L
+        assert (Lc * Lc) / (L * L) == g["cost_fraction"]
+    assert oracle.coreset_len((4, 8, 8), b, 0.25) == 64
+    assert oracle.coreset_len((21, 30, 52), b, 0.5) == 16380
+    assert oracle.coreset_len((33, 45, 80), b, 0.5) == 59400
+    assert oracle.coreset_len((33, 45, 80), b, 0.25) == 30000
+    assert oracle.coreset_len((21, 45, 80), b, 0.25) == 19200
+
+
+@pytest.mark.parametrize("grid,bucket,r", [((4, 6, 4), (2, 3, 2), 0.5), ((5, 7, 5), (2, 3, 2), 0.25),
+                                           ((3, 8, 8), (2, 3, 2), 0.5), ((4, 4, 4), (1, 2, 3), 0.7)])
+def test_selection_vs_numpy_brute_force(grid, bucket, r):
+    L = grid[0] * grid[1] * grid[2]
+    X = np.random.default_rng(7).standard_normal((L, 12))
+    core, src = oracle.coreset_select(grid, bucket, r, X)
+    bc, bs = brute_select(grid, bucket, r, X)
+    assert np.array_equal(core, bc) and np.array_equal(src, bs)
+    assert len(core) == oracle.coreset_len(grid, bucket, r)
+    # kept tokens map to themselves, every token maps to a slot of its own bucket
+    assert np.array_equal(src[core], np.arange(len(core)))
+
+
+def test_multiples_of_the_centre_are_pruned_before_orthogonal_tokens():
+    grid = bucket = (2, 3, 2)  # one bucket of 12, centre local index (1*3+1)*2+1 = 9
+    X = np.zeros((12, 4))
+    X[9] = [1, 2, 0, 0]
+    dup = [0, 3, 5, 10]                     # positive multiples of the centre: cos = 1
+    for j, l in enumerate(dup):
+        X[l] = (j + 1) * X[9]
+    for l in range(12):
+        if l != 9 and l not in dup:
+            X[l] = [0, 0, 1 + l, 0.5]       # orthogonal to the centre: cos = 0
+    core, src = oracle.coreset_select(grid, bucket, 8 / 12, X)  # keep 8, prune 4
+    assert set(range(12)) - set(core.tolist()) == set(dup)
+    assert core[0] == 9 and (src[dup] == 0).all()
+    # negative multiples (cos = -1) are the last to go
+    X[3] = -X[9]
+    core, _ = oracle.coreset_select(grid, bucket, 8 / 12, X)
+    assert 3 in core.tolist()
+
+
+def test_ties_prune_lower_local_index_first_and_zero_norm_scores_zero():
+    grid = bucket = (2, 3, 2)
+    X = np.ones((12, 3))                    # all cosines equal
+    core, src = oracle.coreset_select(grid, bucket, 0.5, X)
+    assert core.tolist() == [9, 6, 7, 8, 10, 11]
+    assert src.tolist() == [0, 0, 0, 0, 0, 0, 1, 2, 3, 0, 4, 5]
+    X = np.zeros((12, 3))                   # zero norms: every score is 0, same tie-break
+    core2, _ = oracle.coreset_select(grid, bucket, 0.5, X)
+    assert core2.tolist() == core.tolist()
+
+
+def test_ratio_one_keeps_everything_and_equals_full_attention():
+    grid, bucket = (3, 5, 4), (2, 3, 2)
+    L = 60
+    Q, K, V = rand_qkv(L, 8, 8)
+    core, src = oracle.coreset_select(grid, bucket, 1.0, K)
+    assert sorted(core.tolist()) == list(range(L))
+    assert np.array_equal(core[src], np.arange(L))          # src_slot inverts core_idx
+    O, _, _ = oracle.attn_coreset(grid, bucket, 1.0, Q, K, V, 0.35)
+    assert np.abs(O - oracle.attn_full(Q, K, V, 0.35)).max() < 1e-12
+
+
+def test_coreset_attention_vs_explicit_gather_and_scatter():
+    grid, bucket, r = (4, 6, 6), (2, 3, 2), 0.5
+    L, d = 144, 8
+    Q, K, V = rand_qkv(L, d, 9)
+    X = np.random.default_rng(10).standard_normal((L, 6))
+    O, core, src = oracle.attn_coreset(grid, bucket, r, Q, K, V, 0.35, X=X)
+    bc, bs = brute_select(grid, bucket, r, X)
+    assert np.array_equal(core, bc) and np.array_equal(src, bs)
+    Oc, _ = dense_attention(Q[bc], K[bc], V[bc], 0.35)
+    assert np.abs(O - Oc[bs]).max() < 1e-12
+    # a pruned token's row is a bit-identical copy of its centre's row
+    pruned = np.setdiff1d(np.arange(L), core)
+    assert len(pruned) == L - len(core) > 0
+    assert np.array_equal(O[pruned], O[core[src[pruned]]])
+    # row subset agrees with the full call; default X is K
+    rows = [143, 5, 5, 77]
+    Osub, _, _ = oracle.attn_coreset(grid, bucket, r, Q, K, V, 0.35, X=X, q_rows=rows)
+    assert np.array_equal(Osub, O[rows])
+    Ok, corek, _ = oracle.attn_coreset(grid, bucket, r, Q, K, V, 0.35)
+    assert np.array_equal(corek, oracle.coreset_select(grid, bucket, r, K)[0])
+
+
+def test_bucket_constant_features_make_coreset_equal_full():
+    grid, bucket = (4, 6, 4), (2, 3, 2)     # divides into 8 whole buckets of 12
+    g = np.random.default_rng(11)
+    c = coords(grid)
+    bid = ((c[:, 0] // 2) * 2 + c[:, 1] // 3) * 2 + c[:, 2] // 2
+    Q, K, V = (g.standard_normal((8, 8))[bid] for _ in range(3))
+    O, core, src = oracle.attn_coreset(grid, bucket, 0.5, Q, K, V, 0.35)
+    assert np.abs(O - oracle.attn_full(Q, K, V, 0.35)).max() < 1e-12
+    # all cosines tie, so each bucket keeps its centre and its highest local indices
+    first = core[:6].tolist()
+    tok = np.arange(96).reshape(grid)[:2, :3, :2].ravel()
+    assert first == [tok[9], tok[6], tok[7], tok[8], tok[10], tok[11]]
+
+
+def test_min_gap_reports_near_ties():
+    grid = bucket = (2, 3, 2)
+    X = np.random.default_rng(12).standard_normal((12, 6))
+    _, _, gap = oracle.coreset_select(grid, bucket, 0.5, X, return_gap=True)
+    assert 0 < gap < 2
+    _, _, gap1 = oracle.coreset_select(grid, bucket, 1.0, X, return_gap=True)
+    assert gap1 == np.inf
