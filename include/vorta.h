@@ -1,0 +1,209 @@
+/*
+ * vorta.h -- C ABI of the B200 (sm_100a) routed-attention library.
+ *
+ * The library computes the attention of one video-diffusion-transformer layer in
+ * which every head is routed to one of three branches (VORTA, Section 3.3,
+ * Eq. 4): full 3D attention (Section 2, Eq. 2), 3D sliding tile attention
+ * (Section 3.2 and Appendix A.1, Algorithm 1), or core-set attention
+ * unpool(attn(pool(.))) with bucketed core-set selection (Section 3.2;
+ * Appendix A.1 "Bucketed coreset selection").
+ *
+ * Conventions shared by all entry points
+ *   - Tokens are 0-based and frame-major: i = (t*H + h)*W + w, L = T*H*W.
+ *   - Q, K, V, O are bf16, contiguous [B, heads, L, d]; d is 64 or 128.
+ *   - "dev" pointers are CUDA device memory, "host" pointers ordinary host
+ *     memory.  The caller owns every buffer it passes and the stream; the library
+ *     owns the plan and the small device tables inside it.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     Calls enqueue work and return; argument errors are reported synchronously
+ *     and launch nothing.
+ *   - Every function returns a vorta_status; nothing throws, aborts or prints.
+ *   - Device-side waits are bounded.  If one expires, the kernel records a code
+ *     and leaves; vorta_device_status() reports it after the stream has drained.
+ *   - A plan may be used from one thread at a time.
+ */
+#ifndef VORTA_H_
+#define VORTA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define VORTA_API __attribute__((visibility("default")))
+#else
+#define VORTA_API
+#endif
+
+typedef struct vorta_plan vorta_plan; /* opaque */
+
+typedef enum {
+    VORTA_OK = 0,
+    VORTA_ERR_INVALID_ARG = 1,  /* null pointer, size out of range, bad route id ... */
+    VORTA_ERR_UNSUPPORTED = 2,  /* valid request this build cannot run (see vorta_plan_create) */
+    VORTA_ERR_ALIGNMENT = 3,    /* a device pointer is not 16-byte aligned */
+    VORTA_ERR_WORKSPACE = 4,    /* workspace missing or too small */
+    VORTA_ERR_CUDA = 5,         /* a CUDA runtime/driver call failed */
+    VORTA_ERR_TIMEOUT = 6,      /* a bounded device-side wait expired */
+    VORTA_ERR_INTERNAL = 7      /* a self-check inside the library failed */
+} vorta_status;
+
+/* Branch ids, in the order of the gate vector [alpha_1, alpha_2, alpha_3] of
+ * Section 3.3, Eq. 3: full, sliding-window, core-set. */
+enum { VORTA_ROUTE_FULL = 0, VORTA_ROUTE_SLIDING = 1, VORTA_ROUTE_CORESET = 2 };
+
+/* vorta_plan_desc.flags */
+enum {
+    VORTA_PLAN_HOST_ONLY = 1 /* geometry and accounting only: needs no GPU, cannot launch */
+};
+
+/* Which attention kernel vorta_routed_attention launches. */
+enum {
+    VORTA_KERNEL_TCGEN05 = 0, /* default: persistent TMA + tcgen05/TMEM kernel */
+    VORTA_KERNEL_SIMT = 1     /* slow CUDA-core kernel over the same work lists (debug aid) */
+};
+
+typedef struct {
+    int32_t B, heads;     /* batch, attention heads; >= 1 */
+    int32_t T, H, W;      /* latent video grid (frames, height, width); T*H*W < 2^31 */
+    int32_t d;            /* head dimension: 64 or 128 */
+    int32_t tile[3];      /* sliding tile extent in tokens (tT, tH, tW) */
+    int32_t window[3];    /* sliding window in TILES per axis (w_F, w_H, w_W of Algorithm 1), >= 1;
+                             an even w acts like w + 1 (the test is |c - k| <= floor(w/2)) */
+    int32_t bucket[3];    /* core-set bucket (t, h, w); {0,0,0} selects the paper's (2, 3, 2) */
+    float coreset_ratio;  /* r_core in (0, 1]: a bucket of n tokens keeps max(1, floor(r*n + 1/2)) */
+    float softmax_scale;  /* multiplies QK^T; 0 selects 1/sqrt(d) */
+    const uint8_t *routes;/* host, [heads]: branch of each head (same for every batch entry) */
+    int32_t flags;        /* 0 or VORTA_PLAN_HOST_ONLY */
+    int32_t device;       /* CUDA device ordinal; -1 = the calling thread's current device */
+} vorta_plan_desc;
+
+typedef struct {
+    int64_t L;                   /* tokens per head */
+    int64_t Lc;                  /* core-set tokens per head (geometry only, data independent) */
+    int32_t tiles_per_axis[3];   /* ceil(dim / tile) */
+    int32_t n_tiles;
+    int32_t n_buckets;
+    int32_t kv_tiles_per_q_tile; /* prod_a min(tiles_a, 2*floor(w_a/2) + 1) */
+    int32_t n_full, n_sliding, n_coreset; /* heads per branch under the current routes */
+    int64_t workspace_bytes;     /* device workspace vorta_routed_attention needs (current routes) */
+    int64_t workspace_bytes_max; /* ... if every head were routed to core-set */
+    int64_t host_call_scratch_bytes; /* device scratch vorta_routed_attention_host needs */
+    /* Algorithmic work: 4*d*(query, key) pairs the method itself attends, per (batch, head). */
+    double flops_full_head;      /* 4 d L^2 */
+    double flops_sliding_head;   /* 4 d * sum over tile pairs in the window of valid tokens products */
+    double flops_coreset_head;   /* 4 d Lc^2 */
+    double flops_layer;          /* B * sum over heads, current routes */
+    double flops_issued_layer;   /* what the tensor cores are really given (padding to 128-row blocks
+                                    and partial tiles included); 0 for a host-only plan */
+    int64_t n_work_items;        /* (head, query block) items in one launch; 0 for a host-only plan */
+    /* Algorithmic bytes of the memory-bound stages, per core-set (batch, head). */
+    int64_t select_bytes_head;   /* L*dx*2 read + (Lc + L)*4 written, with dx = d */
+    int64_t gather_bytes_head;   /* 3 * Lc*d*2 read and written */
+    int64_t scatter_bytes_head;  /* Lc*d*2 read + L*d*2 written */
+} vorta_plan_info_t;
+
+/*
+ * Build a plan for one layer shape: tile grid, window, buckets, core-set offsets,
+ * the block-sparse sliding-tile mask (Algorithm 1, evaluated between tiles by a
+ * CUDA kernel) and the ordered work list of the persistent attention kernel.
+ * Reads desc and desc->routes (host) during the call only.  *out receives the
+ * plan; free it with vorta_plan_destroy.
+ * Unsupported (VORTA_ERR_UNSUPPORTED): d not in {64,128}; a tile with more than
+ * 256 tokens, or with more than 128 tokens and an odd tT; a tile extent > 256;
+ * a bucket with more than 32 tokens.
+ */
+VORTA_API int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out);
+
+/* Replace the per-head routes (Section 3.3: the router decides per diffusion
+ * timestep) and rebuild the work list; geometry tables are kept.  routes_host is
+ * [n] with n == heads.  Synchronises with the plan's device. */
+VORTA_API int vorta_plan_set_routes(vorta_plan *plan, const uint8_t *routes_host, int32_t n);
+
+VORTA_API int vorta_plan_destroy(vorta_plan *plan);
+
+VORTA_API int vorta_plan_info(const vorta_plan *plan, vorta_plan_info_t *out);
+
+/*
+ * Copy the canonical block mask to host memory: out_host is uint8
+ * [n_tiles * n_tiles], BM[qt*n_tiles + kt] = 1 iff key tile kt lies in the window
+ * of query tile qt (Algorithm 1 applied to tile ids, the query tile first moved
+ * to its window-centre tile), with tile id = (tile_T*nt_H + tile_H)*nt_W + tile_W.
+ * Not available on a host-only plan.
+ */
+VORTA_API int vorta_plan_block_mask(const vorta_plan *plan, uint8_t *out_host);
+
+/* Select the attention kernel (VORTA_KERNEL_*).  Default VORTA_KERNEL_TCGEN05. */
+VORTA_API int vorta_plan_set_kernel(vorta_plan *plan, int32_t kernel);
+
+/*
+ * Bucketed core-set selection (Section 3.2; Appendix A.1): for every (b, hx)
+ * slice of X and every bucket, score each token by its cosine similarity to the
+ * bucket's centre token, prune the n - keep(n) most similar (ties: lower local
+ * index first), keep the rest.
+ *   X_dev        bf16 [B, Hx, L, dx], dx a multiple of 8, Hx >= 1
+ *   core_idx_dev int32 [B, Hx, Lc] out: kept token ids, buckets in raster order, in
+ *                each bucket the centre first, then the other kept tokens ascending
+ *   src_slot_dev int32 [B, Hx, L]  out: position in core_idx of the token whose
+ *                attention output each token receives (its own, or its centre's)
+ * Scores are evaluated in fp64 on the device.
+ */
+VORTA_API int vorta_coreset_select(const vorta_plan *plan, const void *X_dev, int32_t Hx, int32_t dx,
+                                   int32_t *core_idx_dev, int32_t *src_slot_dev, void *stream);
+
+/*
+ * One layer of routed attention: O[b, h] = branch_{routes[h]}(Q[b, h], K[b, h], V[b, h]).
+ * Core-set heads: select on X (NULL = on K of that head; else bf16
+ * [B, Hx, L, d] with Hx == 1, shared by all heads, or Hx == heads), gather the
+ * kept rows of Q, K, V, attend, scatter back (Section 3.2, last paragraph).
+ * Sliding heads: Algorithm 1's mask, only the listed tile pairs are computed.
+ *   Q, K, V      device bf16 [B, heads, L, d], 16-byte aligned
+ *   O            device bf16 [B, heads, L, d] out; every element is written
+ *   workspace    device, >= vorta_plan_info().workspace_bytes, 256-byte aligned
+ *                (may be NULL when no head is routed to core-set); contents are
+ *                scratch and undefined afterwards
+ * Launch order on `stream`: select, gather, attention, scatter.
+ */
+VORTA_API int vorta_routed_attention(const vorta_plan *plan, const void *Q, const void *K,
+                                     const void *V, void *O, const void *X_or_null, int32_t Hx,
+                                     void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * The same layer with HOST buffers (bf16 [B, heads, L, d], ideally pinned):
+ * copies Q, K, V to dev_scratch, runs vorta_routed_attention there, copies O
+ * back, all on `stream`; returns after enqueueing (synchronise the stream before
+ * reading O_host).  dev_scratch: device memory of at least
+ * vorta_plan_info().host_call_scratch_bytes, 256-byte aligned.
+ */
+VORTA_API int vorta_routed_attention_host(const vorta_plan *plan, const void *Q_host,
+                                          const void *K_host, const void *V_host, void *O_host,
+                                          void *dev_scratch, size_t dev_scratch_bytes, void *stream);
+
+/*
+ * Stage timing.  With profiling on, vorta_routed_attention records CUDA events
+ * on its stream around its four stages.  After the stream has been synchronised,
+ * vorta_plan_stage_ms returns the last call's durations in milliseconds:
+ * ms[0] select, ms[1] gather, ms[2] attention, ms[3] scatter (0 if a stage did not run).
+ */
+VORTA_API int vorta_plan_set_profiling(vorta_plan *plan, int32_t on);
+VORTA_API int vorta_plan_stage_ms(const vorta_plan *plan, float ms[4]);
+
+/* Number of kernels the last vorta_routed_attention call launched. */
+VORTA_API int vorta_plan_last_launches(const vorta_plan *plan, int32_t *n);
+
+/*
+ * Synchronise `stream` and report whether a kernel of this plan gave up on a
+ * bounded wait: *code_out = 0 if none did, else a non-zero location code.
+ * Returns VORTA_ERR_TIMEOUT in that case and clears the code.
+ */
+VORTA_API int vorta_device_status(const vorta_plan *plan, void *stream, int32_t *code_out);
+
+VORTA_API const char *vorta_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VORTA_H_ */

@@ -1,0 +1,693 @@
+// Host side of libvorta: argument checking, geometry, work lists, tensor maps and
+// the C entry points declared in vorta.h.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <functional>
+#include <new>
+#include <queue>
+
+#include "vorta_internal.h"
+
+using namespace vorta;
+
+struct vorta_plan {
+    Geometry g{};
+    float scale = 0.f;
+    bool host_only = false;
+    int device = 0;
+    int sm_count = 0;
+    std::vector<uint8_t> routes;
+    std::vector<int32_t> seg_start;   // per bucket: first slot of its core_idx segment
+    std::vector<int32_t> kv_count;    // per query tile (read back from the device)
+    std::vector<int32_t> core_heads;  // heads routed to core-set, ascending
+    // device tables
+    uint8_t *d_bm = nullptr;
+    KvEntry *d_kv_list = nullptr;
+    int32_t *d_kv_count = nullptr;
+    uint32_t *d_colmasks = nullptr;
+    int32_t *d_seg_start = nullptr;
+    WorkItem *d_items = nullptr;
+    int32_t *d_cta_begin = nullptr, *d_cta_count = nullptr;
+    int32_t *d_core_slice = nullptr;  // [B * n_core]: compact problem -> b*heads + head
+    int32_t *d_core_xslice = nullptr; // same for a shared X with one head
+    int32_t *d_status = nullptr;
+    int32_t n_items = 0;
+    int64_t items_cap = 0;
+    double flops_issued = 0.0;
+    double sliding_pairs = 0.0;  // sum over listed tile pairs of valid-token products
+    int32_t kernel = VORTA_KERNEL_TCGEN05;
+    // profiling
+    mutable cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+    mutable bool ev_valid[5] = {false, false, false, false, false};
+    bool profiling = false;
+    mutable int32_t last_launches = 0;
+};
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (fn) return fn;
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+        return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+    return fn;
+}
+
+// 5-D bf16 map (d, n1, n2, n3, slices) over a contiguous [slices, n3, n2, n1, d]
+// tensor with a (64, b1, b2, b3, 1) box and the 128-byte swizzle.
+bool make_map(CUtensorMap *m, const void *base, int32_t d, int64_t n1, int64_t n2, int64_t n3,
+              int64_t slices, int32_t b1, int32_t b2, int32_t b3)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[5] = {(cuuint64_t)d, (cuuint64_t)n1, (cuuint64_t)n2, (cuuint64_t)n3,
+                          (cuuint64_t)slices};
+    cuuint64_t row = (cuuint64_t)d * 2;
+    cuuint64_t strides[4] = {row, row * n1, row * n1 * n2, row * n1 * n2 * n3};
+    cuuint32_t box[5] = {64, (cuuint32_t)b1, (cuuint32_t)b2, (cuuint32_t)b3, 1};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(base), dims, strides,
+                    box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+int64_t keep_count(int64_t n, double r)
+{
+    int64_t k = (int64_t)std::floor(r * (double)n + 0.5);
+    return k < 1 ? 1 : k;
+}
+
+inline int64_t align_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
+
+// Workspace layout for n_prob = B * n_core compact problems.
+struct Workspace {
+    int64_t core_idx, src_slot, Qc, Kc, Vc, Oc, total;
+};
+Workspace workspace_layout(const Geometry &g, int64_t n_prob)
+{
+    Workspace w{};
+    int64_t off = 0;
+    w.core_idx = off; off = align_up(off + n_prob * g.Lc * 4, 256);
+    w.src_slot = off; off = align_up(off + n_prob * g.L * 4, 256);
+    int64_t rows = align_up(n_prob * (int64_t)g.Lc * g.d * 2, 256);
+    w.Qc = off; off += rows;
+    w.Kc = off; off += rows;
+    w.Vc = off; off += rows;
+    w.Oc = off; off += rows;
+    w.total = n_prob ? off : 0;
+    return w;
+}
+
+int64_t tensor_bytes(const Geometry &g) { return (int64_t)g.B * g.heads * g.L * g.d * 2; }
+
+void free_device(vorta_plan *p)
+{
+    cudaFree(p->d_bm); cudaFree(p->d_kv_list); cudaFree(p->d_kv_count); cudaFree(p->d_colmasks);
+    cudaFree(p->d_seg_start); cudaFree(p->d_items); cudaFree(p->d_cta_begin);
+    cudaFree(p->d_cta_count); cudaFree(p->d_core_slice); cudaFree(p->d_core_xslice);
+    cudaFree(p->d_status);
+    for (auto &e : p->ev)
+        if (e) cudaEventDestroy(e);
+}
+
+// valid tokens of tile `id` on axis a
+inline int32_t tile_valid(const Geometry &g, int a, int32_t id)
+{
+    const int32_t dim[3] = {g.T, g.H, g.W};
+    return std::min(g.tile[a], dim[a] - id * g.tile[a]);
+}
+
+// sum over (query tile, key tile in its window) of valid(q) * valid(k); separable per axis
+double sliding_valid_pairs(const Geometry &g)
+{
+    double total = 1.0;
+    for (int a = 0; a < 3; ++a) {
+        double s = 0.0;
+        for (int32_t q = 0; q < g.nt[a]; ++q) {
+            int32_t lo = 0, hi = g.nt[a] - 1;
+            if (g.restricted[a]) {
+                int32_t c = std::min(std::max(q, g.half[a]), g.nt[a] - 1 - g.half[a]);
+                lo = c - g.half[a];
+                hi = c + g.half[a];
+            }
+            double keys = 0.0;
+            for (int32_t k = lo; k <= hi; ++k) keys += tile_valid(g, a, k);
+            s += (double)tile_valid(g, a, q) * keys;
+        }
+        total *= s;
+    }
+    return total;
+}
+
+// (Re)build the ordered work list for the current routes and upload it.
+int build_work(vorta_plan *p)
+{
+    const Geometry &g = p->g;
+    p->core_heads.clear();
+    for (int32_t h = 0; h < g.heads; ++h)
+        if (p->routes[h] == VORTA_ROUTE_CORESET) p->core_heads.push_back(h);
+    if (p->host_only) return VORTA_OK;
+
+    const int32_t n_core = (int32_t)p->core_heads.size();
+    std::vector<WorkItem> items;
+    std::vector<double> cost;
+    auto linear_items = [&](int32_t mode, int32_t slice, int32_t len) {
+        int32_t nblk = (len + kBlockM - 1) / kBlockM;
+        int32_t kv = nblk;
+        for (int32_t b0 = 0; b0 < nblk; b0 += 2) {
+            WorkItem w{};
+            w.mode = mode; w.slice = slice; w.kv_count = kv; w.kv_len = len;
+            w.n_mblk = std::min(2, nblk - b0);
+            for (int m = 0; m < w.n_mblk; ++m) w.q_org[m][0] = (b0 + m) * kBlockM;
+            items.push_back(w);
+            cost.push_back((double)w.n_mblk * kv + 2.0);
+        }
+    };
+    for (int32_t b = 0; b < g.B; ++b) {
+        for (int32_t h = 0; h < g.heads; ++h) {
+            int32_t slice = b * g.heads + h;
+            switch (p->routes[h]) {
+            case VORTA_ROUTE_FULL:
+                linear_items(MODE_LINEAR, slice, g.L);
+                break;
+            case VORTA_ROUTE_SLIDING:
+                for (int32_t qt = 0; qt < g.n_tiles; ++qt) {
+                    int32_t q[3] = {qt / (g.nt[2] * g.nt[1]), (qt / g.nt[2]) % g.nt[1], qt % g.nt[2]};
+                    WorkItem w{};
+                    w.mode = MODE_TILES; w.slice = slice;
+                    w.kv_count = p->kv_count[qt];
+                    w.kv_begin = qt * g.max_kv_per_tile;
+                    w.kv_len = 0;
+                    int32_t t0 = q[0] * g.tile[0];
+                    for (int32_t bx = 0; bx < g.boxes_per_tile; ++bx) {
+                        if (t0 + bx * g.box[0] >= g.T) break;
+                        w.q_org[bx][0] = q[2] * g.tile[2];
+                        w.q_org[bx][1] = q[1] * g.tile[1];
+                        w.q_org[bx][2] = t0 + bx * g.box[0];
+                        w.n_mblk = bx + 1;
+                    }
+                    items.push_back(w);
+                    cost.push_back((double)w.n_mblk * w.kv_count * g.bn_tile / 128.0 + 2.0);
+                }
+                break;
+            default: {
+                int32_t k = (int32_t)(std::find(p->core_heads.begin(), p->core_heads.end(), h) -
+                                      p->core_heads.begin());
+                linear_items(MODE_COMPACT, b * n_core + k, g.Lc);
+                break;
+            }
+            }
+        }
+    }
+    // issued tensor-core work: every block is a 128 x bn QK^T and a 128 x d PV
+    double issued = 0.0;
+    for (auto &w : items) {
+        double bn = w.mode == MODE_TILES ? g.bn_tile : 128;
+        issued += (double)w.n_mblk * w.kv_count * 4.0 * kBlockM * bn * g.d;
+    }
+    p->flops_issued = issued;
+
+    // longest-processing-time assignment of items to the persistent CTAs
+    const int32_t grid = p->sm_count;
+    std::vector<int32_t> order(items.size());
+    for (size_t i = 0; i < order.size(); ++i) order[i] = (int32_t)i;
+    std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return cost[a] > cost[b]; });
+    typedef std::pair<double, int32_t> Load;
+    std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
+    for (int32_t c = 0; c < grid; ++c) heap.push(Load(0.0, c));
+    std::vector<std::vector<int32_t>> per_cta(grid);
+    for (int32_t i : order) {
+        Load l = heap.top();
+        heap.pop();
+        per_cta[l.second].push_back(i);
+        heap.push(Load(l.first + cost[i], l.second));
+    }
+    std::vector<WorkItem> sorted;
+    sorted.reserve(items.size());
+    std::vector<int32_t> begin(grid), count(grid);
+    for (int32_t c = 0; c < grid; ++c) {
+        begin[c] = (int32_t)sorted.size();
+        count[c] = (int32_t)per_cta[c].size();
+        for (int32_t i : per_cta[c]) sorted.push_back(items[i]);
+    }
+    p->n_items = (int32_t)sorted.size();
+
+    if ((int64_t)sorted.size() > p->items_cap) {
+        cudaFree(p->d_items);
+        p->d_items = nullptr;
+        p->items_cap = (int64_t)sorted.size();
+        if (cudaMalloc(&p->d_items, sizeof(WorkItem) * std::max<size_t>(sorted.size(), 1)) != cudaSuccess)
+            return VORTA_ERR_CUDA;
+    }
+    std::vector<int32_t> core_slice((size_t)g.B * std::max(n_core, 1)), core_x(core_slice.size());
+    for (int32_t b = 0; b < g.B; ++b)
+        for (int32_t k = 0; k < n_core; ++k) {
+            core_slice[(size_t)b * n_core + k] = b * g.heads + p->core_heads[k];
+            core_x[(size_t)b * n_core + k] = b;
+        }
+    // synchronous copies: the caller may change routes between steps
+    if (!sorted.empty() &&
+        cudaMemcpy(p->d_items, sorted.data(), sizeof(WorkItem) * sorted.size(), cudaMemcpyHostToDevice) != cudaSuccess)
+        return VORTA_ERR_CUDA;
+    if (cudaMemcpy(p->d_cta_begin, begin.data(), sizeof(int32_t) * grid, cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(p->d_cta_count, count.data(), sizeof(int32_t) * grid, cudaMemcpyHostToDevice) != cudaSuccess)
+        return VORTA_ERR_CUDA;
+    if (n_core &&
+        (cudaMemcpy(p->d_core_slice, core_slice.data(), sizeof(int32_t) * g.B * n_core, cudaMemcpyHostToDevice) != cudaSuccess ||
+         cudaMemcpy(p->d_core_xslice, core_x.data(), sizeof(int32_t) * g.B * n_core, cudaMemcpyHostToDevice) != cudaSuccess))
+        return VORTA_ERR_CUDA;
+    return VORTA_OK;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+        changed = ok && prev != dev;
+    }
+    ~DeviceGuard() { if (changed) cudaSetDevice(prev); }
+    bool changed = false;
+};
+
+bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------
+extern "C" {
+
+const char *vorta_status_string(int s)
+{
+    switch (s) {
+    case VORTA_OK: return "ok";
+    case VORTA_ERR_INVALID_ARG: return "invalid argument";
+    case VORTA_ERR_UNSUPPORTED: return "unsupported configuration";
+    case VORTA_ERR_ALIGNMENT: return "misaligned pointer";
+    case VORTA_ERR_WORKSPACE: return "workspace missing or too small";
+    case VORTA_ERR_CUDA: return "CUDA call failed";
+    case VORTA_ERR_TIMEOUT: return "bounded device-side wait expired";
+    case VORTA_ERR_INTERNAL: return "internal self-check failed";
+    default: return "unknown status";
+    }
+}
+
+int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
+{
+    if (!desc || !out) return VORTA_ERR_INVALID_ARG;
+    *out = nullptr;
+    const vorta_plan_desc &D = *desc;
+    if (!D.routes || D.B < 1 || D.heads < 1 || D.T < 1 || D.H < 1 || D.W < 1) return VORTA_ERR_INVALID_ARG;
+    if (D.T > 32767 || D.H > 32767 || D.W > 32767) return VORTA_ERR_INVALID_ARG;
+    int64_t L64 = (int64_t)D.T * D.H * D.W;
+    if (L64 >= (int64_t)1 << 31) return VORTA_ERR_INVALID_ARG;
+    if ((int64_t)D.B * D.heads > 65535) return VORTA_ERR_INVALID_ARG;
+    if (!(D.coreset_ratio > 0.f) || !(D.coreset_ratio <= 1.f)) return VORTA_ERR_INVALID_ARG;
+    if (!(D.softmax_scale >= 0.f) || !std::isfinite(D.softmax_scale)) return VORTA_ERR_INVALID_ARG;
+    if (D.flags & ~VORTA_PLAN_HOST_ONLY) return VORTA_ERR_INVALID_ARG;
+    int32_t bucket[3] = {D.bucket[0], D.bucket[1], D.bucket[2]};
+    if (bucket[0] == 0 && bucket[1] == 0 && bucket[2] == 0) { bucket[0] = 2; bucket[1] = 3; bucket[2] = 2; }
+    for (int a = 0; a < 3; ++a)
+        if (D.tile[a] < 1 || D.window[a] < 1 || bucket[a] < 1) return VORTA_ERR_INVALID_ARG;
+    for (int32_t h = 0; h < D.heads; ++h)
+        if (D.routes[h] > VORTA_ROUTE_CORESET) return VORTA_ERR_INVALID_ARG;
+    if (D.d != 64 && D.d != 128) return VORTA_ERR_UNSUPPORTED;
+    int64_t tile_tokens = (int64_t)D.tile[0] * D.tile[1] * D.tile[2];
+    if (D.tile[0] > 256 || D.tile[1] > 256 || D.tile[2] > 256 || tile_tokens > 256) return VORTA_ERR_UNSUPPORTED;
+    if (tile_tokens > 128 && (D.tile[0] % 2) != 0) return VORTA_ERR_UNSUPPORTED;
+    if ((int64_t)bucket[0] * bucket[1] * bucket[2] > 32) return VORTA_ERR_UNSUPPORTED;
+
+    vorta_plan *p = new (std::nothrow) vorta_plan();
+    if (!p) return VORTA_ERR_INTERNAL;
+    Geometry &g = p->g;
+    g.B = D.B; g.heads = D.heads; g.T = D.T; g.H = D.H; g.W = D.W; g.L = (int32_t)L64; g.d = D.d;
+    const int32_t dim[3] = {D.T, D.H, D.W};
+    g.n_tiles = 1; g.n_buckets = 1;
+    for (int a = 0; a < 3; ++a) {
+        g.tile[a] = D.tile[a];
+        g.nt[a] = (dim[a] + D.tile[a] - 1) / D.tile[a];
+        g.half[a] = D.window[a] / 2;
+        g.restricted[a] = g.nt[a] > 2 * g.half[a] + 1;
+        g.bucket[a] = bucket[a];
+        g.nb[a] = (dim[a] + bucket[a] - 1) / bucket[a];
+        g.n_tiles *= g.nt[a];
+        g.n_buckets *= g.nb[a];
+    }
+    g.ratio = (double)D.coreset_ratio;
+    p->scale = D.softmax_scale > 0.f ? D.softmax_scale : 1.0f / std::sqrt((float)D.d);
+    p->host_only = (D.flags & VORTA_PLAN_HOST_ONLY) != 0;
+    p->routes.assign(D.routes, D.routes + D.heads);
+
+    // core-set segments: prefix sum of keep(n) over the buckets in raster order
+    p->seg_start.resize(g.n_buckets);
+    int64_t Lc = 0;
+    for (int32_t b = 0; b < g.n_buckets; ++b) {
+        int32_t id[3] = {b / (g.nb[2] * g.nb[1]), (b / g.nb[2]) % g.nb[1], b % g.nb[2]};
+        int64_t n = 1;
+        for (int a = 0; a < 3; ++a) n *= std::min(g.bucket[a], dim[a] - g.bucket[a] * id[a]);
+        p->seg_start[b] = (int32_t)Lc;
+        Lc += keep_count(n, g.ratio);
+    }
+    g.Lc = (int32_t)Lc;
+
+    // sliding branch blocking
+    g.boxes_per_tile = tile_tokens > 128 ? 2 : 1;
+    g.box[0] = g.tile[0] / g.boxes_per_tile; g.box[1] = g.tile[1]; g.box[2] = g.tile[2];
+    g.box_rows = g.box[0] * g.box[1] * g.box[2];
+    g.bn_tile = (g.box_rows + 15) / 16 * 16;
+    int32_t kv_tiles = 1;
+    for (int a = 0; a < 3; ++a) kv_tiles *= std::min(g.nt[a], 2 * g.half[a] + 1);
+    g.max_kv_per_tile = kv_tiles * g.boxes_per_tile;
+    p->sliding_pairs = sliding_valid_pairs(g);
+
+    if (p->host_only) {
+        int rc = build_work(p);
+        if (rc != VORTA_OK) { delete p; return rc; }
+        *out = p;
+        return VORTA_OK;
+    }
+
+    // ---- device side ----
+    int dev = D.device;
+    if (dev < 0 && cudaGetDevice(&dev) != cudaSuccess) { delete p; return VORTA_ERR_CUDA; }
+    p->device = dev;
+    DeviceGuard guard(dev);
+    cudaDeviceProp prop;
+    if (!guard.ok || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) { delete p; return VORTA_ERR_CUDA; }
+    if (prop.major != 10) { delete p; return VORTA_ERR_UNSUPPORTED; }
+    p->sm_count = prop.multiProcessorCount;
+
+    // column masks of the sliding branch: class -> valid columns of a KV box
+    std::vector<uint32_t> masks((size_t)kMaxMasks * 4, 0u);
+    for (int32_t id = 1; id < kMaxMasks; ++id) {
+        int32_t c = id - 1, bx = c & 1, pw = (c >> 1) & 1, ph = (c >> 2) & 1, pt = (c >> 3) & 1;
+        if (bx >= g.boxes_per_tile) continue;
+        int32_t et = pt ? dim[0] - (g.nt[0] - 1) * g.tile[0] : g.tile[0];
+        int32_t vt = std::min(std::max(et - bx * g.box[0], 0), g.box[0]);
+        int32_t vh = ph ? dim[1] - (g.nt[1] - 1) * g.tile[1] : g.tile[1];
+        int32_t vw = pw ? dim[2] - (g.nt[2] - 1) * g.tile[2] : g.tile[2];
+        for (int32_t r = 0; r < g.box_rows; ++r) {
+            int32_t lw = r % g.box[2], lh = (r / g.box[2]) % g.box[1], lt = r / (g.box[2] * g.box[1]);
+            if (lw < vw && lh < vh && lt < vt) masks[(size_t)id * 4 + r / 32] |= 1u << (r % 32);
+        }
+    }
+
+    bool ok = true;
+    int64_t nt2 = (int64_t)g.n_tiles * g.n_tiles;
+    ok = ok && cudaMalloc(&p->d_bm, (size_t)nt2) == cudaSuccess;
+    ok = ok && cudaMalloc(&p->d_kv_list, sizeof(KvEntry) * (size_t)g.n_tiles * g.max_kv_per_tile) == cudaSuccess;
+    ok = ok && cudaMalloc(&p->d_kv_count, sizeof(int32_t) * g.n_tiles) == cudaSuccess;
+    ok = ok && cudaMalloc(&p->d_colmasks, sizeof(uint32_t) * masks.size()) == cudaSuccess;
+    ok = ok && cudaMalloc(&p->d_seg_start, sizeof(int32_t) * g.n_buckets) == cudaSuccess;
+    ok = ok && cudaMalloc(&p->d_cta_begin, sizeof(int32_t) * p->sm_count) == cudaSuccess;
+    ok = ok && cudaMalloc(&p->d_cta_count, sizeof(int32_t) * p->sm_count) == cudaSuccess;
+    ok = ok && cudaMalloc(&p->d_core_slice, sizeof(int32_t) * (size_t)g.B * g.heads) == cudaSuccess;
+    ok = ok && cudaMalloc(&p->d_core_xslice, sizeof(int32_t) * (size_t)g.B * g.heads) == cudaSuccess;
+    ok = ok && cudaMalloc(&p->d_status, sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMemset(p->d_status, 0, sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMemcpy(p->d_colmasks, masks.data(), sizeof(uint32_t) * masks.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemcpy(p->d_seg_start, p->seg_start.data(), sizeof(int32_t) * g.n_buckets, cudaMemcpyHostToDevice) == cudaSuccess;
+    for (auto &e : p->ev) ok = ok && cudaEventCreate(&e) == cudaSuccess;
+    // the mask builder runs once per shape; its per-tile counts come back for the work list
+    ok = ok && launch_block_mask(g, p->d_bm, p->d_kv_list, p->d_kv_count, nullptr) == cudaSuccess;
+    p->kv_count.resize(g.n_tiles);
+    ok = ok && cudaMemcpy(p->kv_count.data(), p->d_kv_count, sizeof(int32_t) * g.n_tiles, cudaMemcpyDeviceToHost) == cudaSuccess;
+    ok = ok && attention_sm100_prepare() == cudaSuccess;
+    if (!ok) { cudaGetLastError(); free_device(p); delete p; return VORTA_ERR_CUDA; }
+    // self-check: the lists must hold exactly the blocks the window arithmetic predicts
+    for (int32_t qt = 0; qt < g.n_tiles; ++qt)
+        if (p->kv_count[qt] < 1 || p->kv_count[qt] > g.max_kv_per_tile) { free_device(p); delete p; return VORTA_ERR_INTERNAL; }
+    int rc = build_work(p);
+    if (rc != VORTA_OK) { free_device(p); delete p; return rc; }
+    *out = p;
+    return VORTA_OK;
+}
+
+int vorta_plan_set_routes(vorta_plan *p, const uint8_t *routes, int32_t n)
+{
+    if (!p || !routes || n != p->g.heads) return VORTA_ERR_INVALID_ARG;
+    for (int32_t h = 0; h < n; ++h)
+        if (routes[h] > VORTA_ROUTE_CORESET) return VORTA_ERR_INVALID_ARG;
+    p->routes.assign(routes, routes + n);
+    if (p->host_only) return build_work(p);
+    DeviceGuard guard(p->device);
+    if (!guard.ok || cudaDeviceSynchronize() != cudaSuccess) return VORTA_ERR_CUDA;
+    return build_work(p);
+}
+
+int vorta_plan_destroy(vorta_plan *p)
+{
+    if (!p) return VORTA_ERR_INVALID_ARG;
+    if (!p->host_only) {
+        DeviceGuard guard(p->device);
+        cudaDeviceSynchronize();
+        free_device(p);
+    }
+    delete p;
+    return VORTA_OK;
+}
+
+int vorta_plan_info(const vorta_plan *p, vorta_plan_info_t *o)
+{
+    if (!p || !o) return VORTA_ERR_INVALID_ARG;
+    const Geometry &g = p->g;
+    std::memset(o, 0, sizeof(*o));
+    o->L = g.L; o->Lc = g.Lc;
+    for (int a = 0; a < 3; ++a) o->tiles_per_axis[a] = g.nt[a];
+    o->n_tiles = g.n_tiles; o->n_buckets = g.n_buckets;
+    o->kv_tiles_per_q_tile = g.max_kv_per_tile / g.boxes_per_tile;
+    for (uint8_t r : p->routes) {
+        if (r == VORTA_ROUTE_FULL) ++o->n_full;
+        else if (r == VORTA_ROUTE_SLIDING) ++o->n_sliding;
+        else ++o->n_coreset;
+    }
+    o->workspace_bytes = workspace_layout(g, (int64_t)g.B * o->n_coreset).total;
+    o->workspace_bytes_max = workspace_layout(g, (int64_t)g.B * g.heads).total;
+    o->host_call_scratch_bytes = 4 * align_up(tensor_bytes(g), 256) + o->workspace_bytes;
+    o->flops_full_head = 4.0 * g.d * (double)g.L * (double)g.L;
+    o->flops_sliding_head = 4.0 * g.d * p->sliding_pairs;
+    o->flops_coreset_head = 4.0 * g.d * (double)g.Lc * (double)g.Lc;
+    o->flops_layer = g.B * (o->n_full * o->flops_full_head + o->n_sliding * o->flops_sliding_head +
+                            o->n_coreset * o->flops_coreset_head);
+    o->flops_issued_layer = p->host_only ? 0.0 : p->flops_issued;
+    o->n_work_items = p->host_only ? 0 : p->n_items;
+    o->select_bytes_head = (int64_t)g.L * g.d * 2 + ((int64_t)g.Lc + g.L) * 4;
+    o->gather_bytes_head = 3 * 2 * (int64_t)g.Lc * g.d * 2;
+    o->scatter_bytes_head = ((int64_t)g.Lc + g.L) * g.d * 2;
+    return VORTA_OK;
+}
+
+int vorta_plan_block_mask(const vorta_plan *p, uint8_t *out_host)
+{
+    if (!p || !out_host) return VORTA_ERR_INVALID_ARG;
+    if (p->host_only) return VORTA_ERR_UNSUPPORTED;
+    DeviceGuard guard(p->device);
+    if (!guard.ok) return VORTA_ERR_CUDA;
+    size_t n = (size_t)p->g.n_tiles * p->g.n_tiles;
+    return cudaMemcpy(out_host, p->d_bm, n, cudaMemcpyDeviceToHost) == cudaSuccess ? VORTA_OK : VORTA_ERR_CUDA;
+}
+
+int vorta_plan_set_kernel(vorta_plan *p, int32_t kernel)
+{
+    if (!p || (kernel != VORTA_KERNEL_TCGEN05 && kernel != VORTA_KERNEL_SIMT)) return VORTA_ERR_INVALID_ARG;
+    p->kernel = kernel;
+    return VORTA_OK;
+}
+
+int vorta_plan_set_profiling(vorta_plan *p, int32_t on)
+{
+    if (!p) return VORTA_ERR_INVALID_ARG;
+    p->profiling = on != 0;
+    return VORTA_OK;
+}
+
+int vorta_plan_stage_ms(const vorta_plan *p, float ms[4])
+{
+    if (!p || !ms) return VORTA_ERR_INVALID_ARG;
+    if (p->host_only) return VORTA_ERR_UNSUPPORTED;
+    for (int i = 0; i < 4; ++i) {
+        ms[i] = 0.f;
+        if (p->ev_valid[i] && p->ev_valid[i + 1] &&
+            cudaEventElapsedTime(&ms[i], p->ev[i], p->ev[i + 1]) != cudaSuccess) {
+            cudaGetLastError();
+            return VORTA_ERR_CUDA;
+        }
+    }
+    return VORTA_OK;
+}
+
+int vorta_plan_last_launches(const vorta_plan *p, int32_t *n)
+{
+    if (!p || !n) return VORTA_ERR_INVALID_ARG;
+    *n = p->last_launches;
+    return VORTA_OK;
+}
+
+int vorta_coreset_select(const vorta_plan *p, const void *X, int32_t Hx, int32_t dx, int32_t *core_idx,
+                         int32_t *src_slot, void *stream)
+{
+    if (!p || !X || !core_idx || !src_slot || Hx < 1 || dx < 8 || (dx % 8) != 0) return VORTA_ERR_INVALID_ARG;
+    if (p->host_only) return VORTA_ERR_UNSUPPORTED;
+    if (!aligned(X, 16) || !aligned(core_idx, 4) || !aligned(src_slot, 4)) return VORTA_ERR_ALIGNMENT;
+    DeviceGuard guard(p->device);
+    if (!guard.ok) return VORTA_ERR_CUDA;
+    cudaError_t e = launch_select(p->g, static_cast<const __nv_bfloat16 *>(X), dx, p->g.B * Hx, nullptr,
+                                  p->d_seg_start, core_idx, src_slot, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? VORTA_OK : VORTA_ERR_CUDA;
+}
+
+int vorta_routed_attention(const vorta_plan *p, const void *Q, const void *K, const void *V, void *O,
+                           const void *X, int32_t Hx, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!p || !Q || !K || !V || !O) return VORTA_ERR_INVALID_ARG;
+    if (p->host_only) return VORTA_ERR_UNSUPPORTED;
+    const Geometry &g = p->g;
+    if (X && Hx != 1 && Hx != g.heads) return VORTA_ERR_INVALID_ARG;
+    if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) || (X && !aligned(X, 16)))
+        return VORTA_ERR_ALIGNMENT;
+    const int32_t n_core = (int32_t)p->core_heads.size();
+    const int32_t n_prob = g.B * n_core;
+    Workspace ws = workspace_layout(g, n_prob);
+    if (n_prob > 0) {
+        if (!workspace || (int64_t)workspace_bytes < ws.total) return VORTA_ERR_WORKSPACE;
+        if (!aligned(workspace, 256)) return VORTA_ERR_ALIGNMENT;
+    }
+    DeviceGuard guard(p->device);
+    if (!guard.ok) return VORTA_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    char *wsb = static_cast<char *>(workspace);
+    int32_t *core_idx = n_prob ? reinterpret_cast<int32_t *>(wsb + ws.core_idx) : nullptr;
+    int32_t *src_slot = n_prob ? reinterpret_cast<int32_t *>(wsb + ws.src_slot) : nullptr;
+    __nv_bfloat16 *Qc = n_prob ? reinterpret_cast<__nv_bfloat16 *>(wsb + ws.Qc) : nullptr;
+    __nv_bfloat16 *Kc = n_prob ? reinterpret_cast<__nv_bfloat16 *>(wsb + ws.Kc) : nullptr;
+    __nv_bfloat16 *Vc = n_prob ? reinterpret_cast<__nv_bfloat16 *>(wsb + ws.Vc) : nullptr;
+    __nv_bfloat16 *Oc = n_prob ? reinterpret_cast<__nv_bfloat16 *>(wsb + ws.Oc) : nullptr;
+    const __nv_bfloat16 *q = static_cast<const __nv_bfloat16 *>(Q), *k = static_cast<const __nv_bfloat16 *>(K),
+                        *v = static_cast<const __nv_bfloat16 *>(V);
+    __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(O);
+
+    AttnParams prm{};
+    prm.g = g;
+    prm.scale_log2 = p->scale * 1.4426950408889634f;
+    prm.items = p->d_items; prm.cta_begin = p->d_cta_begin; prm.cta_count = p->d_cta_count;
+    prm.kv_list = p->d_kv_list; prm.colmasks = p->d_colmasks;
+    prm.O = o; prm.Oc = Oc; prm.Q = q; prm.K = k; prm.V = v; prm.Qc = Qc; prm.Kc = Kc; prm.Vc = Vc;
+    prm.status = p->d_status;
+
+    AttnMaps maps;
+    std::memset(&maps, 0, sizeof(maps));
+    if (p->kernel == VORTA_KERNEL_TCGEN05) {
+        const int64_t BH = (int64_t)g.B * g.heads;
+        bool ok = true;
+        const void *src[3] = {q, k, v};
+        CUtensorMap *dst[3] = {maps.q, maps.k, maps.v};
+        for (int t = 0; t < 3 && ok; ++t) {
+            ok = ok && make_map(&dst[t][MODE_LINEAR], src[t], g.d, g.L, 1, 1, BH, kBlockM, 1, 1);
+            ok = ok && make_map(&dst[t][MODE_TILES], src[t], g.d, g.W, g.H, g.T, BH, g.box[2], g.box[1], g.box[0]);
+        }
+        const void *csrc[3] = {Qc, Kc, Vc};
+        for (int t = 0; t < 3 && ok; ++t) {
+            if (n_prob) ok = ok && make_map(&dst[t][MODE_COMPACT], csrc[t], g.d, g.Lc, 1, 1, n_prob, kBlockM, 1, 1);
+            else dst[t][MODE_COMPACT] = dst[t][MODE_LINEAR];
+        }
+        if (!ok) return VORTA_ERR_CUDA;
+    }
+
+    int32_t launches = 0;
+    const bool prof = p->profiling;
+    for (auto &f : p->ev_valid) f = false;
+    auto mark = [&](int i) {
+        if (prof && cudaEventRecord(p->ev[i], s) == cudaSuccess) p->ev_valid[i] = true;
+    };
+    cudaError_t e = cudaSuccess;
+    mark(0);
+    if (n_prob) {
+        const __nv_bfloat16 *xs = X ? static_cast<const __nv_bfloat16 *>(X) : k;
+        const int32_t *xslice = (X && Hx == 1) ? p->d_core_xslice : p->d_core_slice;
+        e = launch_select(g, xs, g.d, n_prob, xslice, p->d_seg_start, core_idx, src_slot, s);
+        if (e != cudaSuccess) return VORTA_ERR_CUDA;
+        ++launches;
+    }
+    mark(1);
+    if (n_prob) {
+        e = launch_gather(g, n_prob, p->d_core_slice, core_idx, q, k, v, Qc, Kc, Vc, s);
+        if (e != cudaSuccess) return VORTA_ERR_CUDA;
+        ++launches;
+    }
+    mark(2);
+    if (p->n_items > 0) {
+        e = p->kernel == VORTA_KERNEL_TCGEN05 ? launch_attention_sm100(prm, maps, p->sm_count, s)
+                                              : launch_attention_simt(prm, p->n_items, s);
+        if (e != cudaSuccess) return VORTA_ERR_CUDA;
+        ++launches;
+    }
+    mark(3);
+    if (n_prob) {
+        e = launch_scatter(g, n_prob, p->d_core_slice, src_slot, Oc, o, s);
+        if (e != cudaSuccess) return VORTA_ERR_CUDA;
+        ++launches;
+    }
+    mark(4);
+    p->last_launches = launches;
+    return VORTA_OK;
+}
+
+int vorta_routed_attention_host(const vorta_plan *p, const void *Qh, const void *Kh, const void *Vh, void *Oh,
+                                void *scratch, size_t scratch_bytes, void *stream)
+{
+    if (!p || !Qh || !Kh || !Vh || !Oh || !scratch) return VORTA_ERR_INVALID_ARG;
+    if (p->host_only) return VORTA_ERR_UNSUPPORTED;
+    vorta_plan_info_t info;
+    vorta_plan_info(p, &info);
+    if ((int64_t)scratch_bytes < info.host_call_scratch_bytes) return VORTA_ERR_WORKSPACE;
+    if (!aligned(scratch, 256)) return VORTA_ERR_ALIGNMENT;
+    DeviceGuard guard(p->device);
+    if (!guard.ok) return VORTA_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int64_t tb = tensor_bytes(p->g), tba = align_up(tb, 256);
+    char *base = static_cast<char *>(scratch);
+    void *dq = base, *dk = base + tba, *dv = base + 2 * tba, *dO = base + 3 * tba, *ws = base + 4 * tba;
+    if (cudaMemcpyAsync(dq, Qh, tb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(dk, Kh, tb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(dv, Vh, tb, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return VORTA_ERR_CUDA;
+    int rc = vorta_routed_attention(p, dq, dk, dv, dO, nullptr, 0, info.workspace_bytes ? ws : nullptr,
+                                    (size_t)info.workspace_bytes, stream);
+    if (rc != VORTA_OK) return rc;
+    if (cudaMemcpyAsync(Oh, dO, tb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return VORTA_ERR_CUDA;
+    return VORTA_OK;
+}
+
+int vorta_device_status(const vorta_plan *p, void *stream, int32_t *code_out)
+{
+    if (!p || !code_out) return VORTA_ERR_INVALID_ARG;
+    if (p->host_only) return VORTA_ERR_UNSUPPORTED;
+    DeviceGuard guard(p->device);
+    if (!guard.ok) return VORTA_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaStreamSynchronize(s) != cudaSuccess) return VORTA_ERR_CUDA;
+    int32_t code = 0;
+    if (cudaMemcpy(&code, p->d_status, sizeof(code), cudaMemcpyDeviceToHost) != cudaSuccess) return VORTA_ERR_CUDA;
+    *code_out = code;
+    if (code != 0) {
+        cudaMemset(p->d_status, 0, sizeof(int32_t));
+        return VORTA_ERR_TIMEOUT;
+    }
+    return VORTA_OK;
+}
+
+}  // extern "C"

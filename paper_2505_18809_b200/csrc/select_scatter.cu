@@ -1,0 +1,289 @@
+// Memory-bound kernels of the routed-attention layer: the block-sparse sliding-tile
+// mask builder, bucketed core-set selection, the gather (pool) of the kept rows
+// and the scatter (unpool) of the attention output.
+#include "vorta_internal.h"
+
+namespace vorta {
+
+// ---------------------------------------------------------------------------------
+// Sliding tile mask between tiles (Appendix A.1, Algorithm 1).
+// ---------------------------------------------------------------------------------
+
+__device__ __forceinline__ void tile_triple(const Geometry &g, int32_t id, int32_t q[3])
+{
+    q[2] = id % g.nt[2];
+    q[1] = (id / g.nt[2]) % g.nt[1];
+    q[0] = id / (g.nt[2] * g.nt[1]);
+}
+
+// One thread per (query tile, key tile): move the query tile to its window-centre
+// tile, then test the per-axis tile distance against floor(w/2).
+__global__ void block_mask_kernel(Geometry g, uint8_t *__restrict__ bm)
+{
+    int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    int64_t total = (int64_t)g.n_tiles * g.n_tiles;
+    if (idx >= total) return;
+    int32_t q[3], k[3];
+    tile_triple(g, (int32_t)(idx / g.n_tiles), q);
+    tile_triple(g, (int32_t)(idx % g.n_tiles), k);
+    bool m = true;
+#pragma unroll
+    for (int a = 0; a < 3; ++a) {
+        if (!g.restricted[a]) continue;
+        int32_t c = min(max(q[a], g.half[a]), g.nt[a] - 1 - g.half[a]);
+        m = m && (abs(c - k[a]) <= g.half[a]);
+    }
+    bm[idx] = m ? 1 : 0;
+}
+
+// One thread per query tile: turn its mask row into the list of KV blocks the
+// attention kernel walks (key tiles ascending; a tile of more than 128 tokens
+// gives two boxes; boxes that lie wholly outside the grid are dropped).
+__global__ void kv_list_kernel(Geometry g, const uint8_t *__restrict__ bm, KvEntry *__restrict__ list,
+                               int32_t *__restrict__ count)
+{
+    int32_t qt = blockIdx.x * blockDim.x + threadIdx.x;
+    if (qt >= g.n_tiles) return;
+    KvEntry *out = list + (int64_t)qt * g.max_kv_per_tile;
+    int32_t n = 0;
+    for (int32_t kt = 0; kt < g.n_tiles; ++kt) {
+        if (!bm[(int64_t)qt * g.n_tiles + kt]) continue;
+        int32_t k[3];
+        tile_triple(g, kt, k);
+        int32_t t0 = k[0] * g.tile[0], h0 = k[1] * g.tile[1], w0 = k[2] * g.tile[2];
+        int32_t pt = (g.T - t0 < g.tile[0]), ph = (g.H - h0 < g.tile[1]), pw = (g.W - w0 < g.tile[2]);
+        for (int32_t bx = 0; bx < g.boxes_per_tile; ++bx) {
+            int32_t tb = t0 + bx * g.box[0];
+            if (tb >= g.T) break;
+            bool whole = !pt && !ph && !pw && g.box_rows == g.bn_tile;
+            if (n < g.max_kv_per_tile) {
+                KvEntry e;
+                e.w0 = (int16_t)w0;
+                e.h0 = (int16_t)h0;
+                e.t0 = (int16_t)tb;
+                e.mask_id = whole ? 0 : (uint16_t)(1 + ((pt * 2 + ph) * 2 + pw) * 2 + bx);
+                out[n] = e;
+            }
+            ++n;
+        }
+    }
+    count[qt] = n;
+}
+
+cudaError_t launch_block_mask(const Geometry &g, uint8_t *bm, KvEntry *kv_list, int32_t *kv_count,
+                              cudaStream_t s)
+{
+    int64_t total = (int64_t)g.n_tiles * g.n_tiles;
+    block_mask_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(g, bm);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    kv_list_kernel<<<(g.n_tiles + 127) / 128, 128, 0, s>>>(g, bm, kv_list, kv_count);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------
+// Bucketed core-set selection (Section 3.2; Appendix A.1).
+// One warp per (problem, bucket).  Eight lanes share a token: each lane takes
+// every eighth 16-byte chunk of the row, products and sums are fp64 (a bf16 x bf16
+// product is exact there), and three shuffle steps finish the row.  Four tokens
+// are scored per pass.
+// ---------------------------------------------------------------------------------
+
+__device__ __forceinline__ double shfl_xor_f64(double v, int m)
+{
+    int lo = __double2loint(v), hi = __double2hiint(v);
+    lo = __shfl_xor_sync(0xffffffffu, lo, m);
+    hi = __shfl_xor_sync(0xffffffffu, hi, m);
+    return __hiloint2double(hi, lo);
+}
+
+__device__ __forceinline__ double shfl_f64(double v, int src)
+{
+    int lo = __double2loint(v), hi = __double2hiint(v);
+    lo = __shfl_sync(0xffffffffu, lo, src);
+    hi = __shfl_sync(0xffffffffu, hi, src);
+    return __hiloint2double(hi, lo);
+}
+
+__device__ __forceinline__ void bf16x8_to_f64(const uint4 &u, double out[8])
+{
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        out[2 * i] = (double)__uint_as_float(w[i] << 16);
+        out[2 * i + 1] = (double)__uint_as_float(w[i] & 0xffff0000u);
+    }
+}
+
+__global__ void __launch_bounds__(256)
+coreset_select_kernel(Geometry g, const __nv_bfloat16 *__restrict__ X, int32_t dx, int32_t n_prob,
+                      const int32_t *__restrict__ prob_slice, const int32_t *__restrict__ seg_start,
+                      int32_t *__restrict__ core_idx, int32_t *__restrict__ src_slot)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (warp >= (int64_t)n_prob * g.n_buckets) return;
+    const int32_t p = (int32_t)(warp / g.n_buckets);
+    const int32_t bkt = (int32_t)(warp % g.n_buckets);
+    const int32_t slice = prob_slice ? prob_slice[p] : p;
+    const __nv_bfloat16 *Xs = X + (int64_t)slice * g.L * dx;
+
+    // the bucket: id, extents cut by the grid, token count, centre
+    int32_t id[3] = {bkt / (g.nb[2] * g.nb[1]), (bkt / g.nb[2]) % g.nb[1], bkt % g.nb[2]};
+    const int32_t dim[3] = {g.T, g.H, g.W};
+    int32_t e[3];
+#pragma unroll
+    for (int a = 0; a < 3; ++a) e[a] = min(g.bucket[a], dim[a] - g.bucket[a] * id[a]);
+    const int32_t n = e[0] * e[1] * e[2];
+    const int32_t centre = ((e[0] / 2) * e[1] + (e[1] / 2)) * e[2] + (e[2] / 2);
+    auto token_of = [&](int32_t l) -> int32_t {
+        int32_t lw = l % e[2], lh = (l / e[2]) % e[1], lt = l / (e[2] * e[1]);
+        return ((id[0] * g.bucket[0] + lt) * g.H + (id[1] * g.bucket[1] + lh)) * g.W +
+               (id[2] * g.bucket[2] + lw);
+    };
+
+    const int sub = lane >> 3, sl = lane & 7;
+    const int32_t chunks = dx >> 3;
+    const uint4 *xc = reinterpret_cast<const uint4 *>(Xs + (int64_t)token_of(centre) * dx);
+
+    double my_score = 0.0;  // lane l ends up with the score of local token l
+    double ncsq = 0.0;
+    for (int32_t pass = 0; pass * 4 < n; ++pass) {
+        const int32_t l = pass * 4 + sub;
+        const bool active = l < n;
+        double dot = 0.0, njsq = 0.0, csq = 0.0;
+        if (active) {
+            const uint4 *xj = reinterpret_cast<const uint4 *>(Xs + (int64_t)token_of(l) * dx);
+            for (int32_t c = sl; c < chunks; c += 8) {
+                double a[8], b[8];
+                bf16x8_to_f64(__ldg(xc + c), a);
+                bf16x8_to_f64(__ldg(xj + c), b);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    dot = fma(a[i], b[i], dot);
+                    njsq = fma(b[i], b[i], njsq);
+                    csq = fma(a[i], a[i], csq);
+                }
+            }
+        }
+#pragma unroll
+        for (int m = 4; m >= 1; m >>= 1) {
+            dot += shfl_xor_f64(dot, m);
+            njsq += shfl_xor_f64(njsq, m);
+            csq += shfl_xor_f64(csq, m);
+        }
+        if (pass == 0) ncsq = shfl_f64(csq, 0);  // token 0 always exists
+        double nc = sqrt(ncsq), nj = sqrt(njsq);
+        double score = (nc == 0.0 || nj == 0.0) ? 0.0 : dot / (nc * nj);
+        double got = shfl_f64(score, (lane & 3) * 8);
+        if ((lane >> 2) == pass) my_score = got;
+    }
+
+    // keep(n) = max(1, floor(r n + 1/2)); the k = n - keep most similar tokens go
+    int32_t keep = (int32_t)floor(g.ratio * (double)n + 0.5);
+    keep = max(keep, 1);
+    const int32_t k = n - keep;
+    const bool is_tok = lane < n, is_centre = lane == centre;
+    int32_t rank = 0;
+    for (int32_t m = 0; m < n; ++m) {
+        double sm = shfl_f64(my_score, m);
+        if (m != centre && (sm > my_score || (sm == my_score && m < lane))) ++rank;
+    }
+    const bool kept = is_tok && (is_centre || rank >= k);
+    const uint32_t kept_others = __ballot_sync(0xffffffffu, kept && !is_centre);
+    if (!is_tok) return;
+    const int32_t seg = seg_start[bkt];
+    const int32_t tok = token_of(lane);
+    int32_t slot = seg;  // the centre's slot: pruned tokens receive its output
+    if (kept && !is_centre) slot = seg + 1 + __popc(kept_others & ((1u << lane) - 1u));
+    if (kept) core_idx[(int64_t)p * g.Lc + slot] = tok;
+    src_slot[(int64_t)p * g.L + tok] = slot;
+}
+
+cudaError_t launch_select(const Geometry &g, const __nv_bfloat16 *X, int32_t dx, int32_t n_prob,
+                          const int32_t *prob_slice, const int32_t *seg_start, int32_t *core_idx,
+                          int32_t *src_slot, cudaStream_t s)
+{
+    int64_t warps = (int64_t)n_prob * g.n_buckets;
+    if (warps == 0) return cudaSuccess;
+    int64_t blocks = (warps + 7) / 8;
+    coreset_select_kernel<<<(unsigned)blocks, 256, 0, s>>>(g, X, dx, n_prob, prob_slice, seg_start,
+                                                           core_idx, src_slot);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------
+// pool: gather the kept rows of Q, K, V into compact [n_prob, Lc, d] tensors.
+// 16 bytes per thread; blockIdx.y picks the tensor.
+// ---------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+gather_rows_kernel(Geometry g, int32_t n_prob, const int32_t *__restrict__ prob_slice,
+                   const int32_t *__restrict__ core_idx, const uint4 *__restrict__ Q,
+                   const uint4 *__restrict__ K, const uint4 *__restrict__ V, uint4 *__restrict__ Qc,
+                   uint4 *__restrict__ Kc, uint4 *__restrict__ Vc)
+{
+    const int32_t cpr = g.d >> 3;  // 16-byte chunks per row
+    const int64_t total = (int64_t)n_prob * g.Lc * cpr;
+    const uint4 *src = blockIdx.y == 0 ? Q : (blockIdx.y == 1 ? K : V);
+    uint4 *dst = blockIdx.y == 0 ? Qc : (blockIdx.y == 1 ? Kc : Vc);
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        int64_t row = i / cpr;
+        int32_t c = (int32_t)(i % cpr);
+        int32_t p = (int32_t)(row / g.Lc);
+        int32_t tok = __ldg(core_idx + row);
+        dst[i] = __ldg(src + ((int64_t)prob_slice[p] * g.L + tok) * cpr + c);
+    }
+}
+
+cudaError_t launch_gather(const Geometry &g, int32_t n_prob, const int32_t *prob_slice,
+                          const int32_t *core_idx, const __nv_bfloat16 *Q, const __nv_bfloat16 *K,
+                          const __nv_bfloat16 *V, __nv_bfloat16 *Qc, __nv_bfloat16 *Kc,
+                          __nv_bfloat16 *Vc, cudaStream_t s)
+{
+    if (n_prob == 0) return cudaSuccess;
+    int64_t total = (int64_t)n_prob * g.Lc * (g.d >> 3);
+    unsigned blocks = (unsigned)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
+    gather_rows_kernel<<<dim3(blocks, 3), 256, 0, s>>>(
+        g, n_prob, prob_slice, core_idx, reinterpret_cast<const uint4 *>(Q),
+        reinterpret_cast<const uint4 *>(K), reinterpret_cast<const uint4 *>(V),
+        reinterpret_cast<uint4 *>(Qc), reinterpret_cast<uint4 *>(Kc), reinterpret_cast<uint4 *>(Vc));
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------
+// unpool: every token of a core-set head receives the output row of its slot
+// (its own row if kept, its bucket centre's row if pruned).
+// ---------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+scatter_rows_kernel(Geometry g, int32_t n_prob, const int32_t *__restrict__ prob_slice,
+                    const int32_t *__restrict__ src_slot, const uint4 *__restrict__ Oc,
+                    uint4 *__restrict__ O)
+{
+    const int32_t cpr = g.d >> 3;
+    const int64_t total = (int64_t)n_prob * g.L * cpr;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        int64_t row = i / cpr;
+        int32_t c = (int32_t)(i % cpr);
+        int32_t p = (int32_t)(row / g.L);
+        int32_t tok = (int32_t)(row % g.L);
+        int32_t slot = __ldg(src_slot + row);
+        O[((int64_t)prob_slice[p] * g.L + tok) * cpr + c] = __ldg(Oc + ((int64_t)p * g.Lc + slot) * cpr + c);
+    }
+}
+
+cudaError_t launch_scatter(const Geometry &g, int32_t n_prob, const int32_t *prob_slice,
+                           const int32_t *src_slot, const __nv_bfloat16 *Oc, __nv_bfloat16 *O,
+                           cudaStream_t s)
+{
+    if (n_prob == 0) return cudaSuccess;
+    int64_t total = (int64_t)n_prob * g.L * (g.d >> 3);
+    unsigned blocks = (unsigned)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
+    scatter_rows_kernel<<<blocks, 256, 0, s>>>(g, n_prob, prob_slice, src_slot,
+                                               reinterpret_cast<const uint4 *>(Oc),
+                                               reinterpret_cast<uint4 *>(O));
+    return cudaGetLastError();
+}
+
+}  // namespace vorta

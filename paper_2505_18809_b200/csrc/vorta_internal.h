@@ -1,0 +1,117 @@
+// Internal declarations shared by the translation units of libvorta.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "vorta.h"
+
+namespace vorta {
+
+// How an attention work item addresses its rows.
+enum : int32_t {
+    MODE_LINEAR = 0,   // full head: 128 consecutive tokens of the original tensors per block
+    MODE_TILES = 1,    // sliding head: one 3D (sub-)tile of the original tensors per block
+    MODE_COMPACT = 2   // core-set head: 128 consecutive rows of the gathered tensors per block
+};
+
+constexpr int kBlockM = 128;       // query rows per M-block (one MMA M)
+constexpr int kMaxMasks = 17;      // column-mask classes of the sliding branch (0 = none)
+constexpr int kAttnThreads = 384;  // tcgen05 kernel: 4 control warps + 2 softmax warpgroups
+
+// Plain geometry, passed to kernels by value.
+struct Geometry {
+    int32_t B, heads;
+    int32_t T, H, W, L, d;
+    int32_t tile[3], nt[3], n_tiles;      // sliding tiles (T, H, W order)
+    int32_t half[3], restricted[3];       // floor(w/2); 0 when the window covers the axis
+    int32_t bucket[3], nb[3], n_buckets;  // core-set buckets
+    int32_t Lc;
+    double ratio;
+    // sliding branch blocking: one block = a TMA box of box[0] x box[1] x box[2] tokens
+    int32_t box[3], box_rows, bn_tile, boxes_per_tile, max_kv_per_tile;
+};
+
+// One KV block of a sliding-tile query: origin of its box and its column-mask class.
+struct KvEntry {
+    int16_t w0, h0, t0;
+    uint16_t mask_id;
+};
+
+// One unit of work of the attention kernel: up to two 128-row query blocks that
+// walk the same sequence of KV blocks.
+struct WorkItem {
+    int32_t mode;
+    int32_t slice;        // 5th tensor-map coordinate: b*heads + head, or the compact problem id
+    int32_t n_mblk;       // 1 or 2
+    int32_t kv_count;     // number of KV blocks
+    int32_t kv_begin;     // MODE_TILES: first entry in the KV list
+    int32_t kv_len;       // linear modes: number of keys (L or Lc)
+    int32_t q_org[2][3];  // per M-block: (w0, h0, t0) of the box, or (row0, 0, 0)
+    int32_t pad[4];
+};
+static_assert(sizeof(WorkItem) == 64, "WorkItem must stay 64 bytes");
+
+// Tensor maps of one attention launch (all 5-D: d, W|rows, H, T, slice).
+struct AttnMaps {
+    CUtensorMap q[3], k[3], v[3];  // indexed by mode
+};
+
+struct AttnParams {
+    Geometry g;
+    float scale_log2;              // softmax scale * log2(e)
+    const WorkItem *items;
+    const int32_t *cta_begin;      // [grid] first item of each CTA
+    const int32_t *cta_count;      // [grid]
+    const KvEntry *kv_list;
+    const uint32_t *colmasks;      // [kMaxMasks][4]
+    __nv_bfloat16 *O;              // [B*heads, L, d]
+    __nv_bfloat16 *Oc;             // [n_compact, Lc, d]
+    const __nv_bfloat16 *Q, *K, *V;     // originals (SIMT kernel)
+    const __nv_bfloat16 *Qc, *Kc, *Vc;  // gathered (SIMT kernel)
+    int32_t *status;               // device word: 0 or the code of an expired wait
+};
+
+// ---- launchers (each returns cudaGetLastError of its launch) ----------------------
+cudaError_t launch_block_mask(const Geometry &g, uint8_t *bm, KvEntry *kv_list, int32_t *kv_count,
+                              cudaStream_t s);
+cudaError_t launch_select(const Geometry &g, const __nv_bfloat16 *X, int32_t dx, int32_t n_prob,
+                          const int32_t *prob_slice, const int32_t *seg_start, int32_t *core_idx,
+                          int32_t *src_slot, cudaStream_t s);
+cudaError_t launch_gather(const Geometry &g, int32_t n_prob, const int32_t *prob_slice,
+                          const int32_t *core_idx, const __nv_bfloat16 *Q, const __nv_bfloat16 *K,
+                          const __nv_bfloat16 *V, __nv_bfloat16 *Qc, __nv_bfloat16 *Kc,
+                          __nv_bfloat16 *Vc, cudaStream_t s);
+cudaError_t launch_scatter(const Geometry &g, int32_t n_prob, const int32_t *prob_slice,
+                           const int32_t *src_slot, const __nv_bfloat16 *Oc, __nv_bfloat16 *O,
+                           cudaStream_t s);
+cudaError_t launch_attention_simt(const AttnParams &p, int32_t n_items, cudaStream_t s);
+cudaError_t launch_attention_sm100(const AttnParams &p, const AttnMaps &maps, int32_t grid,
+                                   cudaStream_t s);
+cudaError_t attention_sm100_prepare();  // opt in to the kernel's dynamic shared memory
+
+// Row r of an M-/KV-block -> token id; false if the row lies outside the grid/sequence.
+__host__ __device__ inline bool block_row_token(const Geometry &g, int32_t mode, const int32_t org[3],
+                                                int32_t len, int32_t r, int32_t *token)
+{
+    if (mode == MODE_TILES) {
+        if (r >= g.box_rows) return false;
+        int32_t lw = r % g.box[2];
+        int32_t lh = (r / g.box[2]) % g.box[1];
+        int32_t lt = r / (g.box[2] * g.box[1]);
+        int32_t w = org[0] + lw, h = org[1] + lh, t = org[2] + lt;
+        if (w >= g.W || h >= g.H || t >= g.T) return false;
+        *token = (t * g.H + h) * g.W + w;
+        return true;
+    }
+    int32_t i = org[0] + r;
+    if (i >= len) return false;
+    *token = i;
+    return true;
+}
+
+}  // namespace vorta

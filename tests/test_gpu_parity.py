@@ -1,0 +1,235 @@
+"""GPU parity: the CUDA library against the CPU oracle, through the C ABI.
+
+Integer results (block masks, core-set indices, scatter maps) must be bit-exact;
+attention outputs must be within max-abs 2e-2 and mean-abs 2e-3 (bf16 in, fp32
+accumulate), per head."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import assert_close, head_f64, oracle_head_rows, sample_rows
+from paper_2505_18809_b200 import binding as vb
+from paper_2505_18809_b200 import build as vbuild
+from paper_2505_18809_b200 import workloads
+from paper_2505_18809_b200.workloads import Workload
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    vbuild.build()
+    vb.lib()
+
+
+def small_workloads():
+    W = Workload
+    return [
+        # name, grid, heads, d, tile, window, ratio, routes, seed, smooth
+        W("tiny-c1", (4, 8, 8), 2, 64, (2, 4, 4), (3, 3, 3), 0.25, (1, 2), 0, False),
+        W("three-routes-d64", (6, 10, 12), 3, 64, (2, 4, 4), (3, 3, 3), 0.5, (0, 1, 2), 21, True),
+        # 4 tiles per axis and more: real windows, ragged H and W, 256-token tiles split in two boxes
+        W("ragged-256tile", (9, 21, 27), 3, 128, (4, 8, 8), (3, 3, 3), 0.5, (1, 0, 2), 22, True),
+        # 64-token tiles (one box per tile), ragged on T
+        W("tile64", (10, 12, 20), 4, 128, (4, 4, 4), (3, 3, 3), 0.25, (1, 1, 2, 0), 23, True),
+        # tile tokens not a multiple of 16 (27 -> padded to 32 columns), window 1 and 5
+        W("tile27", (7, 9, 12), 3, 128, (3, 3, 3), (1, 3, 5), 0.5, (1, 2, 1), 24, True),
+        # several 256-row items per head, tail block of 73 rows, batch of 2
+        W("linear-tail", (3, 17, 19), 2, 128, (1, 8, 8), (3, 3, 3), 0.75, (0, 2), 25, False, 2),
+        # ratio 1: the core-set is a permutation of all tokens
+        W("ratio-one", (4, 6, 8), 2, 64, (2, 3, 4), (3, 3, 3), 1.0, (2, 2), 26, False),
+        # bucket other than the default, grid smaller than one tile on T
+        W("bucket-133", (1, 14, 15), 2, 128, (2, 4, 4), (3, 3, 3), 0.34, (2, 1), 27, True, 1, (1, 3, 3)),
+    ]
+
+
+def run_layer(plan, wl, Q, K, V, kernel):
+    plan.set_kernel(kernel)
+    O = torch.full_like(Q, float("nan"))
+    plan.routed_attention(Q, K, V, O)
+    assert plan.device_status() == 0
+    return O
+
+
+# --------------------------------------------------------------------------- masks
+@pytest.mark.parametrize("grid,tile,window", [
+    ((4, 8, 8), (2, 4, 4), (3, 3, 3)), ((9, 21, 27), (4, 8, 8), (3, 3, 3)),
+    ((7, 9, 12), (3, 3, 3), (1, 3, 5)), ((10, 5, 5), (2, 2, 3), (2, 3, 3)),
+    ((21, 30, 52), (4, 4, 4), (3, 3, 3)), ((33, 45, 80), (4, 8, 8), (3, 3, 3)),
+    ((21, 45, 80), (4, 8, 8), (3, 3, 3)), ((30, 45, 80), (6, 9, 8), (3, 3, 3))])
+def test_block_mask_bit_exact(grid, tile, window):
+    if tile[0] * tile[1] * tile[2] > 256:
+        pytest.skip("tile larger than this build supports")
+    p = vb.Plan(1, 1, grid, 128, tile, window, 0.5, (1,))
+    got = p.block_mask()
+    want = oracle.sta_block_mask(grid, tile, window)
+    assert got.dtype == np.uint8 and np.array_equal(got, want)
+    p.close()
+
+
+# --------------------------------------------------------------------------- selection
+@pytest.mark.parametrize("wl", small_workloads(), ids=lambda w: w.name)
+def test_coreset_select_bit_exact_small(wl):
+    _, K, _ = workloads.make_qkv(wl, DEV)
+    p = vb.Plan.from_workload(wl)
+    core, src = p.coreset_select(K)
+    torch.cuda.synchronize()
+    r = float(np.float32(wl.ratio))
+    for b in range(wl.B):
+        for h in range(wl.heads):
+            c, s = oracle.coreset_select(wl.grid, wl.bucket, r, head_f64(K, b, h))
+            assert np.array_equal(core[b, h].cpu().numpy(), c), (b, h)
+            assert np.array_equal(src[b, h].cpu().numpy(), s), (b, h)
+    p.close()
+
+
+def test_coreset_select_other_feature_width_and_ties():
+    wl = Workload("sel", (5, 7, 6), 2, 128, (2, 4, 4), (3, 3, 3), 0.5, (2, 2), 31, True)
+    p = vb.Plan.from_workload(wl)
+    g = torch.Generator(device=DEV).manual_seed(5)
+    X = torch.randn((1, 3, wl.L, 40), generator=g, device=DEV).to(torch.bfloat16)
+    X[0, 1] = 1.0                      # every cosine ties: the index tie-break decides
+    X[0, 2, ::3] = 0.0                 # zero-norm rows score 0
+    core, src = p.coreset_select(X)
+    for h in range(3):
+        c, s = oracle.coreset_select(wl.grid, wl.bucket, 0.5, head_f64(X, 0, h))
+        assert np.array_equal(core[0, h].cpu().numpy(), c), h
+        assert np.array_equal(src[0, h].cpu().numpy(), s), h
+    p.close()
+
+
+# --------------------------------------------------------------------------- attention, small
+@pytest.mark.parametrize("kernel", [vb.VORTA_KERNEL_SIMT, vb.VORTA_KERNEL_TCGEN05], ids=["simt", "tcgen05"])
+@pytest.mark.parametrize("wl", small_workloads(), ids=lambda w: w.name)
+def test_routed_attention_small_all_rows(wl, kernel):
+    Q, K, V = workloads.make_qkv(wl, DEV)
+    p = vb.Plan.from_workload(wl)
+    O = run_layer(p, wl, Q, K, V, kernel)
+    for b in range(wl.B):
+        for h in range(wl.heads):
+            want = oracle_head_rows(wl, Q, K, V, b, h, None)
+            assert_close(O[b, h], want, f"{wl.name} b{b} h{h} route {wl.routes[h]}")
+    p.close()
+
+
+def test_pruned_rows_copy_their_centre_and_reruns_are_bitwise_equal():
+    wl = small_workloads()[2]
+    Q, K, V = workloads.make_qkv(wl, DEV)
+    p = vb.Plan.from_workload(wl)
+    O1 = run_layer(p, wl, Q, K, V, vb.VORTA_KERNEL_TCGEN05)
+    O2 = run_layer(p, wl, Q, K, V, vb.VORTA_KERNEL_TCGEN05)
+    assert torch.equal(O1.view(torch.int16), O2.view(torch.int16))
+    h = wl.routes.index(2)
+    core, src = oracle.coreset_select(wl.grid, wl.bucket, float(np.float32(wl.ratio)), head_f64(K, 0, h))
+    owner = torch.from_numpy(core[src].astype(np.int64)).to(DEV)
+    assert torch.equal(O1[0, h].view(torch.int16), O1[0, h][owner].view(torch.int16))
+    p.close()
+
+
+def test_routes_can_change_between_steps_and_shared_selection_features():
+    wl = small_workloads()[1]
+    Q, K, V = workloads.make_qkv(wl, DEV)
+    p = vb.Plan.from_workload(wl)
+    for routes in [(2, 2, 2), (0, 0, 0), (1, 1, 1), (2, 0, 1)]:
+        p.set_routes(routes)
+        O = run_layer(p, wl, Q, K, V, vb.VORTA_KERNEL_TCGEN05)
+        for h in range(wl.heads):
+            want = oracle_head_rows(wl, Q, K, V, 0, h, None, route=routes[h])
+            assert_close(O[0, h], want, f"routes {routes} h{h}")
+    # one shared feature tensor for all heads (selection on the block input, Hx = 1)
+    p.set_routes((2, 2, 2))
+    g = torch.Generator(device=DEV).manual_seed(9)
+    X = torch.randn((1, 1, wl.L, wl.d), generator=g, device=DEV).to(torch.bfloat16)
+    O = torch.empty_like(Q)
+    p.routed_attention(Q, K, V, O, X=X)
+    assert p.device_status() == 0
+    for h in range(wl.heads):
+        want = oracle_head_rows(wl, Q, K, V, 0, h, None, route=2, X=head_f64(X, 0, 0))
+        assert_close(O[0, h], want, f"shared X h{h}")
+    p.close()
+
+
+def test_argument_errors_launch_nothing():
+    wl = small_workloads()[1]
+    Q, K, V = workloads.make_qkv(wl, DEV)
+    p = vb.Plan.from_workload(wl)
+    O = torch.zeros_like(Q)
+    info = p.info
+    ws = torch.empty(info.workspace_bytes + 256, dtype=torch.uint8, device=DEV)
+    L = vb.lib()
+    args = lambda q, w, n: (p.handle, q, K.data_ptr(), V.data_ptr(), O.data_ptr(), None, 0, w, n, None)
+    assert L.vorta_routed_attention(*args(Q.data_ptr() + 2, ws.data_ptr(), ws.numel())) == vb.VORTA_ERR_ALIGNMENT
+    assert L.vorta_routed_attention(*args(Q.data_ptr(), ws.data_ptr(), 16)) == vb.VORTA_ERR_WORKSPACE
+    assert L.vorta_routed_attention(*args(Q.data_ptr(), None, 0)) == vb.VORTA_ERR_WORKSPACE
+    assert L.vorta_routed_attention(*args(Q.data_ptr(), ws.data_ptr() + 16, ws.numel() - 16)) == vb.VORTA_ERR_ALIGNMENT
+    assert L.vorta_routed_attention(*args(None, ws.data_ptr(), ws.numel())) == vb.VORTA_ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert float(O.abs().sum()) == 0.0
+    p.close()
+
+
+def test_host_buffer_entry_point_matches_device_path():
+    wl = small_workloads()[3]
+    Q, K, V = workloads.make_qkv(wl, DEV)
+    p = vb.Plan.from_workload(wl)
+    O = run_layer(p, wl, Q, K, V, vb.VORTA_KERNEL_TCGEN05)
+    Qh, Kh, Vh = (t.cpu().pin_memory() for t in (Q, K, V))
+    Oh = torch.empty_like(Qh).pin_memory()
+    scratch = torch.empty(p.info.host_call_scratch_bytes, dtype=torch.uint8, device=DEV)
+    p.routed_attention_host(Qh, Kh, Vh, Oh, scratch)
+    assert p.device_status() == 0
+    assert torch.equal(Oh.view(torch.int16), O.cpu().view(torch.int16))
+    p.close()
+
+
+# --------------------------------------------------------------------------- the named configurations
+def check_config(wl, rows_per_head, kernels=(vb.VORTA_KERNEL_TCGEN05,)):
+    Q, K, V = workloads.make_qkv(wl, DEV)
+    p = vb.Plan.from_workload(wl)
+    # integer stages in full: block mask, indices and scatter map of every core-set head
+    assert np.array_equal(p.block_mask(), oracle.sta_block_mask(wl.grid, wl.tile, wl.window))
+    core_heads = [h for h in range(wl.heads) if wl.routes[h] == 2]
+    if core_heads:
+        core, src = p.coreset_select(K)
+        for h in core_heads:
+            c, s = oracle.coreset_select(wl.grid, wl.bucket, float(np.float32(wl.ratio)), head_f64(K, 0, h))
+            assert np.array_equal(core[0, h].cpu().numpy(), c), h
+            assert np.array_equal(src[0, h].cpu().numpy(), s), h
+        del core, src
+    for kernel in kernels:
+        O = run_layer(p, wl, Q, K, V, kernel)
+        assert bool(torch.isfinite(O.float()).all())
+        worst = 0.0
+        for h in range(wl.heads):
+            rows = None if rows_per_head is None else sample_rows(wl, rows_per_head, 1000 + h)
+            want = oracle_head_rows(wl, Q, K, V, 0, h, rows)
+            got = O[0, h] if rows is None else O[0, h][torch.from_numpy(rows).to(DEV)]
+            mx, _ = assert_close(got, want, f"{wl.name} h{h} route {wl.routes[h]} kernel {kernel}")
+            worst = max(worst, mx)
+        print(f"{wl.name} kernel {kernel}: worst max-abs {worst:.3e}")
+    p.close()
+
+
+def test_config_tiny_all_rows():
+    check_config(workloads.config("tiny"), None, (vb.VORTA_KERNEL_SIMT, vb.VORTA_KERNEL_TCGEN05))
+
+
+def test_config_wan13b_480p_sampled_rows():
+    check_config(workloads.config("wan1.3b-480p"), 96, (vb.VORTA_KERNEL_SIMT, vb.VORTA_KERNEL_TCGEN05))
+
+
+def test_config_hunyuan_720p_sampled_rows():
+    check_config(workloads.config("hunyuan-720p"), 48)
+
+
+def test_config_wan14b_720p_sampled_rows():
+    check_config(workloads.config("wan14b-720p"), 32)
+
+
+def test_config_route_mix_sweep_sampled_rows():
+    # two corners of the sweep: no full heads at ratio .25, half full heads at ratio .5
+    sweep = {w.name: w for w in workloads.route_mix_sweep()}
+    check_config(sweep["hunyuan-720p-full0-r0.25"], 24)
+    check_config(sweep["hunyuan-720p-full0.5-r0.5"], 24)
