@@ -190,6 +190,9 @@ VORTA_API int vorta_routed_attention_host(const vorta_plan *plan, const void *Q_
  */
 VORTA_API int vorta_plan_set_profiling(vorta_plan *plan, int32_t on);
 VORTA_API int vorta_plan_stage_ms(const vorta_plan *plan, float ms[4]);
+/* The same for an earlier call: calls_back = 0 is the last profiled call, 1 the one
+ * before it, ... up to 63.  VORTA_ERR_INVALID_ARG if that call was never made. */
+VORTA_API int vorta_plan_stage_ms_at(const vorta_plan *plan, int32_t calls_back, float ms[4]);
 
 /* Number of kernels the last vorta_routed_attention call launched. */
 VORTA_API int vorta_plan_last_launches(const vorta_plan *plan, int32_t *n);

@@ -27,7 +27,7 @@ EXPORTS = (
     "vorta_plan_create", "vorta_plan_set_routes", "vorta_plan_destroy", "vorta_plan_info",
     "vorta_plan_block_mask", "vorta_plan_set_kernel", "vorta_coreset_select",
     "vorta_routed_attention", "vorta_routed_attention_host", "vorta_plan_set_profiling",
-    "vorta_plan_stage_ms", "vorta_plan_last_launches", "vorta_device_status",
+    "vorta_plan_stage_ms", "vorta_plan_stage_ms_at", "vorta_plan_last_launches", "vorta_device_status",
     "vorta_status_string",
 )
 
@@ -80,6 +80,7 @@ def lib() -> ctypes.CDLL:
     L.vorta_routed_attention_host.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     L.vorta_plan_set_profiling.argtypes = [vp, i32]
     L.vorta_plan_stage_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float * 4)]
+    L.vorta_plan_stage_ms_at.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_float * 4)]
     L.vorta_plan_last_launches.argtypes = [vp, ctypes.POINTER(i32)]
     L.vorta_device_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
     L.vorta_status_string.argtypes = [ctypes.c_int]
@@ -170,6 +171,12 @@ def vorta_plan_stage_ms(plan: int):
     return [float(x) for x in ms]
 
 
+def vorta_plan_stage_ms_at(plan: int, calls_back: int):
+    ms = (ctypes.c_float * 4)()
+    _check(lib().vorta_plan_stage_ms_at(plan, calls_back, ctypes.byref(ms)), "vorta_plan_stage_ms_at")
+    return [float(x) for x in ms]
+
+
 def vorta_plan_last_launches(plan: int) -> int:
     n = ctypes.c_int32()
     _check(lib().vorta_plan_last_launches(plan, ctypes.byref(n)), "vorta_plan_last_launches")
@@ -246,8 +253,9 @@ class Plan:
     def set_profiling(self, on: bool):
         vorta_plan_set_profiling(self.handle, on)
 
-    def stage_ms(self):
-        return vorta_plan_stage_ms(self.handle)
+    def stage_ms(self, calls_back: int = 0):
+        """[select, gather, attention, scatter] milliseconds of a profiled call."""
+        return vorta_plan_stage_ms_at(self.handle, calls_back)
 
     def last_launches(self) -> int:
         return vorta_plan_last_launches(self.handle)

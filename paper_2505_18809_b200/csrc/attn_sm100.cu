@@ -481,8 +481,11 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
                 for (int c = 0; c < 64; c += 2) {
                     const float p0 = ex2(fmaf(__uint_as_float(s[c]), scale, neg_max));
                     const float p1 = ex2(fmaf(__uint_as_float(s[c + 1]), scale, neg_max));
-                    sum += p0 + p1;
-                    s[c >> 1] = pack_bf16(p0, p1);
+                    // the row sum takes the rounded values the PV MMA will really use, so
+                    // that O / sum stays a true weighted mean of V rows
+                    const uint32_t pk = pack_bf16(p0, p1);
+                    sum += __uint_as_float(pk << 16) + __uint_as_float(pk & 0xffff0000u);
+                    s[c >> 1] = pk;
                 }
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {

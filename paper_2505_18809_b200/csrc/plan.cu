@@ -37,9 +37,12 @@ struct vorta_plan {
     double flops_issued = 0.0;
     double sliding_pairs = 0.0;  // sum over listed tile pairs of valid-token products
     int32_t kernel = VORTA_KERNEL_TCGEN05;
-    // profiling
-    mutable cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
-    mutable bool ev_valid[5] = {false, false, false, false, false};
+    // profiling: a ring of event sets, one per call, so that several calls can be
+    // enqueued before their stage times are read
+    static constexpr int kProfSlots = 64;
+    mutable cudaEvent_t ev[kProfSlots][5] = {};
+    mutable bool ev_valid[kProfSlots][5] = {};
+    mutable int64_t prof_calls = 0;  // calls recorded so far
     bool profiling = false;
     mutable int32_t last_launches = 0;
 };
@@ -118,8 +121,9 @@ void free_device(vorta_plan *p)
     cudaFree(p->d_seg_start); cudaFree(p->d_items); cudaFree(p->d_cta_begin);
     cudaFree(p->d_cta_count); cudaFree(p->d_core_slice); cudaFree(p->d_core_xslice);
     cudaFree(p->d_status);
-    for (auto &e : p->ev)
-        if (e) cudaEventDestroy(e);
+    for (auto &set : p->ev)
+        for (auto &e : set)
+            if (e) cudaEventDestroy(e);
 }
 
 // valid tokens of tile `id` on axis a
@@ -421,7 +425,8 @@ int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
     ok = ok && cudaMemset(p->d_status, 0, sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMemcpy(p->d_colmasks, masks.data(), sizeof(uint32_t) * masks.size(), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(p->d_seg_start, p->seg_start.data(), sizeof(int32_t) * g.n_buckets, cudaMemcpyHostToDevice) == cudaSuccess;
-    for (auto &e : p->ev) ok = ok && cudaEventCreate(&e) == cudaSuccess;
+    for (auto &set : p->ev)
+        for (auto &e : set) ok = ok && cudaEventCreate(&e) == cudaSuccess;
     // the mask builder runs once per shape; its per-tile counts come back for the work list
     ok = ok && launch_block_mask(g, p->d_bm, p->d_kv_list, p->d_kv_count, nullptr) == cudaSuccess;
     p->kv_count.resize(g.n_tiles);
@@ -515,20 +520,24 @@ int vorta_plan_set_profiling(vorta_plan *p, int32_t on)
     return VORTA_OK;
 }
 
-int vorta_plan_stage_ms(const vorta_plan *p, float ms[4])
+int vorta_plan_stage_ms_at(const vorta_plan *p, int32_t calls_back, float ms[4])
 {
-    if (!p || !ms) return VORTA_ERR_INVALID_ARG;
+    if (!p || !ms || calls_back < 0 || calls_back >= vorta_plan::kProfSlots) return VORTA_ERR_INVALID_ARG;
     if (p->host_only) return VORTA_ERR_UNSUPPORTED;
+    if (calls_back >= p->prof_calls) return VORTA_ERR_INVALID_ARG;
+    const int slot = (int)((p->prof_calls - 1 - calls_back) % vorta_plan::kProfSlots);
     for (int i = 0; i < 4; ++i) {
         ms[i] = 0.f;
-        if (p->ev_valid[i] && p->ev_valid[i + 1] &&
-            cudaEventElapsedTime(&ms[i], p->ev[i], p->ev[i + 1]) != cudaSuccess) {
+        if (p->ev_valid[slot][i] && p->ev_valid[slot][i + 1] &&
+            cudaEventElapsedTime(&ms[i], p->ev[slot][i], p->ev[slot][i + 1]) != cudaSuccess) {
             cudaGetLastError();
             return VORTA_ERR_CUDA;
         }
     }
     return VORTA_OK;
 }
+
+int vorta_plan_stage_ms(const vorta_plan *p, float ms[4]) { return vorta_plan_stage_ms_at(p, 0, ms); }
 
 int vorta_plan_last_launches(const vorta_plan *p, int32_t *n)
 {
@@ -609,9 +618,13 @@ int vorta_routed_attention(const vorta_plan *p, const void *Q, const void *K, co
 
     int32_t launches = 0;
     const bool prof = p->profiling;
-    for (auto &f : p->ev_valid) f = false;
+    const int pslot = (int)(p->prof_calls % vorta_plan::kProfSlots);
+    if (prof) {
+        for (auto &f : p->ev_valid[pslot]) f = false;
+        ++p->prof_calls;
+    }
     auto mark = [&](int i) {
-        if (prof && cudaEventRecord(p->ev[i], s) == cudaSuccess) p->ev_valid[i] = true;
+        if (prof && cudaEventRecord(p->ev[pslot][i], s) == cudaSuccess) p->ev_valid[pslot][i] = true;
     };
     cudaError_t e = cudaSuccess;
     mark(0);

@@ -92,8 +92,9 @@ def _smooth_field(n_chan: int, grid, g: torch.Generator, device) -> torch.Tensor
     divided by the number of cells really covered), times sqrt(125), plus 0.3*N(0,1)."""
     T, H, W = grid
     x = torch.randn((n_chan, 1, T, H, W), generator=g, device=device, dtype=torch.float32)
-    blur = torch.nn.functional.avg_pool3d(x, kernel_size=5, stride=1, padding=2,
-                                          count_include_pad=False)
+    ones = torch.ones((1, 1, 5, 5, 5), device=device, dtype=torch.float32)
+    cells = torch.nn.functional.conv3d(torch.ones((1, 1, T, H, W), device=device), ones, padding=2)
+    blur = torch.nn.functional.conv3d(x, ones, padding=2) / cells
     blur = blur * math.sqrt(125.0)
     blur += 0.3 * torch.randn((n_chan, 1, T, H, W), generator=g, device=device,
                               dtype=torch.float32)

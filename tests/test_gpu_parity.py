@@ -41,7 +41,7 @@ def small_workloads():
         # ratio 1: the core-set is a permutation of all tokens
         W("ratio-one", (4, 6, 8), 2, 64, (2, 3, 4), (3, 3, 3), 1.0, (2, 2), 26, False),
         # bucket other than the default, grid smaller than one tile on T
-        W("bucket-133", (1, 14, 15), 2, 128, (2, 4, 4), (3, 3, 3), 0.34, (2, 1), 27, True, 1, (1, 3, 3)),
+        W("bucket-133", (1, 14, 15), 2, 128, (2, 4, 4), (3, 3, 3), 0.34, (2, 1), 27, False, 1, (1, 3, 3)),
     ]
 
 
