@@ -1,0 +1,385 @@
+#!/usr/bin/env python
+"""Benchmark of one routed-attention layer (select + gather + attention + scatter).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+A step is one call of vorta_routed_attention on one layer's Q/K/V (seeded
+synthetic, resident in HBM).  The line printed by rank 0 carries:
+  value        effective TFLOP/s = algorithmic FLOPs of the layer / time per step
+               (4*d*pairs the method attends: L^2 full, valid window pairs sliding,
+               Lc^2 core-set), whole job over all ranks
+  ms_per_step  ms per layer
+  roofline     the attention kernel alone: algorithmic FLOPs / its CUDA-event time
+               against the measured dense bf16 peak
+  e2e          the same metric through vorta_routed_attention_host with pinned HOST
+               buffers (H2D of Q, K, V and D2H of O inside the timed region)
+  cpu_baseline the fp64 CPU oracle timed on a bounded sample of rows of the same workload
+With --impl reference the oracle itself is the timed arm.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "routed_attention_effective_tflops"
+UNIT = "TFLOP/s"
+DEFAULT_WORKLOAD = "hunyuan-720p"
+FALLBACK_PEAK_TFLOPS = 1590.0   # used only if MEASURED_PEAKS.json is absent
+# DRAM bytes per attention-kernel launch from the ncu capture summarised under profiles/
+# (None until a capture of this kernel exists).
+ATTENTION_DRAM_TRAFFIC_BYTES = None
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"bf16": float(p["bf16_tflops"]), "bf16_sustained": float(p.get("bf16_tflops_sustained", 0.0)),
+                "hbm": float(p["hbm_gbs"]), "source": "measured"}
+    return {"bf16": FALLBACK_PEAK_TFLOPS, "bf16_sustained": 1400.0, "hbm": 6650.0, "source": "fallback"}
+
+
+def get_workload(name):
+    from paper_2505_18809_b200 import workloads
+    if name in workloads.CONFIG_NAMES or name in workloads.PROFILE_NAMES:
+        return workloads.config(name)
+    for w in workloads.route_mix_sweep():
+        if w.name == name:
+            return w
+    raise SystemExit(f"unknown workload {name}")
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "200"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        def pump():
+            for line in self.proc.stdout:
+                self.rows.append((time.time(), line.strip()))
+        self.thread = threading.Thread(target=pump, daemon=True)
+        self.thread.start()
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()   # the exact child started above
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], None, set()
+        for ts, line in self.rows:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                clk, mx = float(parts[0]), float(parts[1])
+            except ValueError:
+                continue
+            smax = mx
+            if t0 - 0.1 <= ts <= t1 + 0.3:
+                sm.append(clk)
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                      "sw_power_cap"), parts[3:7]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        if not sm:
+            sm = [float(l.split(",")[0]) for _, l in self.rows[-3:] if l and l.split(",")[0].strip().replace(".", "").isdigit()]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": smax,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------- oracle timing
+def _window_keys(wl, token: int) -> int:
+    """Number of keys Algorithm 1 lets this query see (for the FLOP count of a sampled row)."""
+    T, H, W = wl.grid
+    c = (token // (H * W), (token // W) % H, token % W)
+    n = 1
+    for a in range(3):
+        nt = -(-wl.grid[a] // wl.tile[a])
+        half = wl.window[a] // 2
+        if nt <= 2 * half + 1:
+            n *= wl.grid[a]
+            continue
+        q = c[a] // wl.tile[a]
+        centre = min(max(q, half), nt - 1 - half)
+        lo, hi = (centre - half) * wl.tile[a], min((centre + half + 1) * wl.tile[a], wl.grid[a])
+        n *= hi - lo
+    return n
+
+
+def time_oracle(wl, Q, K, V, rows_per_head: int, budget_s: float, seed: int = 0):
+    import numpy as np
+    import torch
+    import oracle
+    scale = 1.0 / math.sqrt(wl.d)
+    Lc = oracle.coreset_len(wl.grid, wl.bucket, float(np.float32(wl.ratio)))
+    g = np.random.default_rng(seed)
+    flops, t_total, heads_done = 0.0, 0.0, 0
+    for h in range(wl.heads):
+        if t_total > budget_s:
+            break
+        q, k, v = (x[0, h].to("cpu", torch.float64).numpy() for x in (Q, K, V))
+        rows = np.sort(g.choice(wl.L, size=min(rows_per_head, wl.L), replace=False)).astype(np.int64)
+        t0 = time.perf_counter()
+        if wl.routes[h] == 0:
+            oracle.attn_full(q, k, v, scale, q_rows=rows)
+            f = 4.0 * wl.d * wl.L * len(rows)
+        elif wl.routes[h] == 1:
+            oracle.attn_sliding(wl.grid, wl.tile, wl.window, q, k, v, scale, q_rows=rows)
+            f = 4.0 * wl.d * sum(_window_keys(wl, int(r)) for r in rows)
+        else:
+            _, _, src = oracle.attn_coreset(wl.grid, wl.bucket, float(np.float32(wl.ratio)), q, k, v, scale,
+                                            q_rows=rows)
+            f = 4.0 * wl.d * Lc * len(set(src[rows].tolist()))
+        t_total += time.perf_counter() - t0
+        flops += f
+        heads_done += 1
+    return flops, t_total, heads_done, oracle.num_threads()
+
+
+# ----------------------------------------------------------------------------- arms
+def run_reference(args):
+    """The oracle as the timed arm: each step is a bounded sample of rows of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import torch
+    import oracle
+    from paper_2505_18809_b200 import workloads
+    oracle.build()
+    wl = get_workload(args.workload)
+    dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+    Q, K, V = workloads.make_qkv(wl, dev)
+    Q, K, V = Q.cpu(), K.cpu(), V.cpu()
+    rows = args.reference_rows
+    for _ in range(args.warmup):
+        time_oracle(wl, Q, K, V, max(1, rows // 4), 5.0)
+    flops, secs = 0.0, 0.0
+    heads = 0
+    for s in range(args.steps):
+        f, t, heads, threads = time_oracle(wl, Q, K, V, rows, 120.0 / max(1, args.steps), seed=s)
+        flops += f
+        secs += t
+    value = flops / secs / 1e12
+    sample = f"{rows} random query rows of each of {heads} heads per step, all their keys"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": wl.name, "grid": list(wl.grid), "heads": wl.heads,
+                                            "d": wl.d, "routes": list(wl.routes)},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2505_18809_b200 import binding as vb
+    from paper_2505_18809_b200 import build as vbuild
+    from paper_2505_18809_b200 import workloads
+
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA library has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    if rank == 0:
+        vbuild.build()
+    if world > 1:
+        dist.barrier()
+    vb.lib()
+
+    wl = get_workload(args.workload)
+    pk = peaks()
+    # every rank holds its own layer (heads are independent: no exchange inside the op)
+    Q, K, V = workloads.make_qkv(wl, dev)
+    O = torch.empty_like(Q)
+    plan = vb.Plan.from_workload(wl, device=local)
+    info = plan.info
+    ws = plan.workspace(dev)
+    plan.set_profiling(True)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def step():
+        plan.routed_attention(Q, K, V, O, workspace=ws)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    assert plan.device_status() == 0
+
+    # ---- timed region: exactly K steps, device time, max over ranks
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_wall0 = time.time()
+    e0.record(stream)
+    launches = 0
+    for _ in range(args.steps):
+        step()
+        launches += plan.last_launches()
+    e1.record(stream)
+    barrier()
+    t_wall1 = time.time()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    assert plan.device_status() == 0
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * info.flops_layer / (ms_step * 1e-3) / 1e12
+
+    # stage times of the timed steps (CUDA events recorded by the library on the same stream)
+    n_hist = min(args.steps, 64)
+    stages = [plan.stage_ms(i) for i in range(n_hist)]
+    st = [sum(s[i] for s in stages) / n_hist for i in range(4)]
+    attn_ms = st[2]
+    n_core = info.n_coreset * wl.B
+
+    out = None
+    if rank == 0:
+        achieved = info.flops_layer / (attn_ms * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "kernel": "attention_sm100_kernel", "achieved": achieved,
+                    "peak": pk["bf16"], "unit": UNIT, "frac": achieved / pk["bf16"],
+                    "peak_source": f"{pk['source']} burst bf16",
+                    "frac_of_sustained": achieved / pk["bf16_sustained"] if pk["bf16_sustained"] else None,
+                    "frac_of_nominal_2250": achieved / 2250.0,
+                    "issued_tflops": info.flops_issued_layer / (attn_ms * 1e-3) / 1e12,
+                    "kernel_ms": attn_ms, "traffic": ATTENTION_DRAM_TRAFFIC_BYTES}
+        gbs = lambda b, ms: (b / (ms * 1e-3) / 1e9) if ms > 0 else None
+        stage = {"select_ms": st[0], "gather_ms": st[1], "attention_ms": st[2], "scatter_ms": st[3],
+                 "select_gbs": gbs(n_core * info.select_bytes_head, st[0]),
+                 "gather_gbs": gbs(n_core * info.gather_bytes_head, st[1]),
+                 "scatter_gbs": gbs(n_core * info.scatter_bytes_head, st[3]),
+                 "hbm_peak_gbs": pk["hbm"]}
+        out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+               "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "ms_per_layer": ms_step,
+               "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+               "data": "synthetic",
+               "config": {"workload": wl.name, "grid": list(wl.grid), "tokens": wl.L, "heads": wl.heads,
+                          "d": wl.d, "tile": list(wl.tile), "window_tiles": list(wl.window),
+                          "coreset_ratio": wl.ratio, "routes": list(wl.routes),
+                          "heads_full_sliding_coreset": [info.n_full, info.n_sliding, info.n_coreset],
+                          "algorithmic_tflop_per_layer": info.flops_layer / 1e12,
+                          "issued_tflop_per_layer": info.flops_issued_layer / 1e12,
+                          "l2": "inputs (3 x %.0f MB) larger than L2" % (Q.numel() * 2 / 1e6),
+                          "per_rank": "one layer per GPU, no collective on the data path"},
+               "frac_of_bf16_peak": value / world / pk["bf16"],
+               "roofline": roofline, "stages": stage, "gpu_launches": launches, "clocks": clocks}
+
+    # ---- end to end through the host-buffer entry point (rank-local, max over ranks)
+    e2e = None
+    if not args.no_e2e:
+        Qh, Kh, Vh = (torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t) for t in (Q, K, V))
+        Oh = torch.empty(Q.shape, dtype=Q.dtype, pin_memory=True)
+        scratch = torch.empty(int(info.host_call_scratch_bytes), dtype=torch.uint8, device=dev)
+        for _ in range(2):
+            plan.routed_attention_host(Qh, Kh, Vh, Oh, scratch)
+        barrier()
+        n_e2e = max(2, min(args.steps, 5))
+        e0.record(stream)
+        for _ in range(n_e2e):
+            plan.routed_attention_host(Qh, Kh, Vh, Oh, scratch)
+        e1.record(stream)
+        barrier()
+        ms_e2e = e0.elapsed_time(e1) / n_e2e
+        if world > 1:
+            t = torch.tensor([ms_e2e], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t.item())
+        tb = Q.numel() * 2
+        e2e = {"value": world * info.flops_layer / (ms_e2e * 1e-3) / 1e12, "unit": UNIT,
+               "ms_per_step": ms_e2e, "steps": n_e2e, "h2d_bytes_per_step": 3 * tb, "d2h_bytes_per_step": tb,
+               "api": "vorta_routed_attention_host (pinned host Q, K, V in; O out)"}
+        del scratch, Qh, Kh, Vh
+    if rank == 0:
+        out["e2e"] = e2e
+
+    # ---- the oracle on the host cores, rank 0 at N = 1 only
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        Qc, Kc, Vc = Q.cpu(), K.cpu(), V.cpu()
+        rows = args.cpu_rows
+        flops, secs, heads, threads = time_oracle(wl, Qc, Kc, Vc, rows, 25.0)
+        out["cpu_baseline"] = {"value": flops / secs / 1e12, "unit": UNIT, "cores": threads, "kind": "oracle",
+                               "seconds": secs,
+                               "sample": f"{rows} random query rows of each of the first {heads} heads "
+                                         f"(of {wl.heads}), all their keys; fp64"}
+    elif rank == 0:
+        out["cpu_baseline"] = None
+    if rank == 0:
+        print(json.dumps(out))
+    plan.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cpu-rows", type=int, default=120, help="oracle rows per head for cpu_baseline")
+    ap.add_argument("--reference-rows", type=int, default=16, help="oracle rows per head per step (--impl reference)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

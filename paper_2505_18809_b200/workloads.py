@@ -68,10 +68,16 @@ def config(name: str) -> Workload:
     if name == "wan14b-720p":
         return Workload(name, (21, 45, 80), 40, 128, (4, 8, 8), (3, 3, 3), 0.25,
                         apportion_routes(40, (0.0, 0.8, 0.2), 3), 3, True)
+    if name == "hunyuan-720p-3h":
+        # profiling case: the HunyuanVideo-720p grid with one head per route, so that a
+        # counter capture of one launch stays short while the inputs still exceed L2
+        return Workload(name, (33, 45, 80), 3, 128, (4, 8, 8), (3, 3, 3), 0.5,
+                        (ROUTE_FULL, ROUTE_SLIDING, ROUTE_CORESET), 2, True)
     raise KeyError(name)
 
 
 CONFIG_NAMES = ("tiny", "wan1.3b-480p", "hunyuan-720p", "wan14b-720p")
+PROFILE_NAMES = ("hunyuan-720p-3h",)
 
 
 def route_mix_sweep() -> List[Workload]:
