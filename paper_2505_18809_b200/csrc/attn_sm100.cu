@@ -51,8 +51,9 @@ enum {
     BAR_KV_FULL = 2,               // +slot
     BAR_KV_EMPTY = 2 + kStages,    // +slot
     BAR_S_FULL = 2 + 2 * kStages,  // +tile
-    BAR_P_FULL = BAR_S_FULL + 2,
-    BAR_PV_DONE = BAR_P_FULL + 2,
+    BAR_P_LO = BAR_S_FULL + 2,     // +tile: P columns of keys [0, 64) written
+    BAR_P_HI = BAR_P_LO + 2,       // +tile: the rest of P written
+    BAR_PV_DONE = BAR_P_HI + 2,
     BAR_O_FREE = BAR_PV_DONE + 2,
     BAR_MMA_DRAINED = BAR_O_FREE + 2,
     BAR_COUNT
@@ -64,6 +65,20 @@ struct Ctl {
     volatile int32_t abort;
 };
 static_assert(sizeof(Ctl) <= 512, "control block outgrew its reservation");
+
+// Optional cycle trace of one CTA (compiled in only with -DVORTA_TRACE; a debugging aid).
+#ifdef VORTA_TRACE
+#define VORTA_TRACE_J0 16
+#define VORTA_TRACE_NJ 8
+#define TRACE(role, j, ev)                                                                      \
+    do {                                                                                         \
+        if (p.trace && blockIdx.x == 0 && it == 0 && (j) >= VORTA_TRACE_J0 &&                    \
+            (j) < VORTA_TRACE_J0 + VORTA_TRACE_NJ)                                               \
+            p.trace[(((role) * VORTA_TRACE_NJ) + ((j) - VORTA_TRACE_J0)) * 8 + (ev)] = clock64(); \
+    } while (0)
+#else
+#define TRACE(role, j, ev) do { } while (0)
+#endif
 
 // ------------------------------------------------------------------ PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
@@ -131,6 +146,28 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, Ctl *ct
     return mbar_wait_slow(bar, parity, ctl, status, code);
 }
 
+// The same wait with a warp-uniform verdict, and a warp-uniform copy of a value all
+// lanes hold: both come out of warp-wide reductions, which the compiler can keep in
+// uniform registers.  The MMA warp needs this: the operands of tcgen05.mma are uniform
+// registers, and only provably uniform values and control flow reach them without a
+// per-instruction detour through vector registers.
+__device__ __forceinline__ bool mbar_wait_uniform(uint32_t bar, uint32_t parity, Ctl *ctl, int32_t *status,
+                                                  int32_t code)
+{
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, ctl, status, code)) != 0;
+}
+
+__device__ __forceinline__ uint32_t uniform_u32(uint32_t v) { return __reduce_max_sync(0xffffffffu, v); }
+
+__device__ __forceinline__ uint32_t elect_one()
+{
+    uint32_t leader;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(leader));
+    return leader;
+}
+
 __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int32_t c0,
                                             int32_t c1, int32_t c2, int32_t c3, int32_t c4)
 {
@@ -146,30 +183,36 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-__device__ __forceinline__ void tc_commit(uint32_t bar)
+// The MMA warp stays converged: every lane runs the (warp-uniform) descriptor
+// arithmetic, and `leader` (1 in lane 0, 0 elsewhere) guards the instruction itself.
+__device__ __forceinline__ void tc_commit(uint32_t bar, uint32_t leader)
 {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    asm volatile(
+        "{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+        ::"r"(bar), "r"(leader)
+        : "memory");
 }
 
 // D[tmem] (+)= A[smem] * B[smem]
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                       uint32_t accumulate)
+                                       uint32_t accumulate, uint32_t leader)
 {
     asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %4, 0;\n\tsetp.ne.b32 q, %5, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(leader)
         : "memory");
 }
 
 // D[tmem] (+)= A[tmem] * B[smem]
 __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                       uint32_t accumulate)
+                                       uint32_t accumulate, uint32_t leader)
 {
     asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %4, 0;\n\tsetp.ne.b32 q, %5, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(leader)
         : "memory");
 }
 
@@ -231,26 +274,6 @@ __device__ __forceinline__ void kv_block_coords(const AttnParams &p, const WorkI
     }
 }
 
-// 64 score columns of this thread's row (only the chunks below `cols` are read)
-__device__ __forceinline__ void load_scores(uint32_t (&s)[64], uint32_t taddr, int32_t cols)
-{
-    uint32_t(&lo)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[0]);
-    uint32_t(&hi)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[32]);
-    ptx::tcgen05_ld_32x32b(lo, taddr);
-    if (cols > 32) ptx::tcgen05_ld_32x32b(hi, taddr + 32);
-    tc_wait_ld();
-}
-
-// columns whose mask bit is 0 are not keys: their score becomes -inf
-__device__ __forceinline__ void mask_scores(uint32_t (&s)[64], uint32_t m0, uint32_t m1)
-{
-#pragma unroll
-    for (int c = 0; c < 32; ++c) {
-        if (!((m0 >> c) & 1u)) s[c] = 0xff800000u;
-        if (!((m1 >> c) & 1u)) s[32 + c] = 0xff800000u;
-    }
-}
-
 // ------------------------------------------------------------------ roles
 template <int D>
 __device__ __forceinline__ void producer_role(const AttnParams &p, const AttnMaps &maps, Ctl *ctl, uint32_t smem_base,
@@ -296,94 +319,111 @@ __device__ __forceinline__ void producer_role(const AttnParams &p, const AttnMap
 
 template <int D>
 __device__ __forceinline__ void mma_role(const AttnParams &p, Ctl *ctl, uint32_t smem_base, uint32_t tmem,
-                                         int32_t begin, int32_t count, int lane)
+                                         int32_t begin, int32_t count)
 {
     const uint32_t bars = smem_u32(ctl->bars);
+    const uint32_t leader = elect_one();
+    tmem = uniform_u32(tmem);
+    begin = (int32_t)uniform_u32((uint32_t)begin);
+    count = (int32_t)uniform_u32((uint32_t)count);
     uint32_t kv_it = 0;
     uint32_t p_cnt[2] = {0, 0}, o_uses[2] = {0, 0};
 
-    // S_m = Q_m K^T over the K block in `slot`
+    // Descriptors of tile 0 / slot 0; the others differ by a multiple of the tile pitch
+    // in the (16-byte granular) address field, so one 64-bit add moves between them.
+    const uint64_t q_desc0 = smem_desc(smem_base + kSmemQ, 16, 1024);
+    const uint64_t k_desc0 = smem_desc(smem_base + kSmemKV, 16, 1024);          // K-major
+    const uint64_t v_desc0 = smem_desc(smem_base + kSmemKV, kHalfBytes, 1024);  // MN-major
+    constexpr uint64_t kTileStep = kTileBytes >> 4;
+
+    // S_m = Q_m K^T over the K block in `slot` (16 channels per MMA)
     auto issue_qk = [&](int m, uint32_t slot, uint32_t idesc) {
-        const uint32_t qa = smem_base + kSmemQ + m * kTileBytes;
-        const uint32_t kb = smem_base + kSmemKV + slot * kTileBytes;
+        const uint64_t qa = q_desc0 + (uint64_t)m * kTileStep;
+        const uint64_t kb = k_desc0 + (uint64_t)slot * kTileStep;
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
-            const uint32_t off = (kk / 4) * kHalfBytes + (kk % 4) * 32;
-            mma_ss(tmem + m * 128, smem_desc(qa + off, 16, 1024), smem_desc(kb + off, 16, 1024), idesc, kk > 0);
+            const uint64_t off = (uint64_t)(((kk / 4) * kHalfBytes + (kk % 4) * 32) >> 4);
+            mma_ss(tmem + m * 128, qa + off, kb + off, idesc, kk > 0 ? 1u : 0u, leader);
         }
     };
     // O_m (+)= P_m V over the V block in `slot`; P is packed bf16 in S_m's columns
-    auto issue_pv = [&](int m, uint32_t slot, uint32_t idesc, int32_t bn, bool first) {
-        const uint32_t vb = smem_base + kSmemKV + slot * kTileBytes;
-        for (int kk = 0; kk < bn / 16; ++kk)
-            mma_ts(tmem + 256 + m * 128, tmem + m * 128 + kk * 8, smem_desc(vb + kk * 2048, kHalfBytes, 1024), idesc,
-                   (!first || kk > 0) ? 1u : 0u);
+    // (16 keys per MMA: steps [K0, K0 + 4) of the block, cut at `ksteps`)
+    auto issue_pv = [&](int m, uint32_t slot, uint32_t idesc, int k0, int ksteps, bool first) {
+        const uint64_t vb = v_desc0 + (uint64_t)slot * kTileStep;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int kk = k0 + i;
+            if (kk < ksteps)
+                mma_ts(tmem + 256 + m * 128, tmem + m * 128 + kk * 8, vb + (uint64_t)(kk * (2048 >> 4)), idesc,
+                       (!first || kk > 0) ? 1u : 0u, leader);
+        }
     };
 
     for (int32_t it = 0; it < count; ++it) {
-        const WorkItem w = p.items[begin + it];
-        const int32_t bn = w.mode == MODE_TILES ? p.g.bn_tile : kBlockM;
-        const int32_t n = w.kv_count, nm = w.n_mblk;
+        const WorkItem *w = p.items + begin + it;
+        const int32_t bn = uniform_u32((uint32_t)w->mode) == MODE_TILES ? p.g.bn_tile : kBlockM;
+        const int32_t n = (int32_t)uniform_u32((uint32_t)w->kv_count);
+        const int32_t nm = (int32_t)uniform_u32((uint32_t)w->n_mblk);
         const uint32_t idesc_qk = instr_desc((uint32_t)bn, 0), idesc_pv = instr_desc((uint32_t)D, 1);
+        const int ksteps = bn / 16;
 
-        if (!mbar_wait(bars + 8 * BAR_Q_FULL, it & 1, ctl, p.status, 201)) return;
+        if (!mbar_wait_uniform(bars + 8 * BAR_Q_FULL, it & 1, ctl, p.status, 201)) return;
         // block 0: both score tiles
         uint32_t slot_k = kv_it % kStages;
-        if (!mbar_wait(bars + 8 * (BAR_KV_FULL + slot_k), (kv_it / kStages) & 1, ctl, p.status, 202)) return;
+        if (!mbar_wait_uniform(bars + 8 * (BAR_KV_FULL + slot_k), (kv_it / kStages) & 1, ctl, p.status, 202)) return;
         ++kv_it;
         tc_fence_after();
-        if (lane == 0) {
-            for (int m = 0; m < nm; ++m) {
-                issue_qk(m, slot_k, idesc_qk);
-                tc_commit(bars + 8 * (BAR_S_FULL + m));
-            }
-            tc_commit(bars + 8 * (BAR_KV_EMPTY + slot_k));
-            if (n == 1) tc_commit(bars + 8 * BAR_Q_EMPTY);
+        for (int m = 0; m < nm; ++m) {
+            issue_qk(m, slot_k, idesc_qk);
+            tc_commit(bars + 8 * (BAR_S_FULL + m), leader);
         }
-        __syncwarp();
+        tc_commit(bars + 8 * (BAR_KV_EMPTY + slot_k), leader);
+        if (n == 1) tc_commit(bars + 8 * BAR_Q_EMPTY, leader);
         for (int32_t j = 0; j < n; ++j) {
             const uint32_t slot_v = kv_it % kStages;
-            if (!mbar_wait(bars + 8 * (BAR_KV_FULL + slot_v), (kv_it / kStages) & 1, ctl, p.status, 203)) return;
+            if (!mbar_wait_uniform(bars + 8 * (BAR_KV_FULL + slot_v), (kv_it / kStages) & 1, ctl, p.status, 203)) return;
             ++kv_it;
             const bool has_next = j + 1 < n;
             slot_k = kv_it % kStages;
             for (int m = 0; m < nm; ++m) {
-                if (!mbar_wait(bars + 8 * (BAR_P_FULL + m), p_cnt[m] & 1, ctl, p.status, 204)) return;
-                ++p_cnt[m];
+                // first half of P: the PV MMAs over keys [0, 64) start while the softmax
+                // threads still work on the second half
+                if (!mbar_wait_uniform(bars + 8 * (BAR_P_LO + m), p_cnt[m] & 1, ctl, p.status, 204)) return;
                 if (j == 0) {
                     // the previous item's epilogue must have read O_m out of TMEM
-                    if (!mbar_wait(bars + 8 * (BAR_O_FREE + m), (o_uses[m] & 1) ^ 1, ctl, p.status, 205)) return;
+                    if (!mbar_wait_uniform(bars + 8 * (BAR_O_FREE + m), (o_uses[m] & 1) ^ 1, ctl, p.status, 205)) return;
                     ++o_uses[m];
                 }
+                tc_fence_after();
+                if (leader) TRACE(m, j, 0);
+                issue_pv(m, slot_v, idesc_pv, 0, ksteps, j == 0);
+                if (leader) TRACE(m, j, 1);
+                if (!mbar_wait_uniform(bars + 8 * (BAR_P_HI + m), p_cnt[m] & 1, ctl, p.status, 208)) return;
+                ++p_cnt[m];
                 if (has_next && m == 0) {
-                    if (!mbar_wait(bars + 8 * (BAR_KV_FULL + slot_k), (kv_it / kStages) & 1, ctl, p.status, 206)) return;
+                    if (!mbar_wait_uniform(bars + 8 * (BAR_KV_FULL + slot_k), (kv_it / kStages) & 1, ctl, p.status, 206)) return;
                 }
                 tc_fence_after();
-                if (lane == 0) {
-                    issue_pv(m, slot_v, idesc_pv, bn, j == 0);
-                    if (!has_next) tc_commit(bars + 8 * (BAR_PV_DONE + m));
-                    if (has_next) {
-                        issue_qk(m, slot_k, idesc_qk);
-                        tc_commit(bars + 8 * (BAR_S_FULL + m));
-                    }
-                }
-                __syncwarp();
-            }
-            if (lane == 0) {
-                tc_commit(bars + 8 * (BAR_KV_EMPTY + slot_v));
+                if (leader) TRACE(m, j, 2);
+                issue_pv(m, slot_v, idesc_pv, 4, ksteps, false);
+                if (!has_next) tc_commit(bars + 8 * (BAR_PV_DONE + m), leader);
                 if (has_next) {
-                    tc_commit(bars + 8 * (BAR_KV_EMPTY + slot_k));
-                    if (j + 2 == n) tc_commit(bars + 8 * BAR_Q_EMPTY);
+                    issue_qk(m, slot_k, idesc_qk);
+                    tc_commit(bars + 8 * (BAR_S_FULL + m), leader);
                 }
+                if (leader) TRACE(m, j, 3);
             }
-            if (has_next) ++kv_it;
-            __syncwarp();
+            tc_commit(bars + 8 * (BAR_KV_EMPTY + slot_v), leader);
+            if (has_next) {
+                tc_commit(bars + 8 * (BAR_KV_EMPTY + slot_k), leader);
+                if (j + 2 == n) tc_commit(bars + 8 * BAR_Q_EMPTY, leader);
+                ++kv_it;
+            }
         }
     }
     // every commit issued above must have landed before the CTA's barriers go away
-    if (lane == 0) tc_commit(bars + 8 * BAR_MMA_DRAINED);
-    __syncwarp();
-    mbar_wait(bars + 8 * BAR_MMA_DRAINED, 0, ctl, p.status, 207);
+    tc_commit(bars + 8 * BAR_MMA_DRAINED, leader);
+    mbar_wait_uniform(bars + 8 * BAR_MMA_DRAINED, 0, ctl, p.status, 207);
 }
 
 template <int D>
@@ -433,21 +473,36 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
                 }
             }
 
+            if (row == 0) TRACE(2 + m, j, 0);
             if (!mbar_wait(bars + 8 * (BAR_S_FULL + m), s_cnt & 1, ctl, p.status, 301 + m)) return;
             ++s_cnt;
             tc_fence_after();
+            if (row == 0) TRACE(2 + m, j, 1);
 
-            // pass 1: the row maximum, 64 columns at a time
-            float mx = -INFINITY;
+            // the whole score row of this thread, one TMEM read
+            uint32_t s[128];
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                if (h * 64 >= bn) break;
-                uint32_t s[64];
-                load_scores(s, t_s + h * 64, bn - h * 64);
-                if (!whole) mask_scores(s, mask[2 * h], mask[2 * h + 1]);
-#pragma unroll
-                for (int c = 0; c < 64; ++c) mx = fmaxf(mx, __uint_as_float(s[c]));
+            for (int c = 0; c < 4; ++c) {
+                uint32_t(&chunk)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[32 * c]);
+                if (c * 32 < bn) ptx::tcgen05_ld_32x32b(chunk, t_s + c * 32);
             }
+            tc_wait_ld();
+            if (row == 0) TRACE(2 + m, j, 2);
+            if (!whole) {
+#pragma unroll
+                for (int c = 0; c < 128; ++c)
+                    if (!((mask[c >> 5] >> (c & 31)) & 1u)) s[c] = 0xff800000u;  // -inf: not a key
+            }
+            // row maximum over four independent chains
+            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < 128; c += 4) {
+                mx0 = fmaxf(mx0, __uint_as_float(s[c]));
+                mx1 = fmaxf(mx1, __uint_as_float(s[c + 1]));
+                mx2 = fmaxf(mx2, __uint_as_float(s[c + 2]));
+                mx3 = fmaxf(mx3, __uint_as_float(s[c + 3]));
+            }
+            const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
             const float m_new = fmaxf(row_max, mx * scale);
             if (j == 0) {
                 row_max = m_new;
@@ -467,36 +522,50 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
                     ptx::tcgen05_st_32x32b(t_o + c * 32, o);
                 }
             }
-            // pass 2: P = exp2(S * scale - max) as packed bf16 over the first bn/2 columns of S.
-            // Half h reads columns [64h, 64h + 64) and writes [32h, 32h + 32): never ahead of a read.
+            // P = exp2(S * scale - max) as packed bf16 over the first bn/2 columns of S, in two
+            // halves: keys [0, 64) -> columns [0, 32), then keys [64, 128) -> columns [32, 64).
+            // A packed word never lands on a score that is still to be read.
             const float neg_max = -row_max;
-            float sum = 0.f;
+            if (row == 0) TRACE(2 + m, j, 3);
+            float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                if (h * 64 >= bn) break;
-                uint32_t s[64];
-                load_scores(s, t_s + h * 64, bn - h * 64);
-                if (!whole) mask_scores(s, mask[2 * h], mask[2 * h + 1]);
+                if (h * 64 < bn) {
 #pragma unroll
-                for (int c = 0; c < 64; c += 2) {
-                    const float p0 = ex2(fmaf(__uint_as_float(s[c]), scale, neg_max));
-                    const float p1 = ex2(fmaf(__uint_as_float(s[c + 1]), scale, neg_max));
-                    // the row sum takes the rounded values the PV MMA will really use, so
-                    // that O / sum stays a true weighted mean of V rows
-                    const uint32_t pk = pack_bf16(p0, p1);
-                    sum += __uint_as_float(pk << 16) + __uint_as_float(pk & 0xffff0000u);
-                    s[c >> 1] = pk;
-                }
+                    for (int c = h * 64; c < h * 64 + 64; c += 8) {
+                        float e[8];
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t(&chunk)[8] = *reinterpret_cast<uint32_t(*)[8]>(&s[8 * c]);
-                    if (h * 64 + c * 16 < bn) ptx::tcgen05_st_32x32b(t_s + h * 32 + c * 8, chunk);
+                        for (int i = 0; i < 8; ++i) e[i] = ex2(fmaf(__uint_as_float(s[c + i]), scale, neg_max));
+                        // the row sum takes the rounded values the PV MMA will really use, so
+                        // that O / sum stays a true weighted mean of V rows
+                        const uint32_t k0 = pack_bf16(e[0], e[1]), k1 = pack_bf16(e[2], e[3]);
+                        const uint32_t k2 = pack_bf16(e[4], e[5]), k3 = pack_bf16(e[6], e[7]);
+                        sum0 += __uint_as_float(k0 << 16) + __uint_as_float(k0 & 0xffff0000u);
+                        sum1 += __uint_as_float(k1 << 16) + __uint_as_float(k1 & 0xffff0000u);
+                        sum2 += __uint_as_float(k2 << 16) + __uint_as_float(k2 & 0xffff0000u);
+                        sum3 += __uint_as_float(k3 << 16) + __uint_as_float(k3 & 0xffff0000u);
+                        s[(c >> 1) + 0] = k0;
+                        s[(c >> 1) + 1] = k1;
+                        s[(c >> 1) + 2] = k2;
+                        s[(c >> 1) + 3] = k3;
+                    }
+                    if (bn >= h * 64 + 64) {
+                        uint32_t(&half)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[32 * h]);
+                        ptx::tcgen05_st_32x32b(t_s + h * 32, half);
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t(&chunk)[8] = *reinterpret_cast<uint32_t(*)[8]>(&s[32 * h + 8 * c]);
+                            if (h * 64 + c * 16 < bn) ptx::tcgen05_st_32x32b(t_s + h * 32 + c * 8, chunk);
+                        }
+                    }
+                    tc_wait_st();
                 }
+                tc_fence_before();
+                mbar_arrive(bars + 8 * ((h == 0 ? BAR_P_LO : BAR_P_HI) + m));
+                if (row == 0) TRACE(2 + m, j, 4 + h);
             }
-            row_sum += sum;
-            tc_wait_st();
-            tc_fence_before();
-            mbar_arrive(bars + 8 * (BAR_P_FULL + m));
+            row_sum += (sum0 + sum1) + (sum2 + sum3);
         }
 
         // epilogue: O / row_sum -> bf16 -> global memory
@@ -547,7 +616,7 @@ attention_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_consta
     if (threadIdx.x == 0) {
         const uint32_t bars = smem_u32(ctl->bars);
         for (int i = 0; i < BAR_COUNT; ++i) {
-            const bool many = (i >= BAR_P_FULL && i < BAR_P_FULL + 2) || (i >= BAR_O_FREE && i < BAR_O_FREE + 2);
+            const bool many = (i >= BAR_P_LO && i < BAR_P_HI + 2) || (i >= BAR_O_FREE && i < BAR_O_FREE + 2);
             mbar_init(bars + 8 * i, many ? 128 : 1);
         }
         ctl->abort = 0;
@@ -570,7 +639,7 @@ attention_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_consta
     if (warp < 4) {
         reg_dec<64>();
         if (warp == 0) producer_role<D>(p, maps, ctl, smem_base, begin, count, lane);
-        else if (warp == 1) mma_role<D>(p, ctl, smem_base, tmem, begin, count, lane);
+        else if (warp == 1) mma_role<D>(p, ctl, smem_base, tmem, begin, count);
     } else {
         reg_inc<216>();
         const int m = (warp - 4) >> 2;

@@ -292,6 +292,16 @@ bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) %
 
 }  // namespace
 
+#ifdef VORTA_TRACE
+static long long *g_vorta_trace = nullptr;
+extern "C" __attribute__((visibility("default"))) int vorta_debug_trace(long long *out_host)
+{
+    if (!g_vorta_trace) return 1;
+    cudaDeviceSynchronize();
+    return cudaMemcpy(out_host, g_vorta_trace, 4 * 8 * 8 * sizeof(long long), cudaMemcpyDeviceToHost) != cudaSuccess;
+}
+#endif
+
 // ------------------------------------------------------------------------------------
 extern "C" {
 
@@ -596,6 +606,15 @@ int vorta_routed_attention(const vorta_plan *p, const void *Q, const void *K, co
     prm.kv_list = p->d_kv_list; prm.colmasks = p->d_colmasks;
     prm.O = o; prm.Oc = Oc; prm.Q = q; prm.K = k; prm.V = v; prm.Qc = Qc; prm.Kc = Kc; prm.Vc = Vc;
     prm.status = p->d_status;
+#ifdef VORTA_TRACE
+    {
+        static long long *d_trace = nullptr;
+        if (!d_trace) cudaMalloc(&d_trace, 4 * 8 * 8 * sizeof(long long));
+        cudaMemsetAsync(d_trace, 0, 4 * 8 * 8 * sizeof(long long), s);
+        prm.trace = d_trace;
+        g_vorta_trace = d_trace;
+    }
+#endif
 
     AttnMaps maps;
     std::memset(&maps, 0, sizeof(maps));

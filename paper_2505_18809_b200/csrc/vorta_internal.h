@@ -74,6 +74,9 @@ struct AttnParams {
     const __nv_bfloat16 *Q, *K, *V;     // originals (SIMT kernel)
     const __nv_bfloat16 *Qc, *Kc, *Vc;  // gathered (SIMT kernel)
     int32_t *status;               // device word: 0 or the code of an expired wait
+#ifdef VORTA_TRACE
+    long long *trace;              // [4 roles][8 blocks][8 events] cycle stamps of CTA 0 (debug builds)
+#endif
 };
 
 // ---- launchers (each returns cudaGetLastError of its launch) ----------------------
