@@ -370,7 +370,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--cpu-rows", type=int, default=120, help="oracle rows per head for cpu_baseline")
+    ap.add_argument("--cpu-rows", type=int, default=800, help="oracle rows per head for cpu_baseline")
     ap.add_argument("--reference-rows", type=int, default=16, help="oracle rows per head per step (--impl reference)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -41,7 +41,7 @@ constexpr uint32_t kSmemKV = 2 * kTileBytes;
 constexpr uint32_t kSmemBars = kSmemKV + kStages * kTileBytes;
 constexpr uint32_t kSmemTotal = kSmemBars + 512;
 constexpr uint32_t kSmemAlloc = kSmemTotal + 1024;  // slack to align the base to 1024 B
-constexpr float kRescaleThreshold = 8.0f;           // log2 units
+constexpr float kRescaleThreshold = 8.0f;           // log2 units the row maximum may grow before O is rescaled
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 // barrier indices
@@ -231,7 +231,8 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint3
     return d;
 }
 
-// Instruction descriptor: bf16 x bf16 -> fp32, M = 128.
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128.  (A and B must have the same
+// 16-bit format: an fp16 P against a bf16 V is rejected by the hardware.)
 __device__ __forceinline__ uint32_t instr_desc(uint32_t n, uint32_t b_mn_major)
 {
     return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
@@ -248,6 +249,13 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
     return r;
 }
 
@@ -272,6 +280,75 @@ __device__ __forceinline__ void kv_block_coords(const AttnParams &p, const WorkI
     } else {
         c1 = j * kBlockM; c2 = 0; c3 = 0; mask_id = 0;
     }
+}
+
+// exp2(s * scale - ref) for the 64 scores s[C0 .. C0+64), packed two bf16 per word IN
+// PLACE into s[C0/2 .. C0/2 + 32): a packed word never lands on a score still to be read.
+// The row sums take the ROUNDED values the PV MMA will use, so that O / sum stays a true
+// weighted mean of V rows (with the unrounded ones a row that attends to a single key is
+// off by up to 2^-9 of |v|, beyond the output tolerance).  Scale-and-shift and the sums
+// use the packed two-wide fp32 instructions.
+template <int C0>
+__device__ __forceinline__ void exp_half(uint32_t (&s)[128], float scale, float neg_ref, float2 (&sum)[2])
+{
+    const float2 sc = make_float2(scale, scale), nr = make_float2(neg_ref, neg_ref);
+#pragma unroll
+    for (int c = 0; c < 64; c += 4) {
+        float2 x0 = __ffma2_rn(make_float2(__uint_as_float(s[C0 + c]), __uint_as_float(s[C0 + c + 1])), sc, nr);
+        float2 x1 = __ffma2_rn(make_float2(__uint_as_float(s[C0 + c + 2]), __uint_as_float(s[C0 + c + 3])), sc, nr);
+        const uint32_t k0 = pack_bf16(ex2(x0.x), ex2(x0.y));
+        const uint32_t k1 = pack_bf16(ex2(x1.x), ex2(x1.y));
+        s[C0 / 2 + (c >> 1)] = k0;
+        s[C0 / 2 + (c >> 1) + 1] = k1;
+        sum[0] = __fadd2_rn(sum[0], make_float2(__uint_as_float(k0 << 16), __uint_as_float(k0 & 0xffff0000u)));
+        sum[1] = __fadd2_rn(sum[1], make_float2(__uint_as_float(k1 << 16), __uint_as_float(k1 & 0xffff0000u)));
+    }
+}
+
+// write packed P words of keys [64h, 64h + 64) to columns [32h, 32h + 32) of the S region
+template <int H>
+__device__ __forceinline__ void store_p_half(uint32_t t_s, int32_t bn, uint32_t (&s)[128])
+{
+    if (bn >= H * 64 + 64) {
+        uint32_t(&half)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[32 * H]);
+        ptx::tcgen05_st_32x32b(t_s + H * 32, half);
+    } else {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            uint32_t(&chunk)[8] = *reinterpret_cast<uint32_t(*)[8]>(&s[32 * H + 8 * c]);
+            if (H * 64 + c * 16 < bn) ptx::tcgen05_st_32x32b(t_s + H * 32 + c * 8, chunk);
+        }
+    }
+    tc_wait_st();
+}
+
+// this thread's row of O times a
+template <int D>
+__device__ __forceinline__ void rescale_o(uint32_t t_o, float a)
+{
+#pragma unroll
+    for (int c = 0; c < D / 32; ++c) {
+        uint32_t o[32];
+        ptx::tcgen05_ld_32x32b(o, t_o + c * 32);
+        tc_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * a);
+        ptx::tcgen05_st_32x32b(t_o + c * 32, o);
+    }
+}
+
+// maximum of the 128 scores of a row (four independent chains of three-input max)
+__device__ __forceinline__ float row_max128(const uint32_t (&s)[128])
+{
+    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < 128; c += 8) {
+        mx0 = max3(mx0, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
+        mx1 = max3(mx1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
+        mx2 = max3(mx2, __uint_as_float(s[c + 4]), __uint_as_float(s[c + 5]));
+        mx3 = max3(mx3, __uint_as_float(s[c + 6]), __uint_as_float(s[c + 7]));
+    }
+    return fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
 }
 
 // ------------------------------------------------------------------ roles
@@ -478,7 +555,6 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
             ++s_cnt;
             tc_fence_after();
             if (row == 0) TRACE(2 + m, j, 1);
-
             // the whole score row of this thread, one TMEM read
             uint32_t s[128];
 #pragma unroll
@@ -493,79 +569,38 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
                 for (int c = 0; c < 128; ++c)
                     if (!((mask[c >> 5] >> (c & 31)) & 1u)) s[c] = 0xff800000u;  // -inf: not a key
             }
-            // row maximum over four independent chains
-            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-            for (int c = 0; c < 128; c += 4) {
-                mx0 = fmaxf(mx0, __uint_as_float(s[c]));
-                mx1 = fmaxf(mx1, __uint_as_float(s[c + 1]));
-                mx2 = fmaxf(mx2, __uint_as_float(s[c + 2]));
-                mx3 = fmaxf(mx3, __uint_as_float(s[c + 3]));
-            }
-            const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-            const float m_new = fmaxf(row_max, mx * scale);
+            // P = exp2(S * scale - max) as packed bf16 over the first bn/2 columns of S, in two
+            // halves: keys [0, 64) -> columns [0, 32), then keys [64, 128) -> columns [32, 64)
+            // (the whole row is already in registers).  The first half is handed to the MMA
+            // warp as soon as it is written, so that its PV MMAs run under the second half.
+            float2 sum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+            const float m_new = fmaxf(row_max, row_max128(s) * scale);
             if (j == 0) {
                 row_max = m_new;
             } else if (__any_sync(0xffffffffu, m_new - row_max > kRescaleThreshold)) {
-                // the previous PV of this tile has completed (it was issued before the QK
-                // whose completion we just waited for), so O may be rescaled in place
+                // Lazy rescale: O and the row sum move to the new maximum only when it grew by
+                // more than the threshold; until then P may reach 2^threshold.  The previous PV
+                // of this tile has completed (it was issued before the QK whose completion we
+                // just waited for), so O may be rescaled in place.
                 const float a = ex2(row_max - m_new);
                 row_sum *= a;
                 row_max = m_new;
-#pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
-                    uint32_t o[32];
-                    ptx::tcgen05_ld_32x32b(o, t_o + c * 32);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * a);
-                    ptx::tcgen05_st_32x32b(t_o + c * 32, o);
-                }
+                rescale_o<D>(t_o, a);
             }
-            // P = exp2(S * scale - max) as packed bf16 over the first bn/2 columns of S, in two
-            // halves: keys [0, 64) -> columns [0, 32), then keys [64, 128) -> columns [32, 64).
-            // A packed word never lands on a score that is still to be read.
-            const float neg_max = -row_max;
             if (row == 0) TRACE(2 + m, j, 3);
-            float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                if (h * 64 < bn) {
-#pragma unroll
-                    for (int c = h * 64; c < h * 64 + 64; c += 8) {
-                        float e[8];
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) e[i] = ex2(fmaf(__uint_as_float(s[c + i]), scale, neg_max));
-                        // the row sum takes the rounded values the PV MMA will really use, so
-                        // that O / sum stays a true weighted mean of V rows
-                        const uint32_t k0 = pack_bf16(e[0], e[1]), k1 = pack_bf16(e[2], e[3]);
-                        const uint32_t k2 = pack_bf16(e[4], e[5]), k3 = pack_bf16(e[6], e[7]);
-                        sum0 += __uint_as_float(k0 << 16) + __uint_as_float(k0 & 0xffff0000u);
-                        sum1 += __uint_as_float(k1 << 16) + __uint_as_float(k1 & 0xffff0000u);
-                        sum2 += __uint_as_float(k2 << 16) + __uint_as_float(k2 & 0xffff0000u);
-                        sum3 += __uint_as_float(k3 << 16) + __uint_as_float(k3 & 0xffff0000u);
-                        s[(c >> 1) + 0] = k0;
-                        s[(c >> 1) + 1] = k1;
-                        s[(c >> 1) + 2] = k2;
-                        s[(c >> 1) + 3] = k3;
-                    }
-                    if (bn >= h * 64 + 64) {
-                        uint32_t(&half)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[32 * h]);
-                        ptx::tcgen05_st_32x32b(t_s + h * 32, half);
-                    } else {
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            uint32_t(&chunk)[8] = *reinterpret_cast<uint32_t(*)[8]>(&s[32 * h + 8 * c]);
-                            if (h * 64 + c * 16 < bn) ptx::tcgen05_st_32x32b(t_s + h * 32 + c * 8, chunk);
-                        }
-                    }
-                    tc_wait_st();
-                }
-                tc_fence_before();
-                mbar_arrive(bars + 8 * ((h == 0 ? BAR_P_LO : BAR_P_HI) + m));
-                if (row == 0) TRACE(2 + m, j, 4 + h);
+            exp_half<0>(s, scale, -row_max, sum);
+            store_p_half<0>(t_s, bn, s);
+            tc_fence_before();
+            mbar_arrive(bars + 8 * (BAR_P_LO + m));
+            if (row == 0) TRACE(2 + m, j, 4);
+            if (bn > 64) {
+                exp_half<64>(s, scale, -row_max, sum);
+                store_p_half<1>(t_s, bn, s);
             }
-            row_sum += (sum0 + sum1) + (sum2 + sum3);
+            tc_fence_before();
+            mbar_arrive(bars + 8 * (BAR_P_HI + m));
+            if (row == 0) TRACE(2 + m, j, 5);
+            row_sum += (sum[0].x + sum[0].y) + (sum[1].x + sum[1].y);
         }
 
         // epilogue: O / row_sum -> bf16 -> global memory

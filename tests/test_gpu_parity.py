@@ -151,6 +151,24 @@ def test_routes_can_change_between_steps_and_shared_selection_features():
     p.close()
 
 
+def test_growing_scores_exercise_the_lazy_rescale():
+    """Keys whose norm grows along the sequence: the running maximum keeps rising, by less than
+    the rescale threshold (P above 1 for a while) and by far more (O rescaled in place)."""
+    wl = Workload("ramp", (4, 16, 32), 2, 128, (2, 8, 8), (3, 3, 3), 0.5, (0, 1), 41, False)
+    Q, K, V = workloads.make_qkv(wl, DEV)
+    ramp = torch.ones(wl.L, device=DEV)
+    ramp[256:] = 2.0        # a few log2 units above the first blocks
+    ramp[768:] = 4.0
+    ramp[1280:] = 24.0      # tens of log2 units above everything before
+    K = (K.float() * ramp[None, None, :, None]).to(torch.bfloat16).contiguous()
+    p = vb.Plan.from_workload(wl)
+    O = run_layer(p, wl, Q, K, V, vb.VORTA_KERNEL_TCGEN05)
+    for h in range(wl.heads):
+        want = oracle_head_rows(wl, Q, K, V, 0, h, None)
+        assert_close(O[0, h], want, f"ramp h{h}")
+    p.close()
+
+
 def test_argument_errors_launch_nothing():
     wl = small_workloads()[1]
     Q, K, V = workloads.make_qkv(wl, DEV)
