@@ -183,6 +183,34 @@ VORTA_API int vorta_routed_attention_host(const vorta_plan *plan, const void *Q_
                                           void *dev_scratch, size_t dev_scratch_bytes, void *stream);
 
 /*
+ * The same layer for callers that cannot allocate device memory -- code running
+ * inside another framework's memory pool with no spare capacity, plug-ins that are
+ * handed fixed tensors and forbidden to call cudaMalloc, services with a frozen
+ * memory budget.  (The paper has no counterpart: this is an interface convenience.)
+ * It behaves like vorta_routed_attention, but the core-set branch's scratch is a
+ * fixed array inside the library of VORTA_STATIC_WORKSPACE_BYTES bytes, which every
+ * GPU that loads the library holds until the process exits.
+ *   - Plans whose vorta_plan_info().workspace_bytes exceeds that size are refused
+ *     with VORTA_ERR_WORKSPACE and nothing is launched.
+ *   - The call itself allocates nothing (no cudaMalloc/cudaFree, no allocating
+ *     library routine).  The first call on each device looks up the array's device
+ *     address (cudaGetSymbolAddress with that device current); make that first call
+ *     before starting any stream capture.
+ *   - All calls on a device share the one array.  It keeps whatever the last call
+ *     left in it; nothing in it needs clearing, because every region is written
+ *     before it is read within a call.  Two calls whose kernels overlap on the GPU
+ *     (different streams, no ordering between them) race on it: order them.
+ * Q, K, V, O, X_or_null, Hx and stream are as for vorta_routed_attention.
+ */
+#define VORTA_STATIC_WORKSPACE_BYTES (16u * 1024u * 1024u)
+VORTA_API int vorta_routed_attention_static(const vorta_plan *plan, const void *Q, const void *K,
+                                            const void *V, void *O, const void *X_or_null, int32_t Hx,
+                                            void *stream);
+
+/* CUDA device ordinal the plan's tables live on (-1 for a host-only plan). */
+VORTA_API int vorta_plan_device(const vorta_plan *plan, int32_t *device);
+
+/*
  * Stage timing.  With profiling on, vorta_routed_attention records CUDA events
  * on its stream around its four stages.  After the stream has been synchronised,
  * vorta_plan_stage_ms returns the last call's durations in milliseconds:

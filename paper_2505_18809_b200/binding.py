@@ -28,8 +28,9 @@ EXPORTS = (
     "vorta_plan_block_mask", "vorta_plan_set_kernel", "vorta_coreset_select",
     "vorta_routed_attention", "vorta_routed_attention_host", "vorta_plan_set_profiling",
     "vorta_plan_stage_ms", "vorta_plan_stage_ms_at", "vorta_plan_last_launches", "vorta_device_status",
-    "vorta_status_string",
+    "vorta_status_string", "vorta_routed_attention_static", "vorta_plan_device",
 )
+VORTA_STATIC_WORKSPACE_BYTES = 16 * 1024 * 1024
 
 
 class vorta_plan_desc(ctypes.Structure):
@@ -78,6 +79,8 @@ def lib() -> ctypes.CDLL:
     L.vorta_coreset_select.argtypes = [vp, vp, i32, i32, vp, vp, vp]
     L.vorta_routed_attention.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp, ctypes.c_size_t, vp]
     L.vorta_routed_attention_host.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+    L.vorta_routed_attention_static.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp]
+    L.vorta_plan_device.argtypes = [vp, ctypes.POINTER(i32)]
     L.vorta_plan_set_profiling.argtypes = [vp, i32]
     L.vorta_plan_stage_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float * 4)]
     L.vorta_plan_stage_ms_at.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_float * 4)]
@@ -159,6 +162,19 @@ def vorta_routed_attention_host(plan: int, Q_ptr: int, K_ptr: int, V_ptr: int, O
     _check(lib().vorta_routed_attention_host(plan, Q_ptr, K_ptr, V_ptr, O_ptr, scratch_ptr,
                                              scratch_bytes, stream),
            "vorta_routed_attention_host")
+
+
+def vorta_routed_attention_static(plan: int, Q_ptr: int, K_ptr: int, V_ptr: int, O_ptr: int,
+                                  X_ptr: Optional[int] = None, Hx: int = 0, stream: int = 0) -> None:
+    """The layer with the library's built-in scratch array: for callers that may not allocate."""
+    _check(lib().vorta_routed_attention_static(plan, Q_ptr, K_ptr, V_ptr, O_ptr, X_ptr, Hx, stream),
+           "vorta_routed_attention_static")
+
+
+def vorta_plan_device(plan: int) -> int:
+    d = ctypes.c_int32()
+    _check(lib().vorta_plan_device(plan, ctypes.byref(d)), "vorta_plan_device")
+    return d.value
 
 
 def vorta_plan_set_profiling(plan: int, on: bool) -> None:

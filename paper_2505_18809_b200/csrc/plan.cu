@@ -506,6 +506,13 @@ int vorta_plan_info(const vorta_plan *p, vorta_plan_info_t *o)
     return VORTA_OK;
 }
 
+int vorta_plan_device(const vorta_plan *p, int32_t *device)
+{
+    if (!p || !device) return VORTA_ERR_INVALID_ARG;
+    *device = p->host_only ? -1 : p->device;
+    return VORTA_OK;
+}
+
 int vorta_plan_block_mask(const vorta_plan *p, uint8_t *out_host)
 {
     if (!p || !out_host) return VORTA_ERR_INVALID_ARG;
