@@ -168,6 +168,24 @@ def time_oracle(wl, Q, K, V, rows_per_head: int, budget_s: float, seed: int = 0)
     return flops, t_total, heads_done, oracle.num_threads()
 
 
+# ----------------------------------------------------------------------------- multi-rank aggregation
+def reduce_max_ms(ms_local: float, world: int, device) -> float:
+    """The job's time is the slowest rank's: max-reduce over the process group (if any)."""
+    if world <= 1:
+        return float(ms_local)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms_local], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tflops(flops_per_rank_step: float, world: int, ms_per_step: float) -> float:
+    """Every rank runs its own layer (heads are independent, nothing is exchanged): the job's
+    throughput is the work of all ranks over the slowest rank's time."""
+    return world * flops_per_rank_step / (ms_per_step * 1e-3) / 1e12
+
+
 # ----------------------------------------------------------------------------- arms
 def run_reference(args):
     """The oracle as the timed arm: each step is a bounded sample of rows of the workload."""
@@ -270,12 +288,9 @@ def run_ours(args):
     ms_total = e0.elapsed_time(e1)
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
     assert plan.device_status() == 0
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = reduce_max_ms(ms_total, world, dev)
     ms_step = ms_total / args.steps
-    value = world * info.flops_layer / (ms_step * 1e-3) / 1e12
+    value = whole_job_tflops(info.flops_layer, world, ms_step)
 
     # stage times of the timed steps (CUDA events recorded by the library on the same stream)
     n_hist = min(args.steps, 64)
@@ -330,13 +345,9 @@ def run_ours(args):
             plan.routed_attention_host(Qh, Kh, Vh, Oh, scratch)
         e1.record(stream)
         barrier()
-        ms_e2e = e0.elapsed_time(e1) / n_e2e
-        if world > 1:
-            t = torch.tensor([ms_e2e], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
+        ms_e2e = reduce_max_ms(e0.elapsed_time(e1) / n_e2e, world, dev)
         tb = Q.numel() * 2
-        e2e = {"value": world * info.flops_layer / (ms_e2e * 1e-3) / 1e12, "unit": UNIT,
+        e2e = {"value": whole_job_tflops(info.flops_layer, world, ms_e2e), "unit": UNIT,
                "ms_per_step": ms_e2e, "steps": n_e2e, "h2d_bytes_per_step": 3 * tb, "d2h_bytes_per_step": tb,
                "api": "vorta_routed_attention_host (pinned host Q, K, V in; O out)"}
         del scratch, Qh, Kh, Vh

@@ -27,6 +27,7 @@ struct vorta_plan {
     int32_t *d_kv_count = nullptr;
     uint32_t *d_colmasks = nullptr;
     int32_t *d_seg_start = nullptr;
+    int32_t *d_bucket_tab = nullptr;  // [8 shape classes][kBucketTabStride]
     WorkItem *d_items = nullptr;
     int32_t *d_cta_begin = nullptr, *d_cta_count = nullptr;
     int32_t *d_core_slice = nullptr;  // [B * n_core]: compact problem -> b*heads + head
@@ -118,7 +119,7 @@ int64_t tensor_bytes(const Geometry &g) { return (int64_t)g.B * g.heads * g.L * 
 void free_device(vorta_plan *p)
 {
     cudaFree(p->d_bm); cudaFree(p->d_kv_list); cudaFree(p->d_kv_count); cudaFree(p->d_colmasks);
-    cudaFree(p->d_seg_start); cudaFree(p->d_items); cudaFree(p->d_cta_begin);
+    cudaFree(p->d_seg_start); cudaFree(p->d_bucket_tab); cudaFree(p->d_items); cudaFree(p->d_cta_begin);
     cudaFree(p->d_cta_count); cudaFree(p->d_core_slice); cudaFree(p->d_core_xslice);
     cudaFree(p->d_status);
     for (auto &set : p->ev)
@@ -420,6 +421,27 @@ int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
         }
     }
 
+    // bucket shape classes (bit 2: cut on T, bit 1: on H, bit 0: on W): token count, centre,
+    // and the token offset of every local index from the bucket's first token
+    std::vector<int32_t> btab((size_t)8 * kBucketTabStride, 0);
+    for (int32_t cls = 0; cls < 8; ++cls) {
+        int32_t e[3];
+        for (int a = 0; a < 3; ++a) {
+            bool cut = (cls >> (2 - a)) & 1;
+            int32_t rem = dim[a] - (g.nb[a] - 1) * g.bucket[a];
+            e[a] = cut ? rem : g.bucket[a];
+        }
+        int32_t n = e[0] * e[1] * e[2];
+        if (n > 32) continue;  // only used for buckets of at most 32 tokens
+        int32_t *t = &btab[(size_t)cls * kBucketTabStride];
+        t[0] = n;
+        t[1] = ((e[0] / 2) * e[1] + (e[1] / 2)) * e[2] + (e[2] / 2);
+        for (int32_t l = 0; l < n; ++l) {
+            int32_t lw = l % e[2], lh = (l / e[2]) % e[1], lt = l / (e[2] * e[1]);
+            t[2 + l] = (lt * g.H + lh) * g.W + lw;
+        }
+    }
+
     bool ok = true;
     int64_t nt2 = (int64_t)g.n_tiles * g.n_tiles;
     ok = ok && cudaMalloc(&p->d_bm, (size_t)nt2) == cudaSuccess;
@@ -427,6 +449,8 @@ int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
     ok = ok && cudaMalloc(&p->d_kv_count, sizeof(int32_t) * g.n_tiles) == cudaSuccess;
     ok = ok && cudaMalloc(&p->d_colmasks, sizeof(uint32_t) * masks.size()) == cudaSuccess;
     ok = ok && cudaMalloc(&p->d_seg_start, sizeof(int32_t) * g.n_buckets) == cudaSuccess;
+    ok = ok && cudaMalloc(&p->d_bucket_tab, sizeof(int32_t) * btab.size()) == cudaSuccess;
+    ok = ok && cudaMemcpy(p->d_bucket_tab, btab.data(), sizeof(int32_t) * btab.size(), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMalloc(&p->d_cta_begin, sizeof(int32_t) * p->sm_count) == cudaSuccess;
     ok = ok && cudaMalloc(&p->d_cta_count, sizeof(int32_t) * p->sm_count) == cudaSuccess;
     ok = ok && cudaMalloc(&p->d_core_slice, sizeof(int32_t) * (size_t)g.B * g.heads) == cudaSuccess;
@@ -572,7 +596,7 @@ int vorta_coreset_select(const vorta_plan *p, const void *X, int32_t Hx, int32_t
     DeviceGuard guard(p->device);
     if (!guard.ok) return VORTA_ERR_CUDA;
     cudaError_t e = launch_select(p->g, static_cast<const __nv_bfloat16 *>(X), dx, p->g.B * Hx, nullptr,
-                                  p->d_seg_start, core_idx, src_slot, static_cast<cudaStream_t>(stream));
+                                  p->d_seg_start, p->d_bucket_tab, core_idx, src_slot, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? VORTA_OK : VORTA_ERR_CUDA;
 }
 
@@ -657,7 +681,7 @@ int vorta_routed_attention(const vorta_plan *p, const void *Q, const void *K, co
     if (n_prob) {
         const __nv_bfloat16 *xs = X ? static_cast<const __nv_bfloat16 *>(X) : k;
         const int32_t *xslice = (X && Hx == 1) ? p->d_core_xslice : p->d_core_slice;
-        e = launch_select(g, xs, g.d, n_prob, xslice, p->d_seg_start, core_idx, src_slot, s);
+        e = launch_select(g, xs, g.d, n_prob, xslice, p->d_seg_start, p->d_bucket_tab, core_idx, src_slot, s);
         if (e != cudaSuccess) return VORTA_ERR_CUDA;
         ++launches;
     }

@@ -200,15 +200,208 @@ coreset_select_kernel(Geometry g, const __nv_bfloat16 *__restrict__ X, int32_t d
     src_slot[(int64_t)p * g.L + tok] = slot;
 }
 
+// The same selection for the common case dx = 128 and buckets of at most 12 tokens
+// (the paper's (2, 3, 2)).  Every lane first issues the loads of all its chunks -- its
+// share of the centre row and of the three token rows it helps to score -- so that a
+// warp has the whole bucket in flight before any arithmetic.
+//
+// Scores are first taken in fp32 (products of bf16 values are exact there; the sums of
+// 128 terms are not): each cosine is then within 2.5e-5 of its true value.  Only the SET
+// of pruned tokens matters, i.e. the order of the k-th and (k+1)-th largest scores, so
+// the fp32 ranking is accepted when those two are at least 2^-13 apart.  Otherwise --
+// near-ties, exact ties, rows with a vanishing or non-finite squared norm in fp32 -- the
+// bucket is scored again in fp64 with the formula of the general kernel, from the same
+// registers, and ranked on those scores.  The results are those of the general kernel.
+__device__ __forceinline__ void bf16x8_to_f32(const uint4 &u, float out[8])
+{
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        out[2 * i] = __uint_as_float(w[i] << 16);
+        out[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+}
+
+__global__ void __launch_bounds__(256, 4)
+coreset_select_d128_kernel(Geometry g, const __nv_bfloat16 *__restrict__ X, const int32_t *__restrict__ prob_slice,
+                           const int32_t *__restrict__ seg_start, const int32_t *__restrict__ bucket_tab,
+                           int32_t *__restrict__ core_idx, int32_t *__restrict__ src_slot)
+{
+    constexpr int32_t dx = 128, kPasses = 3;
+    constexpr float kGuard = 1.220703125e-4f;  // 2^-13
+    // bucket shape classes (which axes the grid cuts): token count, centre, token offsets
+    __shared__ int32_t tab[8 * kBucketTabStride];
+    for (int i = threadIdx.x; i < 8 * kBucketTabStride; i += blockDim.x) tab[i] = bucket_tab[i];
+    __syncthreads();
+
+    const int lane = threadIdx.x & 31;
+    const int32_t bkt = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (bkt >= g.n_buckets) return;
+    const int32_t p = blockIdx.y;
+    const int32_t slice = prob_slice ? prob_slice[p] : p;
+    const __nv_bfloat16 *Xs = X + (int64_t)slice * g.L * dx;
+
+    const int32_t bt = bkt / (g.nb[2] * g.nb[1]), bhw = bkt - bt * (g.nb[2] * g.nb[1]);
+    const int32_t bh = bhw / g.nb[2], bw = bhw - bh * g.nb[2];
+    const int32_t cls = ((g.T - bt * g.bucket[0] < g.bucket[0]) ? 4 : 0) | ((g.H - bh * g.bucket[1] < g.bucket[1]) ? 2 : 0) |
+                        ((g.W - bw * g.bucket[2] < g.bucket[2]) ? 1 : 0);
+    const int32_t *t = tab + cls * kBucketTabStride;
+    const int32_t n = t[0], centre = t[1];
+    const int32_t origin = (bt * g.bucket[0] * g.H + bh * g.bucket[1]) * g.W + bw * g.bucket[2];
+    auto token_of = [&](int32_t l) -> int32_t { return origin + t[2 + l]; };
+
+    const int sub = lane >> 3, sl = lane & 7;
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+    const uint4 *xc = reinterpret_cast<const uint4 *>(Xs + (int64_t)token_of(centre) * dx);
+    const uint4 c0 = __ldg(xc + sl), c1 = __ldg(xc + sl + 8);
+    uint4 r[kPasses][2];
+#pragma unroll
+    for (int pass = 0; pass < kPasses; ++pass) {
+        const int32_t l = pass * 4 + sub;
+        r[pass][0] = zero;
+        r[pass][1] = zero;
+        if (l < n) {
+            const uint4 *xj = reinterpret_cast<const uint4 *>(Xs + (int64_t)token_of(l) * dx);
+            r[pass][0] = __ldg(xj + sl);
+            r[pass][1] = __ldg(xj + sl + 8);
+        }
+    }
+
+    int32_t keep = (int32_t)floor(g.ratio * (double)n + 0.5);
+    keep = max(keep, 1);
+    const int32_t k = n - keep;
+    const bool is_tok = lane < n, is_centre = lane == centre;
+
+    // ---- fp32 scores and ranks
+    float my32 = 0.f;
+    bool doubtful = false;
+    {
+        float csq = 0.f;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            float a[8];
+            bf16x8_to_f32(h ? c1 : c0, a);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) csq = fmaf(a[i], a[i], csq);
+        }
+#pragma unroll
+        for (int m = 4; m >= 1; m >>= 1) csq += __shfl_xor_sync(0xffffffffu, csq, m);
+        doubtful = !(csq > 1e-30f && csq < 1e30f);
+#pragma unroll
+        for (int pass = 0; pass < kPasses; ++pass) {
+            if (pass * 4 >= n) break;  // warp-uniform
+            float dot = 0.f, njsq = 0.f;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                float a[8], b[8];
+                bf16x8_to_f32(h ? c1 : c0, a);
+                bf16x8_to_f32(r[pass][h], b);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    dot = fmaf(a[i], b[i], dot);
+                    njsq = fmaf(b[i], b[i], njsq);
+                }
+            }
+#pragma unroll
+            for (int m = 4; m >= 1; m >>= 1) {
+                dot += __shfl_xor_sync(0xffffffffu, dot, m);
+                njsq += __shfl_xor_sync(0xffffffffu, njsq, m);
+            }
+            if (pass * 4 + sub < n && !(njsq > 1e-30f && njsq < 1e30f)) doubtful = true;
+            const float score = dot * rsqrtf(csq * njsq);
+            const float got = __shfl_sync(0xffffffffu, score, (lane & 3) * 8);
+            if ((lane >> 2) == pass) my32 = got;
+        }
+    }
+    int32_t rank = 0;
+    for (int32_t m = 0; m < n; ++m) {
+        const float sm = __shfl_sync(0xffffffffu, my32, m);
+        if (m != centre && (sm > my32 || (sm == my32 && m < lane))) ++rank;
+    }
+    bool need64 = __any_sync(0xffffffffu, doubtful);
+    if (!need64 && k > 0 && k < n - 1) {
+        // last pruned (rank k-1) against first surviving (rank k) token
+        const uint32_t b_lo = __ballot_sync(0xffffffffu, is_tok && !is_centre && rank == k - 1);
+        const uint32_t b_hi = __ballot_sync(0xffffffffu, is_tok && !is_centre && rank == k);
+        const float s_lo = __shfl_sync(0xffffffffu, my32, __ffs(b_lo) - 1);
+        const float s_hi = __shfl_sync(0xffffffffu, my32, __ffs(b_hi) - 1);
+        need64 = !(s_lo - s_hi >= kGuard);
+    }
+
+    // ---- fp64 scores and ranks for the buckets the guard band does not clear
+    if (need64) {
+        // (the summation order differs from the general kernel's only in grouping by chunk)
+        double csq = 0.0;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            double a[8];
+            bf16x8_to_f64(h ? c1 : c0, a);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) csq = fma(a[i], a[i], csq);
+        }
+#pragma unroll
+        for (int m = 4; m >= 1; m >>= 1) csq += shfl_xor_f64(csq, m);
+        const double nc = sqrt(csq);
+        double my64 = 0.0;
+#pragma unroll 1
+        for (int pass = 0; pass < kPasses; ++pass) {
+            if (pass * 4 >= n) break;
+            double dot = 0.0, njsq = 0.0;
+            const uint4 rp0 = pass == 0 ? r[0][0] : (pass == 1 ? r[1][0] : r[2][0]);
+            const uint4 rp1 = pass == 0 ? r[0][1] : (pass == 1 ? r[1][1] : r[2][1]);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                double a[8], b[8];
+                bf16x8_to_f64(h ? c1 : c0, a);
+                bf16x8_to_f64(h ? rp1 : rp0, b);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    dot = fma(a[i], b[i], dot);
+                    njsq = fma(b[i], b[i], njsq);
+                }
+            }
+#pragma unroll
+            for (int m = 4; m >= 1; m >>= 1) {
+                dot += shfl_xor_f64(dot, m);
+                njsq += shfl_xor_f64(njsq, m);
+            }
+            const double nj = sqrt(njsq);
+            const double score = (nc == 0.0 || nj == 0.0) ? 0.0 : dot / (nc * nj);
+            const double got = shfl_f64(score, (lane & 3) * 8);
+            if ((lane >> 2) == pass) my64 = got;
+        }
+        rank = 0;
+        for (int32_t m = 0; m < n; ++m) {
+            const double sm = shfl_f64(my64, m);
+            if (m != centre && (sm > my64 || (sm == my64 && m < lane))) ++rank;
+        }
+    }
+
+    const bool kept = is_tok && (is_centre || rank >= k);
+    const uint32_t kept_others = __ballot_sync(0xffffffffu, kept && !is_centre);
+    if (!is_tok) return;
+    const int32_t seg = seg_start[bkt];
+    const int32_t tok = token_of(lane);
+    int32_t slot = seg;
+    if (kept && !is_centre) slot = seg + 1 + __popc(kept_others & ((1u << lane) - 1u));
+    if (kept) core_idx[(int64_t)p * g.Lc + slot] = tok;
+    src_slot[(int64_t)p * g.L + tok] = slot;
+}
+
 cudaError_t launch_select(const Geometry &g, const __nv_bfloat16 *X, int32_t dx, int32_t n_prob,
-                          const int32_t *prob_slice, const int32_t *seg_start, int32_t *core_idx,
-                          int32_t *src_slot, cudaStream_t s)
+                          const int32_t *prob_slice, const int32_t *seg_start, const int32_t *bucket_tab,
+                          int32_t *core_idx, int32_t *src_slot, cudaStream_t s)
 {
     int64_t warps = (int64_t)n_prob * g.n_buckets;
     if (warps == 0) return cudaSuccess;
-    int64_t blocks = (warps + 7) / 8;
-    coreset_select_kernel<<<(unsigned)blocks, 256, 0, s>>>(g, X, dx, n_prob, prob_slice, seg_start,
-                                                           core_idx, src_slot);
+    if (dx == 128 && g.bucket[0] * g.bucket[1] * g.bucket[2] <= 12 && n_prob <= 65535) {
+        dim3 grid((unsigned)((g.n_buckets + 7) / 8), (unsigned)n_prob);
+        coreset_select_d128_kernel<<<grid, 256, 0, s>>>(g, X, prob_slice, seg_start, bucket_tab, core_idx, src_slot);
+    } else {
+        int64_t blocks = (warps + 7) / 8;
+        coreset_select_kernel<<<(unsigned)blocks, 256, 0, s>>>(g, X, dx, n_prob, prob_slice, seg_start,
+                                                               core_idx, src_slot);
+    }
     return cudaGetLastError();
 }
 

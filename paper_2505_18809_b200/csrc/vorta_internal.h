@@ -22,6 +22,7 @@ enum : int32_t {
 constexpr int kBlockM = 128;       // query rows per M-block (one MMA M)
 constexpr int kMaxMasks = 17;      // column-mask classes of the sliding branch (0 = none)
 constexpr int kAttnThreads = 384;  // tcgen05 kernel: 4 control warps + 2 softmax warpgroups
+constexpr int kBucketTabStride = 34;  // per bucket shape class: token count, centre, 32 token offsets
 
 // Plain geometry, passed to kernels by value.
 struct Geometry {
@@ -83,8 +84,8 @@ struct AttnParams {
 cudaError_t launch_block_mask(const Geometry &g, uint8_t *bm, KvEntry *kv_list, int32_t *kv_count,
                               cudaStream_t s);
 cudaError_t launch_select(const Geometry &g, const __nv_bfloat16 *X, int32_t dx, int32_t n_prob,
-                          const int32_t *prob_slice, const int32_t *seg_start, int32_t *core_idx,
-                          int32_t *src_slot, cudaStream_t s);
+                          const int32_t *prob_slice, const int32_t *seg_start, const int32_t *bucket_tab,
+                          int32_t *core_idx, int32_t *src_slot, cudaStream_t s);
 cudaError_t launch_gather(const Geometry &g, int32_t n_prob, const int32_t *prob_slice,
                           const int32_t *core_idx, const __nv_bfloat16 *Q, const __nv_bfloat16 *K,
                           const __nv_bfloat16 *V, __nv_bfloat16 *Qc, __nv_bfloat16 *Kc,

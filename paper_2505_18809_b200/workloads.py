@@ -73,11 +73,15 @@ def config(name: str) -> Workload:
         # counter capture of one launch stays short while the inputs still exceed L2
         return Workload(name, (33, 45, 80), 3, 128, (4, 8, 8), (3, 3, 3), 0.5,
                         (ROUTE_FULL, ROUTE_SLIDING, ROUTE_CORESET), 2, True)
+    if name == "hunyuan-720p-8c":
+        # profiling case for the memory-bound stages: eight core-set heads, nothing else
+        return Workload(name, (33, 45, 80), 8, 128, (4, 8, 8), (3, 3, 3), 0.5,
+                        (ROUTE_CORESET,) * 8, 2, True)
     raise KeyError(name)
 
 
 CONFIG_NAMES = ("tiny", "wan1.3b-480p", "hunyuan-720p", "wan14b-720p")
-PROFILE_NAMES = ("hunyuan-720p-3h",)
+PROFILE_NAMES = ("hunyuan-720p-3h", "hunyuan-720p-8c")
 
 
 def route_mix_sweep() -> List[Workload]:

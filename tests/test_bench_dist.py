@@ -1,0 +1,70 @@
+"""The multi-rank logic of bench.py on CPU (gloo, two ranks): the job's time is the slowest
+rank's, the job's throughput the work of all ranks over that time, and the reference arm
+runs on rank 0 only."""
+import os
+import socket
+import subprocess
+import sys
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+import bench  # noqa: E402
+
+
+def _free_port():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def _worker(rank, world, port, out):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    local_ms = [40.0, 52.5][rank]                      # rank 1 is the slow one
+    ms = bench.reduce_max_ms(local_ms, world, "cpu")
+    value = bench.whole_job_tflops(53.45e12, world, ms)
+    dist.barrier()
+    out[rank] = (ms, value)
+    dist.destroy_process_group()
+
+
+def test_two_ranks_report_the_slowest_time_and_the_aggregate():
+    world, port = 2, _free_port()
+    with mp.Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(_worker, args=(world, port, out), nprocs=world, join=True)
+        res = dict(out)
+    assert res[0] == res[1]
+    ms, value = res[0]
+    assert ms == 52.5
+    assert abs(value - 2 * 53.45e12 / 52.5e-3 / 1e12) < 1e-9
+
+
+def test_single_rank_needs_no_process_group():
+    assert bench.reduce_max_ms(7.0, 1, "cpu") == 7.0
+    assert abs(bench.whole_job_tflops(1e12, 1, 1.0) - 1000.0) < 1e-9
+
+
+def test_reference_arm_is_silent_on_other_ranks():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
+                        "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True, timeout=120)
+    assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def test_window_key_count_matches_the_oracle_mask():
+    # the FLOP accounting of sampled sliding rows (bench._window_keys) against the oracle's mask rows
+    import oracle
+    from paper_2505_18809_b200.workloads import Workload
+    wl = Workload("w", (5, 7, 9), 1, 64, (1, 2, 2), (3, 3, 3), 0.5, (1,), 0, False)
+    M = oracle.sta_token_mask(wl.grid, wl.tile, wl.window)
+    for tok in (0, 17, 100, wl.L - 1):
+        assert bench._window_keys(wl, tok) == int(M[tok].sum())
