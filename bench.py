@@ -36,9 +36,16 @@ METRIC = "routed_attention_effective_tflops"
 UNIT = "TFLOP/s"
 DEFAULT_WORKLOAD = "hunyuan-720p"
 FALLBACK_PEAK_TFLOPS = 1590.0   # used only if MEASURED_PEAKS.json is absent
-# DRAM bytes per attention-kernel launch from the ncu capture summarised under profiles/
-# (None until a capture of this kernel exists).
-ATTENTION_DRAM_TRAFFIC_BYTES = None
+# DRAM traffic of the attention kernel: the ncu capture of the three-head profiling case
+# (profiles/attention_sm100_kernel__hunyuan-720p-3h.md) read 477.2 MB and wrote 81.4 MB for 304.0 MB of
+# algorithmic bytes; a launch of another workload is estimated by the same ratio.
+ATTENTION_TRAFFIC_PER_ALGORITHMIC_BYTE = 558.6 / 304.0
+
+
+def attention_algorithmic_bytes(info, wl) -> float:
+    """Q, K, V read and O written once per full or sliding head; the gathered Q, K, V, O per core-set head."""
+    row = wl.d * 2
+    return wl.B * ((info.n_full + info.n_sliding) * 4.0 * info.L * row + info.n_coreset * 4.0 * info.Lc * row)
 
 
 def peaks():
@@ -308,7 +315,10 @@ def run_ours(args):
                     "frac_of_sustained": achieved / pk["bf16_sustained"] if pk["bf16_sustained"] else None,
                     "frac_of_nominal_2250": achieved / 2250.0,
                     "issued_tflops": info.flops_issued_layer / (attn_ms * 1e-3) / 1e12,
-                    "kernel_ms": attn_ms, "traffic": ATTENTION_DRAM_TRAFFIC_BYTES}
+                    "kernel_ms": attn_ms,
+                    "algorithmic_bytes": attention_algorithmic_bytes(info, wl),
+                    "traffic": ATTENTION_TRAFFIC_PER_ALGORITHMIC_BYTE * attention_algorithmic_bytes(info, wl),
+                    "traffic_source": "ncu dram bytes of the 3-head capture scaled by algorithmic bytes"}
         gbs = lambda b, ms: (b / (ms * 1e-3) / 1e9) if ms > 0 else None
         stage = {"select_ms": st[0], "gather_ms": st[1], "attention_ms": st[2], "scatter_ms": st[3],
                  "select_gbs": gbs(n_core * info.select_bytes_head, st[0]),
