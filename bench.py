@@ -269,8 +269,18 @@ def run_ours(args):
             dist.barrier()
             torch.cuda.synchronize()
 
+    flops_step = info.flops_layer
+    if args.mixture:
+        # Eq. 5: every head runs all three branches; the gates only weight the outputs
+        gates = torch.softmax(torch.randn((wl.heads, 3), device=dev), dim=1).contiguous()
+        mix_ws = torch.empty(int(info.mixture_workspace_bytes), dtype=torch.uint8, device=dev)
+        flops_step = wl.B * wl.heads * (info.flops_full_head + info.flops_sliding_head + info.flops_coreset_head)
+
     def step():
-        plan.routed_attention(Q, K, V, O, workspace=ws)
+        if args.mixture:
+            plan.soft_mixture(Q, K, V, gates, O, workspace=mix_ws)
+        else:
+            plan.routed_attention(Q, K, V, O, workspace=ws)
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -297,18 +307,23 @@ def run_ours(args):
     assert plan.device_status() == 0
     ms_total = reduce_max_ms(ms_total, world, dev)
     ms_step = ms_total / args.steps
-    value = whole_job_tflops(info.flops_layer, world, ms_step)
+    value = whole_job_tflops(flops_step, world, ms_step)
 
     # stage times of the timed steps (CUDA events recorded by the library on the same stream)
     n_hist = min(args.steps, 64)
-    stages = [plan.stage_ms(i) for i in range(n_hist)]
+    if args.mixture:
+        plan.set_profiling(True)
+        stages = [[0.0, 0.0, ms_step, 0.0]]     # the mixture call is not split into stages
+        n_hist = 1
+    else:
+        stages = [plan.stage_ms(i) for i in range(n_hist)]
     st = [sum(s[i] for s in stages) / n_hist for i in range(4)]
     attn_ms = st[2]
     n_core = info.n_coreset * wl.B
 
     out = None
     if rank == 0:
-        achieved = info.flops_layer / (attn_ms * 1e-3) / 1e12
+        achieved = flops_step / (attn_ms * 1e-3) / 1e12
         roofline = {"bound": "tensor", "kernel": "attention_sm100_kernel", "achieved": achieved,
                     "peak": pk["bf16"], "unit": UNIT, "frac": achieved / pk["bf16"],
                     "peak_source": f"{pk['source']} burst bf16",
@@ -329,7 +344,8 @@ def run_ours(args):
                "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "ms_per_layer": ms_step,
                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
                "data": "synthetic",
-               "config": {"workload": wl.name, "grid": list(wl.grid), "tokens": wl.L, "heads": wl.heads,
+               "config": {"workload": wl.name + ("+soft-mixture" if args.mixture else ""), "grid": list(wl.grid),
+                          "tokens": wl.L, "heads": wl.heads,
                           "d": wl.d, "tile": list(wl.tile), "window_tiles": list(wl.window),
                           "coreset_ratio": wl.ratio, "routes": list(wl.routes),
                           "heads_full_sliding_coreset": [info.n_full, info.n_sliding, info.n_coreset],
@@ -342,7 +358,7 @@ def run_ours(args):
 
     # ---- end to end through the host-buffer entry point (rank-local, max over ranks)
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not args.mixture:
         Qh, Kh, Vh = (torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t) for t in (Q, K, V))
         Oh = torch.empty(Q.shape, dtype=Q.dtype, pin_memory=True)
         scratch = torch.empty(int(info.host_call_scratch_bytes), dtype=torch.uint8, device=dev)
@@ -393,6 +409,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-rows", type=int, default=800, help="oracle rows per head for cpu_baseline")
     ap.add_argument("--reference-rows", type=int, default=16, help="oracle rows per head per step (--impl reference)")
+    ap.add_argument("--mixture", action="store_true", help="time vorta_soft_mixture (all three branches per head)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

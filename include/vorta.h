@@ -92,6 +92,7 @@ typedef struct {
     int64_t workspace_bytes;     /* device workspace vorta_routed_attention needs (current routes) */
     int64_t workspace_bytes_max; /* ... if every head were routed to core-set */
     int64_t host_call_scratch_bytes; /* device scratch vorta_routed_attention_host needs */
+    int64_t mixture_workspace_bytes; /* device workspace vorta_soft_mixture needs */
     /* Algorithmic work: 4*d*(query, key) pairs the method itself attends, per (batch, head). */
     double flops_full_head;      /* 4 d L^2 */
     double flops_sliding_head;   /* 4 d * sum over tile pairs in the window of valid tokens products */
@@ -181,6 +182,34 @@ VORTA_API int vorta_routed_attention(const vorta_plan *plan, const void *Q, cons
 VORTA_API int vorta_routed_attention_host(const vorta_plan *plan, const void *Q_host,
                                           const void *K_host, const void *V_host, void *O_host,
                                           void *dev_scratch, size_t dev_scratch_bytes, void *stream);
+
+/*
+ * Router (Section 3.3, Eq. 3-4).  gates[h] = softmax(T . W_R[h]) and the branch the
+ * inference rule selects for head h: sliding if its gate is strictly larger than the
+ * other two, core-set likewise, full otherwise (every tie goes to full attention).
+ *   T_dev      f32 [d_model]           timestep embedding
+ *   WR_dev     f32 [heads, d_model, 3] router weights, gate order (full, sliding, core-set)
+ *   gates_dev  f32 [heads, 3] out      routes_dev  uint8 [heads] out (device; copy to the
+ *                                      host and pass to vorta_plan_set_routes)
+ * Logits are accumulated in fp64; the rule is evaluated on the logits, which order
+ * exactly like the gates.
+ */
+VORTA_API int vorta_router_gates(const float *T_dev, const float *WR_dev, int32_t d_model, int32_t heads,
+                                 float *gates_dev, uint8_t *routes_dev, void *stream);
+
+/*
+ * Soft mixture of the three branches (Section 3.3, Eq. 5: the forward pass used to
+ * train the router): O[b, h] = g[h][0] full(.) + g[h][1] sliding(.) + g[h][2] coreset(.).
+ * Every head runs all three branches in ONE attention launch (the plan's routes are
+ * ignored), then the branch outputs are combined in fp32.
+ *   gates_dev  f32 [heads, 3], device
+ *   workspace  device, >= vorta_plan_info().mixture_workspace_bytes, 256-byte aligned
+ * Core-set selection is on K of each head.  The first call builds the work list
+ * (synchronous copies to the device).
+ */
+VORTA_API int vorta_soft_mixture(vorta_plan *plan, const void *Q, const void *K, const void *V,
+                                 const float *gates_dev, void *O, void *workspace, size_t workspace_bytes,
+                                 void *stream);
 
 /*
  * The same layer for callers that cannot allocate device memory -- code running

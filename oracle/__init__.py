@@ -11,6 +11,8 @@ from .vorta_oracle import (  # noqa: F401
     coreset_len,
     coreset_select,
     num_threads,
+    router_gates,
+    soft_mixture,
     sta_block_mask,
     sta_token_mask,
 )

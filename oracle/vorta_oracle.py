@@ -186,3 +186,32 @@ def attn_coreset(grid, bucket, ratio: float, Q, K, V, scale: float, X=None, q_ro
     if got != Lc:
         raise RuntimeError(f"vo_attn_coreset returned {got}, expected {Lc}")
     return O, core_idx, src_slot
+
+
+def router_gates(T, WR):
+    """Router of Section 3.3: gates[h] = softmax(T @ WR[h]) (Eq. 3) and the branch Eq. 4 picks.
+
+    T: [d_model]; WR: [heads, d_model, 3], gate order (full, sliding, core-set).  Returns
+    (gates float64 [heads, 3], routes uint8 [heads]): sliding if its gate is strictly above
+    both others, core-set likewise, full otherwise.
+    """
+    T = _f64(T)
+    WR = _f64(WR)
+    logits = np.einsum("c,hcr->hr", T, WR)
+    logits = logits - logits.max(axis=1, keepdims=True)
+    e = np.exp(logits)
+    gates = e / e.sum(axis=1, keepdims=True)
+    routes = np.zeros(gates.shape[0], dtype=np.uint8)
+    a1, a2, a3 = gates[:, 0], gates[:, 1], gates[:, 2]
+    routes[(a2 > a1) & (a2 > a3)] = 1
+    routes[(a3 > a1) & (a3 > a2)] = 2
+    return gates, routes
+
+
+def soft_mixture(grid, tile, window, bucket, ratio, Q, K, V, scale, gates, q_rows=None):
+    """Eq. 5 for one head: gates[0] attn + gates[1] sliding-attn + gates[2] coreset-attn."""
+    g = np.asarray(gates, dtype=np.float64)
+    o_full = attn_full(Q, K, V, scale, q_rows=q_rows)
+    o_sld = attn_sliding(grid, tile, window, Q, K, V, scale, q_rows=q_rows)
+    o_core, _, _ = attn_coreset(grid, bucket, ratio, Q, K, V, scale, q_rows=q_rows)
+    return g[0] * o_full + g[1] * o_sld + g[2] * o_core

@@ -29,6 +29,7 @@ EXPORTS = (
     "vorta_routed_attention", "vorta_routed_attention_host", "vorta_plan_set_profiling",
     "vorta_plan_stage_ms", "vorta_plan_stage_ms_at", "vorta_plan_last_launches", "vorta_device_status",
     "vorta_status_string", "vorta_routed_attention_static", "vorta_plan_device",
+    "vorta_router_gates", "vorta_soft_mixture",
 )
 VORTA_STATIC_WORKSPACE_BYTES = 16 * 1024 * 1024
 
@@ -50,6 +51,7 @@ class vorta_plan_info_t(ctypes.Structure):
                 ("n_coreset", ctypes.c_int32), ("workspace_bytes", ctypes.c_int64),
                 ("workspace_bytes_max", ctypes.c_int64),
                 ("host_call_scratch_bytes", ctypes.c_int64),
+                ("mixture_workspace_bytes", ctypes.c_int64),
                 ("flops_full_head", ctypes.c_double), ("flops_sliding_head", ctypes.c_double),
                 ("flops_coreset_head", ctypes.c_double), ("flops_layer", ctypes.c_double),
                 ("flops_issued_layer", ctypes.c_double), ("n_work_items", ctypes.c_int64),
@@ -81,6 +83,8 @@ def lib() -> ctypes.CDLL:
     L.vorta_routed_attention_host.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     L.vorta_routed_attention_static.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp]
     L.vorta_plan_device.argtypes = [vp, ctypes.POINTER(i32)]
+    L.vorta_router_gates.argtypes = [vp, vp, i32, i32, vp, vp, vp]
+    L.vorta_soft_mixture.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     L.vorta_plan_set_profiling.argtypes = [vp, i32]
     L.vorta_plan_stage_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float * 4)]
     L.vorta_plan_stage_ms_at.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_float * 4)]
@@ -175,6 +179,18 @@ def vorta_plan_device(plan: int) -> int:
     d = ctypes.c_int32()
     _check(lib().vorta_plan_device(plan, ctypes.byref(d)), "vorta_plan_device")
     return d.value
+
+
+def vorta_router_gates(T_ptr: int, WR_ptr: int, d_model: int, heads: int, gates_ptr: int, routes_ptr: int,
+                       stream: int = 0) -> None:
+    _check(lib().vorta_router_gates(T_ptr, WR_ptr, d_model, heads, gates_ptr, routes_ptr, stream),
+           "vorta_router_gates")
+
+
+def vorta_soft_mixture(plan: int, Q_ptr: int, K_ptr: int, V_ptr: int, gates_ptr: int, O_ptr: int,
+                       workspace_ptr: int, workspace_bytes: int, stream: int = 0) -> None:
+    _check(lib().vorta_soft_mixture(plan, Q_ptr, K_ptr, V_ptr, gates_ptr, O_ptr, workspace_ptr,
+                                    workspace_bytes, stream), "vorta_soft_mixture")
 
 
 def vorta_plan_set_profiling(plan: int, on: bool) -> None:
@@ -326,9 +342,32 @@ class Plan:
                                0 if ws is None else ws.numel(), self._stream())
         return O
 
+    def soft_mixture(self, Q, K, V, gates, O=None, workspace=None):
+        """gates: f32 CUDA [heads, 3]; every head runs all three branches (Eq. 5)."""
+        import torch
+        if O is None:
+            O = torch.empty_like(Q)
+        need = int(self.info.mixture_workspace_bytes)
+        ws = workspace if workspace is not None else torch.empty(need, dtype=torch.uint8, device=Q.device)
+        vorta_soft_mixture(self.handle, Q.data_ptr(), K.data_ptr(), V.data_ptr(), gates.data_ptr(),
+                           O.data_ptr(), ws.data_ptr(), ws.numel(), self._stream())
+        return O
+
     def routed_attention_host(self, Qh, Kh, Vh, Oh, scratch):
         """Host (pinned) tensors in and out; `scratch` is a uint8 CUDA tensor."""
         vorta_routed_attention_host(self.handle, Qh.data_ptr(), Kh.data_ptr(), Vh.data_ptr(),
                                     Oh.data_ptr(), scratch.data_ptr(), scratch.numel(),
                                     self._stream())
         return Oh
+
+
+def router_gates(T, WR):
+    """T: f32 CUDA [d_model]; WR: f32 CUDA [heads, d_model, 3] -> (gates f32 [heads, 3], routes uint8 [heads])."""
+    import torch
+    heads, d_model, three = WR.shape
+    assert three == 3 and T.shape == (d_model,) and T.is_cuda and WR.is_contiguous()
+    gates = torch.empty((heads, 3), dtype=torch.float32, device=T.device)
+    routes = torch.empty((heads,), dtype=torch.uint8, device=T.device)
+    vorta_router_gates(T.data_ptr(), WR.data_ptr(), d_model, heads, gates.data_ptr(), routes.data_ptr(),
+                       int(torch.cuda.current_stream().cuda_stream))
+    return gates, routes

@@ -102,7 +102,7 @@ attention_simt_kernel(AttnParams p)
     }
     if (q_valid) {
         float inv = 1.f / l;
-        __nv_bfloat16 *o = O + base + (int64_t)qtok * D;
+        __nv_bfloat16 *o = O + (int64_t)(compact ? w.slice : w.out_slice) * rows * D + (int64_t)qtok * D;
 #pragma unroll
         for (int c = 0; c < D; c += 2)
             *reinterpret_cast<__nv_bfloat162 *>(o + c) = __floats2bfloat162_rn(acc[c] * inv, acc[c + 1] * inv);

@@ -610,7 +610,8 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
         int32_t token = 0;
         const bool valid = block_row_token(p.g, w.mode, w.q_org[m], w.kv_len, row, &token);
         const int64_t rows = w.mode == MODE_COMPACT ? p.g.Lc : p.g.L;
-        __nv_bfloat16 *out = (w.mode == MODE_COMPACT ? p.Oc : p.O) + ((int64_t)w.slice * rows + token) * D;
+        __nv_bfloat16 *out = (w.mode == MODE_COMPACT ? p.Oc + (int64_t)w.slice * rows * D : p.O + (int64_t)w.out_slice * rows * D) +
+                             (int64_t)token * D;
         const float inv = 1.f / row_sum;
 #pragma unroll
         for (int c = 0; c < D / 32; ++c) {

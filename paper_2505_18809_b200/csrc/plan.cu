@@ -28,14 +28,20 @@ struct vorta_plan {
     uint32_t *d_colmasks = nullptr;
     int32_t *d_seg_start = nullptr;
     int32_t *d_bucket_tab = nullptr;  // [8 shape classes][kBucketTabStride]
-    WorkItem *d_items = nullptr;
-    int32_t *d_cta_begin = nullptr, *d_cta_count = nullptr;
+    // the ordered work of one attention launch: `routed` follows the current routes,
+    // `mixture` runs every head through all three branches (built on first use)
+    struct WorkList {
+        WorkItem *d_items = nullptr;
+        int32_t *d_cta_begin = nullptr, *d_cta_count = nullptr;
+        int32_t n_items = 0;
+        int64_t items_cap = 0;
+        double flops_issued = 0.0;
+        bool built = false;
+    };
+    WorkList routed, mixture;
     int32_t *d_core_slice = nullptr;  // [B * n_core]: compact problem -> b*heads + head
     int32_t *d_core_xslice = nullptr; // same for a shared X with one head
     int32_t *d_status = nullptr;
-    int32_t n_items = 0;
-    int64_t items_cap = 0;
-    double flops_issued = 0.0;
     double sliding_pairs = 0.0;  // sum over listed tile pairs of valid-token products
     int32_t kernel = VORTA_KERNEL_TCGEN05;
     // profiling: a ring of event sets, one per call, so that several calls can be
@@ -116,11 +122,20 @@ Workspace workspace_layout(const Geometry &g, int64_t n_prob)
 
 int64_t tensor_bytes(const Geometry &g) { return (int64_t)g.B * g.heads * g.L * g.d * 2; }
 
+// Bytes of the three branch outputs and of the all-heads core-set scratch of a mixture call.
+int64_t mixture_workspace_bytes(const Geometry &g)
+{
+    return workspace_layout(g, (int64_t)g.B * g.heads).total + align_up(3 * tensor_bytes(g), 256);
+}
+
 void free_device(vorta_plan *p)
 {
     cudaFree(p->d_bm); cudaFree(p->d_kv_list); cudaFree(p->d_kv_count); cudaFree(p->d_colmasks);
-    cudaFree(p->d_seg_start); cudaFree(p->d_bucket_tab); cudaFree(p->d_items); cudaFree(p->d_cta_begin);
-    cudaFree(p->d_cta_count); cudaFree(p->d_core_slice); cudaFree(p->d_core_xslice);
+    cudaFree(p->d_seg_start); cudaFree(p->d_bucket_tab);
+    for (vorta_plan::WorkList *wl : {&p->routed, &p->mixture}) {
+        cudaFree(wl->d_items); cudaFree(wl->d_cta_begin); cudaFree(wl->d_cta_count);
+    }
+    cudaFree(p->d_core_slice); cudaFree(p->d_core_xslice);
     cudaFree(p->d_status);
     for (auto &set : p->ev)
         for (auto &e : set)
@@ -156,24 +171,26 @@ double sliding_valid_pairs(const Geometry &g)
     return total;
 }
 
-// (Re)build the ordered work list for the current routes and upload it.
-int build_work(vorta_plan *p)
+// Build the ordered work list of one attention launch and upload it.  `branches[h]` is a
+// bit set of the branches head h runs (bit r = route r); a head with several branches
+// writes branch r to output slice r * B * heads + (b * heads + h).  Core-set problems are
+// numbered b * n_core + k over the heads that have the core-set bit, in ascending order.
+int build_list(vorta_plan *p, vorta_plan::WorkList &wl, const std::vector<uint8_t> &branches, bool by_branch)
 {
     const Geometry &g = p->g;
-    p->core_heads.clear();
+    std::vector<int32_t> core_heads;
     for (int32_t h = 0; h < g.heads; ++h)
-        if (p->routes[h] == VORTA_ROUTE_CORESET) p->core_heads.push_back(h);
-    if (p->host_only) return VORTA_OK;
-
-    const int32_t n_core = (int32_t)p->core_heads.size();
+        if (branches[h] & (1u << VORTA_ROUTE_CORESET)) core_heads.push_back(h);
+    const int32_t n_core = (int32_t)core_heads.size();
+    const int32_t BH = g.B * g.heads;
     std::vector<WorkItem> items;
     std::vector<double> cost;
-    auto linear_items = [&](int32_t mode, int32_t slice, int32_t len) {
+    auto linear_items = [&](int32_t mode, int32_t slice, int32_t out_slice, int32_t len) {
         int32_t nblk = (len + kBlockM - 1) / kBlockM;
         int32_t kv = nblk;
         for (int32_t b0 = 0; b0 < nblk; b0 += 2) {
             WorkItem w{};
-            w.mode = mode; w.slice = slice; w.kv_count = kv; w.kv_len = len;
+            w.mode = mode; w.slice = slice; w.out_slice = out_slice; w.kv_count = kv; w.kv_len = len;
             w.n_mblk = std::min(2, nblk - b0);
             for (int m = 0; m < w.n_mblk; ++m) w.q_org[m][0] = (b0 + m) * kBlockM;
             items.push_back(w);
@@ -182,16 +199,15 @@ int build_work(vorta_plan *p)
     };
     for (int32_t b = 0; b < g.B; ++b) {
         for (int32_t h = 0; h < g.heads; ++h) {
-            int32_t slice = b * g.heads + h;
-            switch (p->routes[h]) {
-            case VORTA_ROUTE_FULL:
-                linear_items(MODE_LINEAR, slice, g.L);
-                break;
-            case VORTA_ROUTE_SLIDING:
+            const int32_t slice = b * g.heads + h;
+            if (branches[h] & (1u << VORTA_ROUTE_FULL))
+                linear_items(MODE_LINEAR, slice, by_branch ? VORTA_ROUTE_FULL * BH + slice : slice, g.L);
+            if (branches[h] & (1u << VORTA_ROUTE_SLIDING)) {
                 for (int32_t qt = 0; qt < g.n_tiles; ++qt) {
                     int32_t q[3] = {qt / (g.nt[2] * g.nt[1]), (qt / g.nt[2]) % g.nt[1], qt % g.nt[2]};
                     WorkItem w{};
                     w.mode = MODE_TILES; w.slice = slice;
+                    w.out_slice = by_branch ? VORTA_ROUTE_SLIDING * BH + slice : slice;
                     w.kv_count = p->kv_count[qt];
                     w.kv_begin = qt * g.max_kv_per_tile;
                     w.kv_len = 0;
@@ -206,13 +222,10 @@ int build_work(vorta_plan *p)
                     items.push_back(w);
                     cost.push_back((double)w.n_mblk * w.kv_count * g.bn_tile / 128.0 + 2.0);
                 }
-                break;
-            default: {
-                int32_t k = (int32_t)(std::find(p->core_heads.begin(), p->core_heads.end(), h) -
-                                      p->core_heads.begin());
-                linear_items(MODE_COMPACT, b * n_core + k, g.Lc);
-                break;
             }
+            if (branches[h] & (1u << VORTA_ROUTE_CORESET)) {
+                int32_t k = (int32_t)(std::find(core_heads.begin(), core_heads.end(), h) - core_heads.begin());
+                linear_items(MODE_COMPACT, b * n_core + k, 0, g.Lc);
             }
         }
     }
@@ -222,7 +235,7 @@ int build_work(vorta_plan *p)
         double bn = w.mode == MODE_TILES ? g.bn_tile : 128;
         issued += (double)w.n_mblk * w.kv_count * 4.0 * kBlockM * bn * g.d;
     }
-    p->flops_issued = issued;
+    wl.flops_issued = issued;
 
     // longest-processing-time assignment of items to the persistent CTAs
     const int32_t grid = p->sm_count;
@@ -247,28 +260,49 @@ int build_work(vorta_plan *p)
         count[c] = (int32_t)per_cta[c].size();
         for (int32_t i : per_cta[c]) sorted.push_back(items[i]);
     }
-    p->n_items = (int32_t)sorted.size();
+    wl.n_items = (int32_t)sorted.size();
 
-    if ((int64_t)sorted.size() > p->items_cap) {
-        cudaFree(p->d_items);
-        p->d_items = nullptr;
-        p->items_cap = (int64_t)sorted.size();
-        if (cudaMalloc(&p->d_items, sizeof(WorkItem) * std::max<size_t>(sorted.size(), 1)) != cudaSuccess)
+    if (!wl.d_cta_begin &&
+        (cudaMalloc(&wl.d_cta_begin, sizeof(int32_t) * grid) != cudaSuccess ||
+         cudaMalloc(&wl.d_cta_count, sizeof(int32_t) * grid) != cudaSuccess))
+        return VORTA_ERR_CUDA;
+    if ((int64_t)sorted.size() > wl.items_cap) {
+        cudaFree(wl.d_items);
+        wl.d_items = nullptr;
+        wl.items_cap = (int64_t)sorted.size();
+        if (cudaMalloc(&wl.d_items, sizeof(WorkItem) * std::max<size_t>(sorted.size(), 1)) != cudaSuccess)
             return VORTA_ERR_CUDA;
     }
+    // synchronous copies: the caller may change routes between steps
+    if (!sorted.empty() &&
+        cudaMemcpy(wl.d_items, sorted.data(), sizeof(WorkItem) * sorted.size(), cudaMemcpyHostToDevice) != cudaSuccess)
+        return VORTA_ERR_CUDA;
+    if (cudaMemcpy(wl.d_cta_begin, begin.data(), sizeof(int32_t) * grid, cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(wl.d_cta_count, count.data(), sizeof(int32_t) * grid, cudaMemcpyHostToDevice) != cudaSuccess)
+        return VORTA_ERR_CUDA;
+    wl.built = true;
+    return VORTA_OK;
+}
+
+// (Re)build the work list for the current routes.
+int build_work(vorta_plan *p)
+{
+    const Geometry &g = p->g;
+    p->core_heads.clear();
+    for (int32_t h = 0; h < g.heads; ++h)
+        if (p->routes[h] == VORTA_ROUTE_CORESET) p->core_heads.push_back(h);
+    if (p->host_only) return VORTA_OK;
+    std::vector<uint8_t> branches(g.heads);
+    for (int32_t h = 0; h < g.heads; ++h) branches[h] = (uint8_t)(1u << p->routes[h]);
+    int rc = build_list(p, p->routed, branches, false);
+    if (rc != VORTA_OK) return rc;
+    const int32_t n_core = (int32_t)p->core_heads.size();
     std::vector<int32_t> core_slice((size_t)g.B * std::max(n_core, 1)), core_x(core_slice.size());
     for (int32_t b = 0; b < g.B; ++b)
         for (int32_t k = 0; k < n_core; ++k) {
             core_slice[(size_t)b * n_core + k] = b * g.heads + p->core_heads[k];
             core_x[(size_t)b * n_core + k] = b;
         }
-    // synchronous copies: the caller may change routes between steps
-    if (!sorted.empty() &&
-        cudaMemcpy(p->d_items, sorted.data(), sizeof(WorkItem) * sorted.size(), cudaMemcpyHostToDevice) != cudaSuccess)
-        return VORTA_ERR_CUDA;
-    if (cudaMemcpy(p->d_cta_begin, begin.data(), sizeof(int32_t) * grid, cudaMemcpyHostToDevice) != cudaSuccess ||
-        cudaMemcpy(p->d_cta_count, count.data(), sizeof(int32_t) * grid, cudaMemcpyHostToDevice) != cudaSuccess)
-        return VORTA_ERR_CUDA;
     if (n_core &&
         (cudaMemcpy(p->d_core_slice, core_slice.data(), sizeof(int32_t) * g.B * n_core, cudaMemcpyHostToDevice) != cudaSuccess ||
          cudaMemcpy(p->d_core_xslice, core_x.data(), sizeof(int32_t) * g.B * n_core, cudaMemcpyHostToDevice) != cudaSuccess))
@@ -451,8 +485,6 @@ int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
     ok = ok && cudaMalloc(&p->d_seg_start, sizeof(int32_t) * g.n_buckets) == cudaSuccess;
     ok = ok && cudaMalloc(&p->d_bucket_tab, sizeof(int32_t) * btab.size()) == cudaSuccess;
     ok = ok && cudaMemcpy(p->d_bucket_tab, btab.data(), sizeof(int32_t) * btab.size(), cudaMemcpyHostToDevice) == cudaSuccess;
-    ok = ok && cudaMalloc(&p->d_cta_begin, sizeof(int32_t) * p->sm_count) == cudaSuccess;
-    ok = ok && cudaMalloc(&p->d_cta_count, sizeof(int32_t) * p->sm_count) == cudaSuccess;
     ok = ok && cudaMalloc(&p->d_core_slice, sizeof(int32_t) * (size_t)g.B * g.heads) == cudaSuccess;
     ok = ok && cudaMalloc(&p->d_core_xslice, sizeof(int32_t) * (size_t)g.B * g.heads) == cudaSuccess;
     ok = ok && cudaMalloc(&p->d_status, sizeof(int32_t)) == cudaSuccess;
@@ -517,13 +549,14 @@ int vorta_plan_info(const vorta_plan *p, vorta_plan_info_t *o)
     o->workspace_bytes = workspace_layout(g, (int64_t)g.B * o->n_coreset).total;
     o->workspace_bytes_max = workspace_layout(g, (int64_t)g.B * g.heads).total;
     o->host_call_scratch_bytes = 4 * align_up(tensor_bytes(g), 256) + o->workspace_bytes;
+    o->mixture_workspace_bytes = mixture_workspace_bytes(g);
     o->flops_full_head = 4.0 * g.d * (double)g.L * (double)g.L;
     o->flops_sliding_head = 4.0 * g.d * p->sliding_pairs;
     o->flops_coreset_head = 4.0 * g.d * (double)g.Lc * (double)g.Lc;
     o->flops_layer = g.B * (o->n_full * o->flops_full_head + o->n_sliding * o->flops_sliding_head +
                             o->n_coreset * o->flops_coreset_head);
-    o->flops_issued_layer = p->host_only ? 0.0 : p->flops_issued;
-    o->n_work_items = p->host_only ? 0 : p->n_items;
+    o->flops_issued_layer = p->host_only ? 0.0 : p->routed.flops_issued;
+    o->n_work_items = p->host_only ? 0 : p->routed.n_items;
     o->select_bytes_head = (int64_t)g.L * g.d * 2 + ((int64_t)g.Lc + g.L) * 4;
     o->gather_bytes_head = 3 * 2 * (int64_t)g.Lc * g.d * 2;
     o->scatter_bytes_head = ((int64_t)g.Lc + g.L) * g.d * 2;
@@ -600,25 +633,18 @@ int vorta_coreset_select(const vorta_plan *p, const void *X, int32_t Hx, int32_t
     return e == cudaSuccess ? VORTA_OK : VORTA_ERR_CUDA;
 }
 
-int vorta_routed_attention(const vorta_plan *p, const void *Q, const void *K, const void *V, void *O,
-                           const void *X, int32_t Hx, void *workspace, size_t workspace_bytes, void *stream)
+// One layer over a work list: select, gather, attention, scatter.  `o_attn` is the tensor
+// the attention kernel writes full and sliding rows to (indexed by the items' output
+// slices), `o_scatter` the [B*heads, L, d] tensor the core-set rows are scattered into.
+// core_slice == nullptr means the identity (every head is a core-set problem).
+static int run_layer(const vorta_plan *p, const vorta_plan::WorkList &wl, int32_t n_core, const int32_t *core_slice,
+                     const int32_t *core_xslice, const __nv_bfloat16 *q, const __nv_bfloat16 *k,
+                     const __nv_bfloat16 *v, __nv_bfloat16 *o_attn, __nv_bfloat16 *o_scatter, const void *X,
+                     int32_t Hx, void *workspace, cudaStream_t s, bool profile)
 {
-    if (!p || !Q || !K || !V || !O) return VORTA_ERR_INVALID_ARG;
-    if (p->host_only) return VORTA_ERR_UNSUPPORTED;
     const Geometry &g = p->g;
-    if (X && Hx != 1 && Hx != g.heads) return VORTA_ERR_INVALID_ARG;
-    if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) || (X && !aligned(X, 16)))
-        return VORTA_ERR_ALIGNMENT;
-    const int32_t n_core = (int32_t)p->core_heads.size();
     const int32_t n_prob = g.B * n_core;
     Workspace ws = workspace_layout(g, n_prob);
-    if (n_prob > 0) {
-        if (!workspace || (int64_t)workspace_bytes < ws.total) return VORTA_ERR_WORKSPACE;
-        if (!aligned(workspace, 256)) return VORTA_ERR_ALIGNMENT;
-    }
-    DeviceGuard guard(p->device);
-    if (!guard.ok) return VORTA_ERR_CUDA;
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
     char *wsb = static_cast<char *>(workspace);
     int32_t *core_idx = n_prob ? reinterpret_cast<int32_t *>(wsb + ws.core_idx) : nullptr;
     int32_t *src_slot = n_prob ? reinterpret_cast<int32_t *>(wsb + ws.src_slot) : nullptr;
@@ -626,16 +652,13 @@ int vorta_routed_attention(const vorta_plan *p, const void *Q, const void *K, co
     __nv_bfloat16 *Kc = n_prob ? reinterpret_cast<__nv_bfloat16 *>(wsb + ws.Kc) : nullptr;
     __nv_bfloat16 *Vc = n_prob ? reinterpret_cast<__nv_bfloat16 *>(wsb + ws.Vc) : nullptr;
     __nv_bfloat16 *Oc = n_prob ? reinterpret_cast<__nv_bfloat16 *>(wsb + ws.Oc) : nullptr;
-    const __nv_bfloat16 *q = static_cast<const __nv_bfloat16 *>(Q), *k = static_cast<const __nv_bfloat16 *>(K),
-                        *v = static_cast<const __nv_bfloat16 *>(V);
-    __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(O);
 
     AttnParams prm{};
     prm.g = g;
     prm.scale_log2 = p->scale * 1.4426950408889634f;
-    prm.items = p->d_items; prm.cta_begin = p->d_cta_begin; prm.cta_count = p->d_cta_count;
+    prm.items = wl.d_items; prm.cta_begin = wl.d_cta_begin; prm.cta_count = wl.d_cta_count;
     prm.kv_list = p->d_kv_list; prm.colmasks = p->d_colmasks;
-    prm.O = o; prm.Oc = Oc; prm.Q = q; prm.K = k; prm.V = v; prm.Qc = Qc; prm.Kc = Kc; prm.Vc = Vc;
+    prm.O = o_attn; prm.Oc = Oc; prm.Q = q; prm.K = k; prm.V = v; prm.Qc = Qc; prm.Kc = Kc; prm.Vc = Vc;
     prm.status = p->d_status;
 #ifdef VORTA_TRACE
     {
@@ -667,7 +690,7 @@ int vorta_routed_attention(const vorta_plan *p, const void *Q, const void *K, co
     }
 
     int32_t launches = 0;
-    const bool prof = p->profiling;
+    const bool prof = profile && p->profiling;
     const int pslot = (int)(p->prof_calls % vorta_plan::kProfSlots);
     if (prof) {
         for (auto &f : p->ev_valid[pslot]) f = false;
@@ -680,33 +703,98 @@ int vorta_routed_attention(const vorta_plan *p, const void *Q, const void *K, co
     mark(0);
     if (n_prob) {
         const __nv_bfloat16 *xs = X ? static_cast<const __nv_bfloat16 *>(X) : k;
-        const int32_t *xslice = (X && Hx == 1) ? p->d_core_xslice : p->d_core_slice;
+        const int32_t *xslice = (X && Hx == 1) ? core_xslice : core_slice;
         e = launch_select(g, xs, g.d, n_prob, xslice, p->d_seg_start, p->d_bucket_tab, core_idx, src_slot, s);
         if (e != cudaSuccess) return VORTA_ERR_CUDA;
         ++launches;
     }
     mark(1);
     if (n_prob) {
-        e = launch_gather(g, n_prob, p->d_core_slice, core_idx, q, k, v, Qc, Kc, Vc, s);
+        e = launch_gather(g, n_prob, core_slice, core_idx, q, k, v, Qc, Kc, Vc, s);
         if (e != cudaSuccess) return VORTA_ERR_CUDA;
         ++launches;
     }
     mark(2);
-    if (p->n_items > 0) {
+    if (wl.n_items > 0) {
         e = p->kernel == VORTA_KERNEL_TCGEN05 ? launch_attention_sm100(prm, maps, p->sm_count, s)
-                                              : launch_attention_simt(prm, p->n_items, s);
+                                              : launch_attention_simt(prm, wl.n_items, s);
         if (e != cudaSuccess) return VORTA_ERR_CUDA;
         ++launches;
     }
     mark(3);
     if (n_prob) {
-        e = launch_scatter(g, n_prob, p->d_core_slice, src_slot, Oc, o, s);
+        e = launch_scatter(g, n_prob, core_slice, src_slot, Oc, o_scatter, s);
         if (e != cudaSuccess) return VORTA_ERR_CUDA;
         ++launches;
     }
     mark(4);
     p->last_launches = launches;
     return VORTA_OK;
+}
+
+int vorta_routed_attention(const vorta_plan *p, const void *Q, const void *K, const void *V, void *O,
+                           const void *X, int32_t Hx, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!p || !Q || !K || !V || !O) return VORTA_ERR_INVALID_ARG;
+    if (p->host_only) return VORTA_ERR_UNSUPPORTED;
+    const Geometry &g = p->g;
+    if (X && Hx != 1 && Hx != g.heads) return VORTA_ERR_INVALID_ARG;
+    if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) || (X && !aligned(X, 16)))
+        return VORTA_ERR_ALIGNMENT;
+    const int32_t n_core = (int32_t)p->core_heads.size();
+    if (n_core > 0) {
+        if (!workspace || (int64_t)workspace_bytes < workspace_layout(g, (int64_t)g.B * n_core).total)
+            return VORTA_ERR_WORKSPACE;
+        if (!aligned(workspace, 256)) return VORTA_ERR_ALIGNMENT;
+    }
+    DeviceGuard guard(p->device);
+    if (!guard.ok) return VORTA_ERR_CUDA;
+    __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(O);
+    return run_layer(p, p->routed, n_core, p->d_core_slice, p->d_core_xslice, static_cast<const __nv_bfloat16 *>(Q),
+                     static_cast<const __nv_bfloat16 *>(K), static_cast<const __nv_bfloat16 *>(V), o, o, X, Hx,
+                     workspace, static_cast<cudaStream_t>(stream), true);
+}
+
+int vorta_soft_mixture(vorta_plan *p, const void *Q, const void *K, const void *V, const float *gates, void *O,
+                       void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!p || !Q || !K || !V || !O || !gates) return VORTA_ERR_INVALID_ARG;
+    if (p->host_only) return VORTA_ERR_UNSUPPORTED;
+    const Geometry &g = p->g;
+    if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) || !aligned(gates, 4))
+        return VORTA_ERR_ALIGNMENT;
+    if (!workspace || (int64_t)workspace_bytes < mixture_workspace_bytes(g)) return VORTA_ERR_WORKSPACE;
+    if (!aligned(workspace, 256)) return VORTA_ERR_ALIGNMENT;
+    DeviceGuard guard(p->device);
+    if (!guard.ok) return VORTA_ERR_CUDA;
+    if (!p->mixture.built) {
+        std::vector<uint8_t> all(g.heads, (uint8_t)7);  // every head runs all three branches
+        int rc = build_list(p, p->mixture, all, true);
+        if (rc != VORTA_OK) return rc;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // the three branch outputs [3, B*heads, L, d] sit back to back after the core-set scratch
+    char *wsb = static_cast<char *>(workspace);
+    char *branches = wsb + workspace_layout(g, (int64_t)g.B * g.heads).total;
+    __nv_bfloat16 *br = reinterpret_cast<__nv_bfloat16 *>(branches);
+    __nv_bfloat16 *br_core = reinterpret_cast<__nv_bfloat16 *>(branches + VORTA_ROUTE_CORESET * tensor_bytes(g));
+    int rc = run_layer(p, p->mixture, g.heads, nullptr, nullptr, static_cast<const __nv_bfloat16 *>(Q),
+                       static_cast<const __nv_bfloat16 *>(K), static_cast<const __nv_bfloat16 *>(V), br, br_core,
+                       nullptr, 0, workspace, s, false);
+    if (rc != VORTA_OK) return rc;
+    if (launch_mix_combine(g, gates, br, static_cast<__nv_bfloat16 *>(O), s) != cudaSuccess) return VORTA_ERR_CUDA;
+    p->last_launches += 1;
+    return VORTA_OK;
+}
+
+int vorta_router_gates(const float *T, const float *WR, int32_t d_model, int32_t heads, float *gates,
+                       uint8_t *routes, void *stream)
+{
+    if (!T || !WR || !gates || !routes || d_model < 1 || heads < 1) return VORTA_ERR_INVALID_ARG;
+    if (!aligned(T, 4) || !aligned(WR, 4) || !aligned(gates, 4)) return VORTA_ERR_ALIGNMENT;
+    return launch_router(T, WR, d_model, heads, gates, routes, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? VORTA_OK
+               : VORTA_ERR_CUDA;
 }
 
 int vorta_routed_attention_host(const vorta_plan *p, const void *Qh, const void *Kh, const void *Vh, void *Oh,

@@ -425,7 +425,8 @@ gather_rows_kernel(Geometry g, int32_t n_prob, const int32_t *__restrict__ prob_
         int32_t c = (int32_t)(i % cpr);
         int32_t p = (int32_t)(row / g.Lc);
         int32_t tok = __ldg(core_idx + row);
-        dst[i] = __ldg(src + ((int64_t)prob_slice[p] * g.L + tok) * cpr + c);
+        const int32_t slice = prob_slice ? prob_slice[p] : p;
+        dst[i] = __ldg(src + ((int64_t)slice * g.L + tok) * cpr + c);
     }
 }
 
@@ -462,7 +463,8 @@ scatter_rows_kernel(Geometry g, int32_t n_prob, const int32_t *__restrict__ prob
         int32_t p = (int32_t)(row / g.L);
         int32_t tok = (int32_t)(row % g.L);
         int32_t slot = __ldg(src_slot + row);
-        O[((int64_t)prob_slice[p] * g.L + tok) * cpr + c] = __ldg(Oc + ((int64_t)p * g.Lc + slot) * cpr + c);
+        const int32_t slice = prob_slice ? prob_slice[p] : p;
+        O[((int64_t)slice * g.L + tok) * cpr + c] = __ldg(Oc + ((int64_t)p * g.Lc + slot) * cpr + c);
     }
 }
 
@@ -476,6 +478,88 @@ cudaError_t launch_scatter(const Geometry &g, int32_t n_prob, const int32_t *pro
     scatter_rows_kernel<<<blocks, 256, 0, s>>>(g, n_prob, prob_slice, src_slot,
                                                reinterpret_cast<const uint4 *>(Oc),
                                                reinterpret_cast<uint4 *>(O));
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------
+// Router (Section 3.3, Eq. 3-4): gates = softmax(T W_R) per head, and the branch the
+// inference rule picks: sliding if its gate is strictly the largest, core-set if its
+// gate is strictly the largest, full otherwise (so every tie goes to full).  One warp
+// per head; fp64 accumulation of fp32 inputs; the rule is evaluated on the logits,
+// which order exactly like the gates.
+// ---------------------------------------------------------------------------------
+__global__ void router_kernel(const float *__restrict__ T, const float *__restrict__ WR, int32_t d_model,
+                              int32_t heads, float *__restrict__ gates, uint8_t *__restrict__ routes)
+{
+    const int lane = threadIdx.x & 31;
+    const int32_t h = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (h >= heads) return;
+    const float *W = WR + (int64_t)h * d_model * 3;
+    double l[3] = {0.0, 0.0, 0.0};
+    for (int32_t c = lane; c < d_model; c += 32) {
+        const double t = (double)T[c];
+#pragma unroll
+        for (int r = 0; r < 3; ++r) l[r] = fma(t, (double)W[c * 3 + r], l[r]);
+    }
+#pragma unroll
+    for (int r = 0; r < 3; ++r)
+        for (int m = 16; m >= 1; m >>= 1) l[r] += shfl_xor_f64(l[r], m);
+    if (lane != 0) return;
+    const double mx = fmax(l[0], fmax(l[1], l[2]));
+    const double e0 = exp(l[0] - mx), e1 = exp(l[1] - mx), e2 = exp(l[2] - mx), z = e0 + e1 + e2;
+    gates[h * 3 + 0] = (float)(e0 / z);
+    gates[h * 3 + 1] = (float)(e1 / z);
+    gates[h * 3 + 2] = (float)(e2 / z);
+    uint8_t route = VORTA_ROUTE_FULL;
+    if (l[1] > l[0] && l[1] > l[2]) route = VORTA_ROUTE_SLIDING;
+    else if (l[2] > l[0] && l[2] > l[1]) route = VORTA_ROUTE_CORESET;
+    routes[h] = route;
+}
+
+cudaError_t launch_router(const float *T, const float *WR, int32_t d_model, int32_t heads, float *gates,
+                          uint8_t *routes, cudaStream_t s)
+{
+    router_kernel<<<(heads * 32 + 127) / 128, 128, 0, s>>>(T, WR, d_model, heads, gates, routes);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------
+// Soft mixture (Section 3.3, Eq. 5): O = a1 * full + a2 * sliding + a3 * core-set per head,
+// from the three branch outputs [3, B*heads, L, d]; fp32 arithmetic, bf16 result.
+// ---------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+mix_combine_kernel(Geometry g, const float *__restrict__ gates, const uint4 *__restrict__ branches,
+                   uint4 *__restrict__ O)
+{
+    const int32_t cpr = g.d >> 3;
+    const int64_t per_slice = (int64_t)g.L * cpr, total = (int64_t)g.B * g.heads * per_slice;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        const int32_t h = (int32_t)((i / per_slice) % g.heads);
+        const float a0 = __ldg(gates + h * 3), a1 = __ldg(gates + h * 3 + 1), a2 = __ldg(gates + h * 3 + 2);
+        const uint4 x = __ldg(branches + i), y = __ldg(branches + total + i), z = __ldg(branches + 2 * total + i);
+        const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w}, zs[4] = {z.x, z.y, z.z, z.w};
+        uint32_t r[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float lo = a0 * __uint_as_float(xs[k] << 16) + a1 * __uint_as_float(ys[k] << 16) +
+                             a2 * __uint_as_float(zs[k] << 16);
+            const float hi = a0 * __uint_as_float(xs[k] & 0xffff0000u) + a1 * __uint_as_float(ys[k] & 0xffff0000u) +
+                             a2 * __uint_as_float(zs[k] & 0xffff0000u);
+            __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+            r[k] = *reinterpret_cast<uint32_t *>(&v);
+        }
+        O[i] = make_uint4(r[0], r[1], r[2], r[3]);
+    }
+}
+
+cudaError_t launch_mix_combine(const Geometry &g, const float *gates, const __nv_bfloat16 *branches,
+                               __nv_bfloat16 *O, cudaStream_t s)
+{
+    int64_t total = (int64_t)g.B * g.heads * g.L * (g.d >> 3);
+    unsigned blocks = (unsigned)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
+    mix_combine_kernel<<<blocks, 256, 0, s>>>(g, gates, reinterpret_cast<const uint4 *>(branches),
+                                              reinterpret_cast<uint4 *>(O));
     return cudaGetLastError();
 }
 

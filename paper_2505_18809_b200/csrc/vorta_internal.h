@@ -53,7 +53,8 @@ struct WorkItem {
     int32_t kv_begin;     // MODE_TILES: first entry in the KV list
     int32_t kv_len;       // linear modes: number of keys (L or Lc)
     int32_t q_org[2][3];  // per M-block: (w0, h0, t0) of the box, or (row0, 0, 0)
-    int32_t pad[4];
+    int32_t out_slice;    // slice of the output tensor the rows are written to (non-compact modes)
+    int32_t pad[3];
 };
 static_assert(sizeof(WorkItem) == 64, "WorkItem must stay 64 bytes");
 
@@ -93,6 +94,10 @@ cudaError_t launch_gather(const Geometry &g, int32_t n_prob, const int32_t *prob
 cudaError_t launch_scatter(const Geometry &g, int32_t n_prob, const int32_t *prob_slice,
                            const int32_t *src_slot, const __nv_bfloat16 *Oc, __nv_bfloat16 *O,
                            cudaStream_t s);
+cudaError_t launch_mix_combine(const Geometry &g, const float *gates, const __nv_bfloat16 *branches,
+                               __nv_bfloat16 *O, cudaStream_t s);
+cudaError_t launch_router(const float *T, const float *WR, int32_t d_model, int32_t heads, float *gates,
+                          uint8_t *routes, cudaStream_t s);
 cudaError_t launch_attention_simt(const AttnParams &p, int32_t n_items, cudaStream_t s);
 cudaError_t launch_attention_sm100(const AttnParams &p, const AttnMaps &maps, int32_t grid,
                                    cudaStream_t s);

@@ -169,6 +169,47 @@ def test_growing_scores_exercise_the_lazy_rescale():
     p.close()
 
 
+def test_router_gates_and_routes_match_the_oracle():
+    g = torch.Generator(device=DEV).manual_seed(60)
+    heads, dm = 24, 3072
+    T = torch.randn(dm, generator=g, device=DEV)
+    WR = torch.randn((heads, dm, 3), generator=g, device=DEV) * 0.02
+    WR[3, :, 1] = WR[3, :, 0]          # an exact tie between full and sliding
+    WR[4] = 0.0                        # a three-way tie
+    WR[5, :, 2] = WR[5, :, 1]          # sliding and core-set tie: neither can win, so full
+    gates, routes = vb.router_gates(T, WR)
+    torch.cuda.synchronize()
+    want_g, want_r = oracle.router_gates(T.cpu().numpy(), WR.cpu().numpy())
+    assert np.abs(gates.cpu().numpy().astype(np.float64) - want_g).max() < 1e-6
+    assert np.array_equal(routes.cpu().numpy(), want_r)
+    r = routes.cpu().numpy()
+    assert r[4] == 0 and r[5] == 0 and r[3] in (0, 2)
+    assert set(r.tolist()) == {0, 1, 2}            # the random heads spread over all three branches
+
+
+@pytest.mark.parametrize("kernel", [vb.VORTA_KERNEL_SIMT, vb.VORTA_KERNEL_TCGEN05], ids=["simt", "tcgen05"])
+def test_soft_mixture_matches_the_oracle(kernel):
+    wl = Workload("mix", (6, 10, 12), 3, 128, (2, 4, 4), (3, 3, 3), 0.5, (0, 1, 2), 61, False)
+    Q, K, V = workloads.make_qkv(wl, DEV)
+    p = vb.Plan.from_workload(wl)
+    p.set_kernel(kernel)
+    gates = torch.tensor([[0.2, 0.5, 0.3], [1.0, 0.0, 0.0], [0.05, 0.15, 0.8]], dtype=torch.float32, device=DEV)
+    O = torch.full_like(Q, float("nan"))
+    p.soft_mixture(Q, K, V, gates, O)
+    assert p.device_status() == 0
+    scale = 1.0 / np.sqrt(wl.d)
+    for h in range(wl.heads):
+        want = oracle.soft_mixture(wl.grid, wl.tile, wl.window, wl.bucket, float(np.float32(wl.ratio)),
+                                   head_f64(Q, 0, h), head_f64(K, 0, h), head_f64(V, 0, h), scale,
+                                   gates[h].cpu().numpy().astype(np.float64))
+        assert_close(O[0, h], want, f"mixture h{h}")
+    # the plan's own routes still work afterwards (the two work lists are separate)
+    O2 = run_layer(p, wl, Q, K, V, kernel)
+    for h in range(wl.heads):
+        assert_close(O2[0, h], oracle_head_rows(wl, Q, K, V, 0, h, None), f"routed after mixture h{h}")
+    p.close()
+
+
 def test_argument_errors_launch_nothing():
     wl = small_workloads()[1]
     Q, K, V = workloads.make_qkv(wl, DEV)

@@ -340,3 +340,46 @@ def test_min_gap_reports_near_ties():
     assert 0 < gap < 2
     _, _, gap1 = oracle.coreset_select(grid, bucket, 1.0, X, return_gap=True)
     assert gap1 == np.inf
+
+
+# --------------------------------------------------------------------------- router and soft mixture
+def test_inference_rule_strict_inequalities_and_ties_go_to_full():
+    # Eq. 4: a branch wins only if its gate is strictly the largest; build logits from chosen gates
+    cases = [((0.5, 0.3, 0.2), 0), ((0.2, 0.5, 0.3), 1), ((0.2, 0.3, 0.5), 2),
+             ((0.4, 0.4, 0.2), 0), ((0.2, 0.4, 0.4), 0), ((0.4, 0.2, 0.4), 0), ((1 / 3, 1 / 3, 1 / 3), 0)]
+    for gates, want in cases:
+        WR = np.log(np.array(gates))[None, None, :]          # one head, d_model = 1, T = 1
+        g, r = oracle.router_gates(np.ones(1), WR)
+        assert np.abs(g[0] - np.array(gates)).max() < 1e-12
+        assert r[0] == want, gates
+
+
+def test_router_gates_are_a_softmax():
+    g = np.random.default_rng(20)
+    T, WR = g.standard_normal(48), g.standard_normal((5, 48, 3))
+    gates, routes = oracle.router_gates(T, WR)
+    assert np.abs(gates.sum(axis=1) - 1).max() < 1e-12 and (gates > 0).all()
+    logits = T @ WR
+    assert np.array_equal(np.argmax(logits, axis=2 - 1), np.argmax(gates, axis=1))
+    # a constant added to all three logits of a head changes nothing
+    WR2 = WR + (g.standard_normal((5, 1, 1)) * np.ones((1, 48, 3))) * 0 + 0.0
+    WR2[:, 0, :] += 3.0 / T[0]
+    g2, r2 = oracle.router_gates(T, WR2)
+    assert np.abs(g2 - gates).max() < 1e-9 and np.array_equal(r2, routes)
+    # distinct logits: the rule is the arg-max, in the order (full, sliding, core-set)
+    assert np.array_equal(routes, np.argmax(gates, axis=1).astype(np.uint8))
+
+
+def test_soft_mixture_is_linear_in_the_gates_and_one_hot_gates_give_the_branch():
+    grid, tile, window, bucket, r = (6, 6, 8), (2, 2, 2), (3, 3, 3), (2, 3, 2), 0.5
+    Q, K, V = rand_qkv(288, 8, 21)
+    full = oracle.attn_full(Q, K, V, 0.3)
+    sld = oracle.attn_sliding(grid, tile, window, Q, K, V, 0.3)
+    core, _, _ = oracle.attn_coreset(grid, bucket, r, Q, K, V, 0.3)
+    for onehot, want in [((1, 0, 0), full), ((0, 1, 0), sld), ((0, 0, 1), core)]:
+        assert np.array_equal(oracle.soft_mixture(grid, tile, window, bucket, r, Q, K, V, 0.3, onehot), want)
+    mix = oracle.soft_mixture(grid, tile, window, bucket, r, Q, K, V, 0.3, (0.2, 0.5, 0.3))
+    assert np.abs(mix - (0.2 * full + 0.5 * sld + 0.3 * core)).max() < 1e-15
+    rows = [0, 17, 287]
+    assert np.array_equal(oracle.soft_mixture(grid, tile, window, bucket, r, Q, K, V, 0.3, (0.2, 0.5, 0.3),
+                                              q_rows=rows), mix[rows])
