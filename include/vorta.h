@@ -57,7 +57,12 @@ enum { VORTA_ROUTE_FULL = 0, VORTA_ROUTE_SLIDING = 1, VORTA_ROUTE_CORESET = 2 };
 
 /* vorta_plan_desc.flags */
 enum {
-    VORTA_PLAN_HOST_ONLY = 1 /* geometry and accounting only: needs no GPU, cannot launch */
+    VORTA_PLAN_HOST_ONLY = 1, /* geometry and accounting only: needs no GPU, cannot launch */
+    VORTA_PLAN_POOL_MERGE = 2 /* core-set heads: the centre's rows of Q, K, V become the mean over the
+                                 centre and the tokens pruned from its bucket before attending (Section 3.2,
+                                 "merged into the center"; the paper does not give the operator).  With a
+                                 bucket that keeps one token this is average pooling: bucket (2,1,1),
+                                 (1,2,1) or (1,1,2) at ratio 0.5 are the AP variants of Section 4.2. */
 };
 
 /* Which attention kernel vorta_routed_attention launches. */
@@ -77,7 +82,7 @@ typedef struct {
     float coreset_ratio;  /* r_core in (0, 1]: a bucket of n tokens keeps max(1, floor(r*n + 1/2)) */
     float softmax_scale;  /* multiplies QK^T; 0 selects 1/sqrt(d) */
     const uint8_t *routes;/* host, [heads]: branch of each head (same for every batch entry) */
-    int32_t flags;        /* 0 or VORTA_PLAN_HOST_ONLY */
+    int32_t flags;        /* bit set of VORTA_PLAN_* */
     int32_t device;       /* CUDA device ordinal; -1 = the calling thread's current device */
 } vorta_plan_desc;
 

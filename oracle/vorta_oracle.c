@@ -17,8 +17,8 @@
  *   - a video axis with fewer tiles than the window spans is unrestricted;
  *   - the similarity of bucketed core-set selection is the cosine;
  *   - keep(n) = max(1, floor(r*n + 1/2)) tokens survive in a bucket of n tokens;
- *   - pruned tokens are NOT merged into the centre: they only receive the
- *     centre's output row at unpool time.
+ *   - by default pruned tokens are NOT merged into the centre: they only receive
+ *     the centre's output row at unpool time; the optional merge is the plain mean.
  *
  * Pinned by tests/test_oracle_pins.py against: brute-force dense attention with
  * explicit masks built a different way (numpy), torch's fp64
@@ -404,26 +404,58 @@ VO_API int64_t vo_coreset_select(const int32_t v[3], const int32_t b[3], double 
  * of the slot src_slot names.  core_idx [Lc] and src_slot [L] are returned too.
  * O is [nq, d].  Returns Lc, or -1 on allocation failure.
  */
-VO_API int64_t vo_attn_coreset(const int32_t v[3], const int32_t b[3], double r, int32_t d,
-                               const double *Q, const double *K, const double *V, const double *X,
-                               int32_t dx, double scale, int64_t nq, const int64_t *q_rows,
-                               double *O, int32_t *core_idx, int32_t *src_slot)
+/*
+ * merge != 0: the pruned tokens' information is merged into the centre (Section 3.2: "their
+ * representational information is merged into the center"; the operator is not given -- the
+ * reading here is the plain mean): the centre's rows of Q, K and V in the compact sequences
+ * become the mean over the centre and the tokens pruned from its bucket.  With a bucket
+ * that keeps one token this is average pooling (the AP variants of Section 4.2).
+ */
+VO_API int64_t vo_attn_coreset_ex(const int32_t v[3], const int32_t b[3], double r, int32_t d,
+                                  const double *Q, const double *K, const double *V, const double *X,
+                                  int32_t dx, double scale, int64_t nq, const int64_t *q_rows,
+                                  double *O, int32_t *core_idx, int32_t *src_slot, int merge)
 {
     int64_t L = (int64_t)v[0] * v[1] * v[2];
     int64_t Lc = vo_coreset_select(v, b, r, X, dx, core_idx, src_slot, NULL);
     if (Lc < 0) return -1;
 
     /* pool: the compact sequences */
+    double *Qc = (double *)malloc(sizeof(double) * (size_t)(Lc * d));
     double *Kc = (double *)malloc(sizeof(double) * (size_t)(Lc * d));
     double *Vc = (double *)malloc(sizeof(double) * (size_t)(Lc * d));
+    int64_t *members = (int64_t *)malloc(sizeof(int64_t) * (size_t)Lc);
+    if (!Qc || !members) return -1;
     /* which slots are needed, and where their output goes */
     int64_t *slot_of_row = (int64_t *)malloc(sizeof(int64_t) * (size_t)nq);
     int64_t *need = (int64_t *)malloc(sizeof(int64_t) * (size_t)Lc); /* slot -> dense id or -1 */
     if (!Kc || !Vc || !slot_of_row || !need) return -1;
     for (int64_t s = 0; s < Lc; ++s) {
+        memcpy(Qc + s * d, Q + (int64_t)core_idx[s] * d, sizeof(double) * (size_t)d);
         memcpy(Kc + s * d, K + (int64_t)core_idx[s] * d, sizeof(double) * (size_t)d);
         memcpy(Vc + s * d, V + (int64_t)core_idx[s] * d, sizeof(double) * (size_t)d);
         need[s] = -1;
+        members[s] = 1;
+    }
+    if (merge) {
+        /* add every pruned token's rows to its centre's slot, then divide by the head count */
+        for (int64_t i = 0; i < L; ++i) {
+            int64_t s = src_slot[i];
+            if (core_idx[s] == i) continue; /* kept: it is its own slot */
+            for (int32_t c = 0; c < d; ++c) {
+                Qc[s * d + c] += Q[i * d + c];
+                Kc[s * d + c] += K[i * d + c];
+                Vc[s * d + c] += V[i * d + c];
+            }
+            members[s] += 1;
+        }
+        for (int64_t s = 0; s < Lc; ++s)
+            if (members[s] > 1)
+                for (int32_t c = 0; c < d; ++c) {
+                    Qc[s * d + c] /= (double)members[s];
+                    Kc[s * d + c] /= (double)members[s];
+                    Vc[s * d + c] /= (double)members[s];
+                }
     }
     int64_t n_need = 0;
     for (int64_t rr = 0; rr < nq; ++rr) {
@@ -452,7 +484,7 @@ VO_API int64_t vo_attn_coreset(const int32_t v[3], const int32_t b[3], double r,
         if (!err) {
 #pragma omp for schedule(dynamic, 4)
             for (int64_t u = 0; u < n_need; ++u) {
-                const double *q = Q + (int64_t)core_idx[slots[u]] * d;
+                const double *q = Qc + slots[u] * d;
                 attend_row(q, Kc, Vc, d, NULL, Lc, scale, Oc + u * d, sbuf);
             }
         }
@@ -462,13 +494,23 @@ VO_API int64_t vo_attn_coreset(const int32_t v[3], const int32_t b[3], double r,
     for (int64_t rr = 0; rr < nq; ++rr)
         memcpy(O + rr * d, Oc + need[slot_of_row[rr]] * d, sizeof(double) * (size_t)d);
 
+    free(Qc);
     free(Kc);
     free(Vc);
+    free(members);
     free(slot_of_row);
     free(need);
     free(slots);
     free(Oc);
     return err ? -1 : Lc;
+}
+
+VO_API int64_t vo_attn_coreset(const int32_t v[3], const int32_t b[3], double r, int32_t d,
+                               const double *Q, const double *K, const double *V, const double *X,
+                               int32_t dx, double scale, int64_t nq, const int64_t *q_rows,
+                               double *O, int32_t *core_idx, int32_t *src_slot)
+{
+    return vo_attn_coreset_ex(v, b, r, d, Q, K, V, X, dx, scale, nq, q_rows, O, core_idx, src_slot, 0);
 }
 
 VO_API int vo_num_threads(void)

@@ -62,6 +62,8 @@ def _load() -> ctypes.CDLL:
                                     _f64p, _f64p, ctypes.c_int32, ctypes.c_double, ctypes.c_int64,
                                     _i64p, _f64p, _i32p, _i32p]
     lib.vo_attn_coreset.restype = ctypes.c_int64
+    lib.vo_attn_coreset_ex.argtypes = lib.vo_attn_coreset.argtypes + [ctypes.c_int]
+    lib.vo_attn_coreset_ex.restype = ctypes.c_int64
     lib.vo_num_threads.argtypes = []
     lib.vo_num_threads.restype = ctypes.c_int
     _lib = lib
@@ -165,10 +167,12 @@ def coreset_select(grid, bucket, ratio: float, X, return_gap: bool = False):
     return (core_idx, src_slot, gap.value) if return_gap else (core_idx, src_slot)
 
 
-def attn_coreset(grid, bucket, ratio: float, Q, K, V, scale: float, X=None, q_rows=None):
+def attn_coreset(grid, bucket, ratio: float, Q, K, V, scale: float, X=None, q_rows=None,
+                 merge: bool = False):
     """Core-set attention (unpool . attn . pool) for one head.
 
-    X defaults to K.  Returns (O [nq, d], core_idx, src_slot).
+    X defaults to K.  merge: the centre's Q, K, V rows become the mean over the centre and
+    the tokens pruned from its bucket.  Returns (O [nq, d], core_idx, src_slot).
     """
     Q, K, V = _f64(Q), _f64(K), _f64(V)
     X = K if X is None else _f64(X)
@@ -179,10 +183,10 @@ def attn_coreset(grid, bucket, ratio: float, Q, K, V, scale: float, X=None, q_ro
     O = np.zeros((nq, d), dtype=np.float64)
     core_idx = np.zeros(Lc, dtype=np.int32)
     src_slot = np.zeros(L, dtype=np.int32)
-    got = _load().vo_attn_coreset(_triple(grid), _triple(bucket), float(ratio), d, _ptr(Q, _f64p),
-                                  _ptr(K, _f64p), _ptr(V, _f64p), _ptr(X, _f64p), X.shape[1],
-                                  float(scale), nq, _ptr(rows, _i64p), _ptr(O, _f64p),
-                                  _ptr(core_idx, _i32p), _ptr(src_slot, _i32p))
+    got = _load().vo_attn_coreset_ex(_triple(grid), _triple(bucket), float(ratio), d, _ptr(Q, _f64p),
+                                     _ptr(K, _f64p), _ptr(V, _f64p), _ptr(X, _f64p), X.shape[1],
+                                     float(scale), nq, _ptr(rows, _i64p), _ptr(O, _f64p),
+                                     _ptr(core_idx, _i32p), _ptr(src_slot, _i32p), int(bool(merge)))
     if got != Lc:
         raise RuntimeError(f"vo_attn_coreset returned {got}, expected {Lc}")
     return O, core_idx, src_slot

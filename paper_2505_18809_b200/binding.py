@@ -21,6 +21,7 @@ VORTA_ERR_INVALID_ARG, VORTA_ERR_UNSUPPORTED, VORTA_ERR_ALIGNMENT = 1, 2, 3
 VORTA_ERR_WORKSPACE, VORTA_ERR_CUDA, VORTA_ERR_TIMEOUT, VORTA_ERR_INTERNAL = 4, 5, 6, 7
 VORTA_ROUTE_FULL, VORTA_ROUTE_SLIDING, VORTA_ROUTE_CORESET = 0, 1, 2
 VORTA_PLAN_HOST_ONLY = 1
+VORTA_PLAN_POOL_MERGE = 2
 VORTA_KERNEL_TCGEN05, VORTA_KERNEL_SIMT = 0, 1
 
 EXPORTS = (
@@ -249,9 +250,9 @@ class Plan:
     """Owns one vorta_plan; methods take torch CUDA tensors and pass their pointers on."""
 
     def __init__(self, B, heads, grid, d, tile, window, ratio, routes, bucket=(0, 0, 0),
-                 scale=0.0, host_only=False, device=-1):
-        self.desc = make_desc(B, heads, grid, d, tile, window, ratio, routes, bucket, scale,
-                              VORTA_PLAN_HOST_ONLY if host_only else 0, device)
+                 scale=0.0, host_only=False, device=-1, merge=False):
+        flags = (VORTA_PLAN_HOST_ONLY if host_only else 0) | (VORTA_PLAN_POOL_MERGE if merge else 0)
+        self.desc = make_desc(B, heads, grid, d, tile, window, ratio, routes, bucket, scale, flags, device)
         self.handle = vorta_plan_create(self.desc)
         self.B, self.heads, self.grid, self.d = B, heads, tuple(grid), d
         self._workspace = None
@@ -259,7 +260,7 @@ class Plan:
     @classmethod
     def from_workload(cls, wl, host_only=False, device=-1):
         return cls(wl.B, wl.heads, wl.grid, wl.d, wl.tile, wl.window, wl.ratio, wl.routes,
-                   wl.bucket, 0.0, host_only, device)
+                   wl.bucket, 0.0, host_only, device, getattr(wl, "merge", False))
 
     def close(self):
         if getattr(self, "handle", None):

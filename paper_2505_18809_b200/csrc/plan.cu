@@ -15,6 +15,7 @@ struct vorta_plan {
     Geometry g{};
     float scale = 0.f;
     bool host_only = false;
+    bool pool_merge = false;  // merge the pruned tokens into their centre (mean) before attending
     int device = 0;
     int sm_count = 0;
     std::vector<uint8_t> routes;
@@ -367,7 +368,7 @@ int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
     if ((int64_t)D.B * D.heads > 65535) return VORTA_ERR_INVALID_ARG;
     if (!(D.coreset_ratio > 0.f) || !(D.coreset_ratio <= 1.f)) return VORTA_ERR_INVALID_ARG;
     if (!(D.softmax_scale >= 0.f) || !std::isfinite(D.softmax_scale)) return VORTA_ERR_INVALID_ARG;
-    if (D.flags & ~VORTA_PLAN_HOST_ONLY) return VORTA_ERR_INVALID_ARG;
+    if (D.flags & ~(VORTA_PLAN_HOST_ONLY | VORTA_PLAN_POOL_MERGE)) return VORTA_ERR_INVALID_ARG;
     int32_t bucket[3] = {D.bucket[0], D.bucket[1], D.bucket[2]};
     if (bucket[0] == 0 && bucket[1] == 0 && bucket[2] == 0) { bucket[0] = 2; bucket[1] = 3; bucket[2] = 2; }
     for (int a = 0; a < 3; ++a)
@@ -399,6 +400,7 @@ int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
     g.ratio = (double)D.coreset_ratio;
     p->scale = D.softmax_scale > 0.f ? D.softmax_scale : 1.0f / std::sqrt((float)D.d);
     p->host_only = (D.flags & VORTA_PLAN_HOST_ONLY) != 0;
+    p->pool_merge = (D.flags & VORTA_PLAN_POOL_MERGE) != 0;
     p->routes.assign(D.routes, D.routes + D.heads);
 
     // core-set segments: prefix sum of keep(n) over the buckets in raster order
@@ -713,6 +715,11 @@ static int run_layer(const vorta_plan *p, const vorta_plan::WorkList &wl, int32_
         e = launch_gather(g, n_prob, core_slice, core_idx, q, k, v, Qc, Kc, Vc, s);
         if (e != cudaSuccess) return VORTA_ERR_CUDA;
         ++launches;
+        if (p->pool_merge) {
+            e = launch_merge(g, n_prob, core_slice, p->d_seg_start, p->d_bucket_tab, src_slot, q, k, v, Qc, Kc, Vc, s);
+            if (e != cudaSuccess) return VORTA_ERR_CUDA;
+            ++launches;
+        }
     }
     mark(2);
     if (wl.n_items > 0) {

@@ -446,6 +446,82 @@ cudaError_t launch_gather(const Geometry &g, int32_t n_prob, const int32_t *prob
 }
 
 // ---------------------------------------------------------------------------------
+// Optional merge (Section 3.2: the pruned tokens' information is merged into the centre;
+// read here as the plain mean): after the gather, the centre's compact rows of Q, K and V
+// become the mean over the centre and the tokens pruned from its bucket.  One warp per
+// (problem, bucket); a lane owns one 16-byte chunk of one of the three rows; fp32 sums,
+// one rounding to bf16.
+// ---------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+merge_centres_kernel(Geometry g, const int32_t *__restrict__ prob_slice, const int32_t *__restrict__ seg_start,
+                     const int32_t *__restrict__ bucket_tab, const int32_t *__restrict__ src_slot,
+                     const uint4 *__restrict__ Q, const uint4 *__restrict__ K, const uint4 *__restrict__ V,
+                     uint4 *__restrict__ Qc, uint4 *__restrict__ Kc, uint4 *__restrict__ Vc)
+{
+    __shared__ int32_t tab[8 * kBucketTabStride];
+    for (int i = threadIdx.x; i < 8 * kBucketTabStride; i += blockDim.x) tab[i] = bucket_tab[i];
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const int32_t bkt = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (bkt >= g.n_buckets) return;
+    const int32_t p = blockIdx.y;
+    const int32_t slice = prob_slice ? prob_slice[p] : p;
+    const int32_t bt = bkt / (g.nb[2] * g.nb[1]), bhw = bkt - bt * (g.nb[2] * g.nb[1]);
+    const int32_t bh = bhw / g.nb[2], bw = bhw - bh * g.nb[2];
+    const int32_t cls = ((g.T - bt * g.bucket[0] < g.bucket[0]) ? 4 : 0) | ((g.H - bh * g.bucket[1] < g.bucket[1]) ? 2 : 0) |
+                        ((g.W - bw * g.bucket[2] < g.bucket[2]) ? 1 : 0);
+    const int32_t *t = tab + cls * kBucketTabStride;
+    const int32_t n = t[0], centre = t[1];
+    const int32_t origin = (bt * g.bucket[0] * g.H + bh * g.bucket[1]) * g.W + bw * g.bucket[2];
+    const int32_t seg = seg_start[bkt];
+    const int32_t my_tok = lane < n ? origin + t[2 + lane] : 0;
+    const bool mine = lane < n && (lane == centre || src_slot[(int64_t)p * g.L + my_tok] == seg);
+    uint32_t members = __ballot_sync(0xffffffffu, mine);  // the centre and the tokens pruned into it
+    const int32_t count = __popc(members);
+    if (count <= 1) return;  // warp-uniform
+    const int32_t cpr = g.d >> 3;
+    const float inv = 1.f / (float)count;
+    for (int32_t idx = lane; idx < 3 * cpr; idx += 32) {
+        const int32_t which = idx / cpr, c = idx - which * cpr;
+        const uint4 *src = which == 0 ? Q : (which == 1 ? K : V);
+        uint4 *dst = which == 0 ? Qc : (which == 1 ? Kc : Vc);
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        for (uint32_t m = members; m; m &= m - 1) {
+            const int32_t l = __ffs(m) - 1;
+            const int32_t tok = origin + t[2 + l];
+            const uint4 u = __ldg(src + ((int64_t)slice * g.L + tok) * cpr + c);
+            const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                acc[2 * i] += __uint_as_float(w[i] << 16);
+                acc[2 * i + 1] += __uint_as_float(w[i] & 0xffff0000u);
+            }
+        }
+        uint32_t r[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            __nv_bfloat162 v = __floats2bfloat162_rn(acc[2 * i] * inv, acc[2 * i + 1] * inv);
+            r[i] = *reinterpret_cast<uint32_t *>(&v);
+        }
+        dst[((int64_t)p * g.Lc + seg) * cpr + c] = make_uint4(r[0], r[1], r[2], r[3]);
+    }
+}
+
+cudaError_t launch_merge(const Geometry &g, int32_t n_prob, const int32_t *prob_slice, const int32_t *seg_start,
+                         const int32_t *bucket_tab, const int32_t *src_slot, const __nv_bfloat16 *Q,
+                         const __nv_bfloat16 *K, const __nv_bfloat16 *V, __nv_bfloat16 *Qc, __nv_bfloat16 *Kc,
+                         __nv_bfloat16 *Vc, cudaStream_t s)
+{
+    if (n_prob == 0) return cudaSuccess;
+    dim3 grid((unsigned)((g.n_buckets + 7) / 8), (unsigned)n_prob);
+    merge_centres_kernel<<<grid, 256, 0, s>>>(g, prob_slice, seg_start, bucket_tab, src_slot,
+                                              reinterpret_cast<const uint4 *>(Q), reinterpret_cast<const uint4 *>(K),
+                                              reinterpret_cast<const uint4 *>(V), reinterpret_cast<uint4 *>(Qc),
+                                              reinterpret_cast<uint4 *>(Kc), reinterpret_cast<uint4 *>(Vc));
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------
 // unpool: every token of a core-set head receives the output row of its slot
 // (its own row if kept, its bucket centre's row if pruned).
 // ---------------------------------------------------------------------------------

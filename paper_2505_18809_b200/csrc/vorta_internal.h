@@ -91,6 +91,10 @@ cudaError_t launch_gather(const Geometry &g, int32_t n_prob, const int32_t *prob
                           const int32_t *core_idx, const __nv_bfloat16 *Q, const __nv_bfloat16 *K,
                           const __nv_bfloat16 *V, __nv_bfloat16 *Qc, __nv_bfloat16 *Kc,
                           __nv_bfloat16 *Vc, cudaStream_t s);
+cudaError_t launch_merge(const Geometry &g, int32_t n_prob, const int32_t *prob_slice, const int32_t *seg_start,
+                         const int32_t *bucket_tab, const int32_t *src_slot, const __nv_bfloat16 *Q,
+                         const __nv_bfloat16 *K, const __nv_bfloat16 *V, __nv_bfloat16 *Qc, __nv_bfloat16 *Kc,
+                         __nv_bfloat16 *Vc, cudaStream_t s);
 cudaError_t launch_scatter(const Geometry &g, int32_t n_prob, const int32_t *prob_slice,
                            const int32_t *src_slot, const __nv_bfloat16 *Oc, __nv_bfloat16 *O,
                            cudaStream_t s);

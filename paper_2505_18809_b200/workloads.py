@@ -34,6 +34,7 @@ class Workload:
     smooth: bool                        # False: plain N(0,1)
     B: int = 1
     bucket: Tuple[int, int, int] = (2, 3, 2)
+    merge: bool = False                 # core-set heads merge pruned tokens into the centre (mean)
 
     @property
     def L(self) -> int:

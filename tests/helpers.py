@@ -30,7 +30,8 @@ def oracle_head_rows(wl, Q, K, V, b, h, rows, scale=None, X=None, route=None):
     x = None if X is None else X
     # the float ratio is what the library sees (the ABI carries a float)
     r = float(np.float32(wl.ratio))
-    O, _, _ = oracle.attn_coreset(wl.grid, wl.bucket, r, q, k, v, scale, X=x, q_rows=rows)
+    O, _, _ = oracle.attn_coreset(wl.grid, wl.bucket, r, q, k, v, scale, X=x, q_rows=rows,
+                                  merge=getattr(wl, "merge", False))
     return O
 
 

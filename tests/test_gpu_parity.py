@@ -210,6 +210,26 @@ def test_soft_mixture_matches_the_oracle(kernel):
     p.close()
 
 
+@pytest.mark.parametrize("kernel", [vb.VORTA_KERNEL_SIMT, vb.VORTA_KERNEL_TCGEN05], ids=["simt", "tcgen05"])
+@pytest.mark.parametrize("bucket,ratio", [((2, 3, 2), 0.5), ((2, 1, 1), 0.5), ((1, 2, 1), 0.5), ((1, 1, 2), 0.5),
+                                          ((2, 3, 2), 0.25)])
+def test_merge_into_centre_and_average_pool_variants(bucket, ratio, kernel):
+    # ragged grid on every axis for the (2,3,2) bucket; with one survivor per bucket the merge is average pooling
+    wl = Workload("merge", (5, 10, 9), 2, 128, (2, 4, 4), (3, 3, 3), ratio, (2, 2), 70, False, 1, bucket, True)
+    Q, K, V = workloads.make_qkv(wl, DEV)
+    p = vb.Plan.from_workload(wl)
+    O = run_layer(p, wl, Q, K, V, kernel)
+    for h in range(wl.heads):
+        assert_close(O[0, h], oracle_head_rows(wl, Q, K, V, 0, h, None), f"merge {bucket} h{h}")
+    # without the flag the same plan gives the unmerged result, which differs
+    plain = Workload("plain", wl.grid, wl.heads, wl.d, wl.tile, wl.window, ratio, wl.routes, 70, False, 1, bucket)
+    p2 = vb.Plan.from_workload(plain)
+    O2 = run_layer(p2, plain, Q, K, V, kernel)
+    assert float((O2.float() - O.float()).abs().max()) > 1e-2
+    p.close()
+    p2.close()
+
+
 def test_argument_errors_launch_nothing():
     wl = small_workloads()[1]
     Q, K, V = workloads.make_qkv(wl, DEV)

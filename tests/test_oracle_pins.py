@@ -383,3 +383,53 @@ def test_soft_mixture_is_linear_in_the_gates_and_one_hot_gates_give_the_branch()
     rows = [0, 17, 287]
     assert np.array_equal(oracle.soft_mixture(grid, tile, window, bucket, r, Q, K, V, 0.3, (0.2, 0.5, 0.3),
                                               q_rows=rows), mix[rows])
+
+
+# --------------------------------------------------------------------------- merge into the centre
+def test_merge_with_one_survivor_per_bucket_is_average_pooling():
+    # bucket (2,1,1), ratio .5: each pair of frames keeps one token holding the pair's mean,
+    # i.e. average pooling over T (the AP_211 variant of Section 4.2), then nearest unpooling
+    grid, d = (6, 3, 4), 8
+    L = 72
+    Q, K, V = rand_qkv(L, d, 30)
+    O, core, src = oracle.attn_coreset(grid, (2, 1, 1), 0.5, Q, K, V, 0.35, merge=True)
+    pool = lambda X: X.reshape(3, 2, 12, d).mean(axis=1).reshape(36, d)
+    Op, _ = dense_attention(pool(Q), pool(K), pool(V), 0.35)
+    want = np.repeat(Op.reshape(3, 1, 12, d), 2, axis=1).reshape(L, d)
+    assert len(core) == 36
+    assert np.abs(O - want).max() < 1e-12
+    for bucket, shape in [((1, 3, 1), (6, 1, 3, 4)), ((1, 1, 2), (6, 3, 2, 2))]:
+        Ob, cb, _ = oracle.attn_coreset(grid, bucket, 1 / 3 if bucket[1] == 3 else 0.5, Q, K, V, 0.35, merge=True)
+        assert len(cb) == L // (3 if bucket[1] == 3 else 2)
+
+
+def test_merge_changes_nothing_when_nothing_is_pruned_or_buckets_are_constant():
+    grid, bucket = (4, 6, 4), (2, 3, 2)
+    Q, K, V = rand_qkv(96, 8, 31)
+    a, _, _ = oracle.attn_coreset(grid, bucket, 1.0, Q, K, V, 0.35, merge=True)
+    b, _, _ = oracle.attn_coreset(grid, bucket, 1.0, Q, K, V, 0.35)
+    assert np.array_equal(a, b)
+    g = np.random.default_rng(32)
+    c = coords(grid)
+    bid = ((c[:, 0] // 2) * 2 + c[:, 1] // 3) * 2 + c[:, 2] // 2
+    Qc, Kc, Vc = (g.standard_normal((8, 8))[bid] for _ in range(3))
+    m, _, _ = oracle.attn_coreset(grid, bucket, 0.5, Qc, Kc, Vc, 0.35, merge=True)
+    assert np.abs(m - oracle.attn_full(Qc, Kc, Vc, 0.35)).max() < 1e-12
+
+
+def test_merge_vs_explicit_numpy():
+    grid, bucket, r = (4, 6, 6), (2, 3, 2), 0.5
+    L, d = 144, 8
+    Q, K, V = rand_qkv(L, d, 33)
+    O, core, src = oracle.attn_coreset(grid, bucket, r, Q, K, V, 0.35, merge=True)
+    bc, bs = brute_select(grid, bucket, r, K)
+    assert np.array_equal(core, bc)
+    Qm, Km, Vm = Q[bc].copy(), K[bc].copy(), V[bc].copy()
+    for s in range(len(bc)):
+        grp = np.where(bs == s)[0]
+        if len(grp) > 1:
+            Qm[s], Km[s], Vm[s] = Q[grp].mean(0), K[grp].mean(0), V[grp].mean(0)
+    Oc, _ = dense_attention(Qm, Km, Vm, 0.35)
+    assert np.abs(O - Oc[bs]).max() < 1e-12
+    plain, _, _ = oracle.attn_coreset(grid, bucket, r, Q, K, V, 0.35)
+    assert np.abs(O - plain).max() > 1e-3
