@@ -261,6 +261,8 @@ def run_ours(args):
     info = plan.info
     ws = plan.workspace(dev)
     plan.set_profiling(True)
+    if args.kernel >= 0:
+        plan.set_kernel(args.kernel)
     stream = torch.cuda.current_stream()
 
     def barrier():
@@ -409,6 +411,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-rows", type=int, default=800, help="oracle rows per head for cpu_baseline")
     ap.add_argument("--reference-rows", type=int, default=16, help="oracle rows per head per step (--impl reference)")
+    ap.add_argument("--kernel", type=int, default=-1, help="attention kernel id (see vorta.h); -1 = library default")
     ap.add_argument("--mixture", action="store_true", help="time vorta_soft_mixture (all three branches per head)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

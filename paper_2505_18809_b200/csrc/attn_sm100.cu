@@ -8,22 +8,32 @@
 //                  the row-major [T, H, W, d] layout;
 //   core-set head  like a full head, over the gathered rows.
 //
-// Warp roles (384 threads):
+// Warp roles (320 threads, so that every thread may hold 200 registers):
 //   warp 0        TMA producer: Q once per item, then K_j, V_j into a 4-slot ring
-//   warp 1        MMA issuer: S = Q K^T and O += P V as tcgen05.mma, accumulators in TMEM
-//   warp 2        TMEM allocation
-//   warps 4-7     softmax of tile 0 (one thread per query row = one TMEM lane)
-//   warps 8-11    softmax of tile 1
-// TMEM columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P (bf16) is
-// written over the first half of its S.  Softmax is the usual online form in the
-// log2 domain with a lazy accumulator rescale (only when the row maximum grew by
-// more than 2^8), done by the softmax threads themselves between two PV MMAs.
+//   warp 1        TMEM allocation; MMA issuer: S = Q K^T and O += P V as tcgen05.mma,
+//                 accumulators in TMEM
+//   warps 2-5     softmax of tile 0 (one thread per query row = one TMEM lane; a warp
+//                 reaches the 32 lanes of TMEM quadrant warp % 4)
+//   warps 6-9     softmax of tile 1
+// TMEM columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512).  A KV block of up
+// to 128 keys is worked through as sub-blocks of up to 64 keys, and the S region of a
+// tile is two 64-column buffers that successive sub-blocks alternate between: while
+// the softmax threads turn S(u) into P(u) (bf16, written over the first half of the
+// same buffer) the scores S(u+1) already wait in the other buffer, and the MMA warp
+// issues O += P(u) V(u) followed by S(u+2) = Q K(u+2)^T into the buffer P(u) leaves.
+// The softmax threads therefore never wait for the tensor pipe in steady state, and
+// the tensor pipe always has the other tile's MMAs queued.  Softmax is the usual
+// online form in the log2 domain with a lazy accumulator rescale (only when the row
+// maximum grew by more than 2^8), done by the softmax threads themselves once the
+// PV MMAs issued so far have completed.
 //
 // Every wait is bounded: a wait that sees no progress for about two seconds
 // records a code in the status word, raises the CTA's abort flag and every role
 // leaves its loop; the CTA then gives outstanding copies time to land, frees its
 // TMEM and returns.
 #include <cuda/ptx>
+
+#include <type_traits>
 
 #include "vorta_internal.h"
 
@@ -50,11 +60,9 @@ enum {
     BAR_Q_EMPTY = 1,
     BAR_KV_FULL = 2,               // +slot
     BAR_KV_EMPTY = 2 + kStages,    // +slot
-    BAR_S_FULL = 2 + 2 * kStages,  // +tile
-    BAR_P_LO = BAR_S_FULL + 2,     // +tile: P columns of keys [0, 64) written
-    BAR_P_HI = BAR_P_LO + 2,       // +tile: the rest of P written
-    BAR_PV_DONE = BAR_P_HI + 2,
-    BAR_O_FREE = BAR_PV_DONE + 2,
+    BAR_S_FULL = 2 + 2 * kStages,  // +2 * tile + buffer: S(u) written (and every MMA issued before it done)
+    BAR_P_READY = BAR_S_FULL + 4,  // +2 * tile + buffer: P(u) written over S(u)
+    BAR_O_FREE = BAR_P_READY + 4,  // +tile: the epilogue has read O out of TMEM
     BAR_MMA_DRAINED = BAR_O_FREE + 2,
     BAR_COUNT
 };
@@ -63,6 +71,7 @@ struct Ctl {
     uint64_t bars[BAR_COUNT];
     uint32_t tmem_base;
     volatile int32_t abort;
+    uint32_t colmasks[kMaxMasks * 4];  // copy of the plan's column-mask classes
 };
 static_assert(sizeof(Ctl) <= 512, "control block outgrew its reservation");
 
@@ -259,18 +268,7 @@ __device__ __forceinline__ float max3(float a, float b, float c)
     return r;
 }
 
-template <int REGS>
-__device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS)); }
-template <int REGS>
-__device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS)); }
-
-// Coordinates of block `j` of the item's KV sequence and its column mask.
-struct KvBlock {
-    int32_t c1, c2, c3;
-    uint32_t mask[4];
-    bool whole;  // all 128 columns valid
-};
-
+// Coordinates of block `j` of the item's KV sequence and its column-mask class.
 __device__ __forceinline__ void kv_block_coords(const AttnParams &p, const WorkItem &w, int32_t j, int32_t &c1,
                                                 int32_t &c2, int32_t &c3, uint32_t &mask_id)
 {
@@ -282,41 +280,39 @@ __device__ __forceinline__ void kv_block_coords(const AttnParams &p, const WorkI
     }
 }
 
-// exp2(s * scale - ref) for the 64 scores s[C0 .. C0+64), packed two bf16 per word IN
-// PLACE into s[C0/2 .. C0/2 + 32): a packed word never lands on a score still to be read.
+// exp2(s * scale - ref) for the 64 scores of a sub-block, packed two bf16 per word IN
+// PLACE into s[0 .. 32): a packed word never lands on a score still to be read.
 // The row sums take the ROUNDED values the PV MMA will use, so that O / sum stays a true
 // weighted mean of V rows (with the unrounded ones a row that attends to a single key is
 // off by up to 2^-9 of |v|, beyond the output tolerance).  Scale-and-shift and the sums
 // use the packed two-wide fp32 instructions.
-template <int C0>
-__device__ __forceinline__ void exp_half(uint32_t (&s)[128], float scale, float neg_ref, float2 (&sum)[2])
+__device__ __forceinline__ void exp_block(uint32_t (&s)[64], float scale, float neg_ref, float2 (&sum)[2])
 {
     const float2 sc = make_float2(scale, scale), nr = make_float2(neg_ref, neg_ref);
 #pragma unroll
     for (int c = 0; c < 64; c += 4) {
-        float2 x0 = __ffma2_rn(make_float2(__uint_as_float(s[C0 + c]), __uint_as_float(s[C0 + c + 1])), sc, nr);
-        float2 x1 = __ffma2_rn(make_float2(__uint_as_float(s[C0 + c + 2]), __uint_as_float(s[C0 + c + 3])), sc, nr);
+        float2 x0 = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), sc, nr);
+        float2 x1 = __ffma2_rn(make_float2(__uint_as_float(s[c + 2]), __uint_as_float(s[c + 3])), sc, nr);
         const uint32_t k0 = pack_bf16(ex2(x0.x), ex2(x0.y));
         const uint32_t k1 = pack_bf16(ex2(x1.x), ex2(x1.y));
-        s[C0 / 2 + (c >> 1)] = k0;
-        s[C0 / 2 + (c >> 1) + 1] = k1;
+        s[c >> 1] = k0;
+        s[(c >> 1) + 1] = k1;
         sum[0] = __fadd2_rn(sum[0], make_float2(__uint_as_float(k0 << 16), __uint_as_float(k0 & 0xffff0000u)));
         sum[1] = __fadd2_rn(sum[1], make_float2(__uint_as_float(k1 << 16), __uint_as_float(k1 & 0xffff0000u)));
     }
 }
 
-// write packed P words of keys [64h, 64h + 64) to columns [32h, 32h + 32) of the S region
-template <int H>
-__device__ __forceinline__ void store_p_half(uint32_t t_s, int32_t bn, uint32_t (&s)[128])
+// write the packed P words of a sub-block of `width` keys to the first width/2 columns at t_p
+__device__ __forceinline__ void store_p(uint32_t t_p, int32_t width, uint32_t (&s)[64])
 {
-    if (bn >= H * 64 + 64) {
-        uint32_t(&half)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[32 * H]);
-        ptx::tcgen05_st_32x32b(t_s + H * 32, half);
+    if (width == 64) {
+        uint32_t(&all)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[0]);
+        ptx::tcgen05_st_32x32b(t_p, all);
     } else {
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-            uint32_t(&chunk)[8] = *reinterpret_cast<uint32_t(*)[8]>(&s[32 * H + 8 * c]);
-            if (H * 64 + c * 16 < bn) ptx::tcgen05_st_32x32b(t_s + H * 32 + c * 8, chunk);
+            uint32_t(&chunk)[8] = *reinterpret_cast<uint32_t(*)[8]>(&s[8 * c]);
+            if (c * 16 < width) ptx::tcgen05_st_32x32b(t_p + c * 8, chunk);
         }
     }
     tc_wait_st();
@@ -337,12 +333,12 @@ __device__ __forceinline__ void rescale_o(uint32_t t_o, float a)
     }
 }
 
-// maximum of the 128 scores of a row (four independent chains of three-input max)
-__device__ __forceinline__ float row_max128(const uint32_t (&s)[128])
+// maximum of the 64 scores of a sub-block (four independent chains of three-input max)
+__device__ __forceinline__ float row_max64(const uint32_t (&s)[64])
 {
     float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-    for (int c = 0; c < 128; c += 8) {
+    for (int c = 0; c < 64; c += 8) {
         mx0 = max3(mx0, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
         mx1 = max3(mx1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
         mx2 = max3(mx2, __uint_as_float(s[c + 4]), __uint_as_float(s[c + 5]));
@@ -403,8 +399,8 @@ __device__ __forceinline__ void mma_role(const AttnParams &p, Ctl *ctl, uint32_t
     tmem = uniform_u32(tmem);
     begin = (int32_t)uniform_u32((uint32_t)begin);
     count = (int32_t)uniform_u32((uint32_t)count);
-    uint32_t kv_it = 0;
-    uint32_t p_cnt[2] = {0, 0}, o_uses[2] = {0, 0};
+    uint32_t kv_base = 0;  // ring position of the item's first K block (K_j at +2j, V_j at +2j+1)
+    uint32_t p_par = 0, o_par = 0;  // phase parities: bit 2m+b of P_READY[m][b], bit m of O_FREE[m]
 
     // Descriptors of tile 0 / slot 0; the others differ by a multiple of the tile pitch
     // in the (16-byte granular) address field, so one 64-bit add moves between them.
@@ -412,28 +408,31 @@ __device__ __forceinline__ void mma_role(const AttnParams &p, Ctl *ctl, uint32_t
     const uint64_t k_desc0 = smem_desc(smem_base + kSmemKV, 16, 1024);          // K-major
     const uint64_t v_desc0 = smem_desc(smem_base + kSmemKV, kHalfBytes, 1024);  // MN-major
     constexpr uint64_t kTileStep = kTileBytes >> 4;
+    constexpr uint64_t kSubStep = (64 * 128) >> 4;  // 64 keys further down a K or V tile
+    const uint32_t idesc_pv = instr_desc((uint32_t)D, 1);
 
-    // S_m = Q_m K^T over the K block in `slot` (16 channels per MMA)
-    auto issue_qk = [&](int m, uint32_t slot, uint32_t idesc) {
+    auto wait_kv = [&](uint32_t pos, int32_t code) {
+        return mbar_wait_uniform(bars + 8 * (BAR_KV_FULL + pos % kStages), (pos / kStages) & 1, ctl, p.status, code);
+    };
+    auto free_kv = [&](uint32_t pos) { tc_commit(bars + 8 * (BAR_KV_EMPTY + pos % kStages), leader); };
+    // S_m[buffer b] = Q_m K^T over sub-block h of the K block at ring position pos (16 channels per MMA)
+    auto issue_qk = [&](int m, uint32_t pos, int b, int h, uint32_t idesc) {
         const uint64_t qa = q_desc0 + (uint64_t)m * kTileStep;
-        const uint64_t kb = k_desc0 + (uint64_t)slot * kTileStep;
+        const uint64_t kb = k_desc0 + (uint64_t)(pos % kStages) * kTileStep + (uint64_t)h * kSubStep;
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
             const uint64_t off = (uint64_t)(((kk / 4) * kHalfBytes + (kk % 4) * 32) >> 4);
-            mma_ss(tmem + m * 128, qa + off, kb + off, idesc, kk > 0 ? 1u : 0u, leader);
+            mma_ss(tmem + m * 128 + b * 64, qa + off, kb + off, idesc, kk > 0 ? 1u : 0u, leader);
         }
     };
-    // O_m (+)= P_m V over the V block in `slot`; P is packed bf16 in S_m's columns
-    // (16 keys per MMA: steps [K0, K0 + 4) of the block, cut at `ksteps`)
-    auto issue_pv = [&](int m, uint32_t slot, uint32_t idesc, int k0, int ksteps, bool first) {
-        const uint64_t vb = v_desc0 + (uint64_t)slot * kTileStep;
+    // O_m (+)= P_m[buffer b] V over sub-block h of the V block at pos (16 keys per MMA)
+    auto issue_pv = [&](int m, uint32_t pos, int b, int h, int ksteps, bool first) {
+        const uint64_t vb = v_desc0 + (uint64_t)(pos % kStages) * kTileStep + (uint64_t)h * kSubStep;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int kk = k0 + i;
-            if (kk < ksteps)
-                mma_ts(tmem + 256 + m * 128, tmem + m * 128 + kk * 8, vb + (uint64_t)(kk * (2048 >> 4)), idesc,
-                       (!first || kk > 0) ? 1u : 0u, leader);
-        }
+        for (int i = 0; i < 4; ++i)
+            if (i < ksteps)
+                mma_ts(tmem + 256 + m * 128, tmem + m * 128 + b * 64 + i * 8, vb + (uint64_t)(i * (2048 >> 4)), idesc_pv,
+                       (!first || i > 0) ? 1u : 0u, leader);
     };
 
     for (int32_t it = 0; it < count; ++it) {
@@ -441,62 +440,53 @@ __device__ __forceinline__ void mma_role(const AttnParams &p, Ctl *ctl, uint32_t
         const int32_t bn = uniform_u32((uint32_t)w->mode) == MODE_TILES ? p.g.bn_tile : kBlockM;
         const int32_t n = (int32_t)uniform_u32((uint32_t)w->kv_count);
         const int32_t nm = (int32_t)uniform_u32((uint32_t)w->n_mblk);
-        const uint32_t idesc_qk = instr_desc((uint32_t)bn, 0), idesc_pv = instr_desc((uint32_t)D, 1);
-        const int ksteps = bn / 16;
+        const int32_t spb = bn > 64 ? 2 : 1;  // sub-blocks per KV block
+        const int32_t n_sub = n * spb;
+        const int32_t width0 = min(bn, 64), width1 = max(bn - 64, 16);
+        const uint32_t idesc_qk0 = instr_desc((uint32_t)width0, 0), idesc_qk1 = instr_desc((uint32_t)width1, 0);
 
         if (!mbar_wait_uniform(bars + 8 * BAR_Q_FULL, it & 1, ctl, p.status, 201)) return;
-        // block 0: both score tiles
-        uint32_t slot_k = kv_it % kStages;
-        if (!mbar_wait_uniform(bars + 8 * (BAR_KV_FULL + slot_k), (kv_it / kStages) & 1, ctl, p.status, 202)) return;
-        ++kv_it;
-        tc_fence_after();
-        for (int m = 0; m < nm; ++m) {
-            issue_qk(m, slot_k, idesc_qk);
-            tc_commit(bars + 8 * (BAR_S_FULL + m), leader);
-        }
-        tc_commit(bars + 8 * (BAR_KV_EMPTY + slot_k), leader);
-        if (n == 1) tc_commit(bars + 8 * BAR_Q_EMPTY, leader);
-        for (int32_t j = 0; j < n; ++j) {
-            const uint32_t slot_v = kv_it % kStages;
-            if (!mbar_wait_uniform(bars + 8 * (BAR_KV_FULL + slot_v), (kv_it / kStages) & 1, ctl, p.status, 203)) return;
-            ++kv_it;
-            const bool has_next = j + 1 < n;
-            slot_k = kv_it % kStages;
+        // the first two score sub-blocks of both tiles
+        for (int32_t u = 0; u < min(n_sub, 2); ++u) {
+            const int32_t j = u / spb, h = u - j * spb;
+            if (h == 0 && !wait_kv(kv_base + 2 * j, 202)) return;
+            tc_fence_after();
             for (int m = 0; m < nm; ++m) {
-                // first half of P: the PV MMAs over keys [0, 64) start while the softmax
-                // threads still work on the second half
-                if (!mbar_wait_uniform(bars + 8 * (BAR_P_LO + m), p_cnt[m] & 1, ctl, p.status, 204)) return;
-                if (j == 0) {
-                    // the previous item's epilogue must have read O_m out of TMEM
-                    if (!mbar_wait_uniform(bars + 8 * (BAR_O_FREE + m), (o_uses[m] & 1) ^ 1, ctl, p.status, 205)) return;
-                    ++o_uses[m];
-                }
-                tc_fence_after();
-                if (leader) TRACE(m, j, 0);
-                issue_pv(m, slot_v, idesc_pv, 0, ksteps, j == 0);
-                if (leader) TRACE(m, j, 1);
-                if (!mbar_wait_uniform(bars + 8 * (BAR_P_HI + m), p_cnt[m] & 1, ctl, p.status, 208)) return;
-                ++p_cnt[m];
-                if (has_next && m == 0) {
-                    if (!mbar_wait_uniform(bars + 8 * (BAR_KV_FULL + slot_k), (kv_it / kStages) & 1, ctl, p.status, 206)) return;
-                }
-                tc_fence_after();
-                if (leader) TRACE(m, j, 2);
-                issue_pv(m, slot_v, idesc_pv, 4, ksteps, false);
-                if (!has_next) tc_commit(bars + 8 * (BAR_PV_DONE + m), leader);
-                if (has_next) {
-                    issue_qk(m, slot_k, idesc_qk);
-                    tc_commit(bars + 8 * (BAR_S_FULL + m), leader);
-                }
-                if (leader) TRACE(m, j, 3);
+                issue_qk(m, kv_base + 2 * j, u & 1, h, h ? idesc_qk1 : idesc_qk0);
+                tc_commit(bars + 8 * (BAR_S_FULL + 2 * m + (u & 1)), leader);
             }
-            tc_commit(bars + 8 * (BAR_KV_EMPTY + slot_v), leader);
-            if (has_next) {
-                tc_commit(bars + 8 * (BAR_KV_EMPTY + slot_k), leader);
-                if (j + 2 == n) tc_commit(bars + 8 * BAR_Q_EMPTY, leader);
-                ++kv_it;
-            }
+            if (h == spb - 1) free_kv(kv_base + 2 * j);
         }
+        if (n_sub <= 2) tc_commit(bars + 8 * BAR_Q_EMPTY, leader);
+
+        for (int32_t u = 0; u < n_sub; ++u) {
+            const int32_t jv = u / spb, h = u - jv * spb, b = u & 1;
+            const int32_t u2 = u + 2, jk = u2 / spb, h2 = u2 - jk * spb;
+            const bool has2 = u2 < n_sub;
+            const uint32_t pos_v = kv_base + 2 * jv + 1, pos_k = kv_base + 2 * jk;
+            if (h == 0 && !wait_kv(pos_v, 203)) return;
+            if (has2 && h2 == 0 && !wait_kv(pos_k, 206)) return;
+            for (int m = 0; m < nm; ++m) {
+                if (!mbar_wait_uniform(bars + 8 * (BAR_P_READY + 2 * m + b), (p_par >> (2 * m + b)) & 1, ctl, p.status, 204)) return;
+                p_par ^= 1u << (2 * m + b);
+                if (u == 0) {
+                    // the previous item's epilogue must have read O_m out of TMEM
+                    if (!mbar_wait_uniform(bars + 8 * (BAR_O_FREE + m), ((o_par >> m) & 1) ^ 1, ctl, p.status, 205)) return;
+                    o_par ^= 1u << m;
+                }
+                tc_fence_after();
+                if (leader) TRACE(m, u, 0);
+                issue_pv(m, pos_v, b, h, (h ? width1 : width0) >> 4, u == 0);
+                if (has2) issue_qk(m, pos_k, b, h2, h2 ? idesc_qk1 : idesc_qk0);
+                // S(u+2) is ready; and, for the lazy rescale and the epilogue: PV(u) is done
+                tc_commit(bars + 8 * (BAR_S_FULL + 2 * m + b), leader);
+                if (leader) TRACE(m, u, 1);
+            }
+            if (h == spb - 1) free_kv(pos_v);
+            if (has2 && h2 == spb - 1) free_kv(pos_k);
+            if (has2 && u2 == n_sub - 1) tc_commit(bars + 8 * BAR_Q_EMPTY, leader);
+        }
+        kv_base += 2 * (uint32_t)n;
     }
     // every commit issued above must have landed before the CTA's barriers go away
     tc_commit(bars + 8 * BAR_MMA_DRAINED, leader);
@@ -508,109 +498,137 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
                                              int32_t count, int m, int row, int warp_q)
 {
     const uint32_t bars = smem_u32(ctl->bars);
+    const int lane = row & 31;
     const uint32_t lane_base = (uint32_t)(warp_q * 32) << 16;
-    const uint32_t t_s = tmem + lane_base + m * 128;        // scores, later P
+    const uint32_t t_s = tmem + lane_base + m * 128;        // scores, later P (two 64-column buffers)
     const uint32_t t_o = tmem + lane_base + 256 + m * 128;  // output accumulator
     const float scale = p.scale_log2;
-    uint32_t s_cnt = 0, part = 0;
+    uint32_t s_par = 0;  // bit b: parity of the next phase of S_FULL[m][b] this thread will consume
 
     for (int32_t it = 0; it < count; ++it) {
-        const WorkItem w = p.items[begin + it];
-        if (m >= w.n_mblk) continue;
-        const int32_t bn = w.mode == MODE_TILES ? p.g.bn_tile : kBlockM;
+        const WorkItem *wp = p.items + begin + it;
+        if (m >= wp->n_mblk) continue;
+        const int32_t w_mode = wp->mode, w_kv_len = wp->kv_len, w_kv_count = wp->kv_count;
+        const KvEntry *kv_entries = p.kv_list + wp->kv_begin;
+        const int32_t bn = w_mode == MODE_TILES ? p.g.bn_tile : kBlockM;
+        const int32_t sh = bn > 64 ? 1 : 0;  // log2 of the sub-blocks per KV block
+        const int32_t n_sub = w_kv_count << sh;
+        const int32_t width0 = min(bn, 64), width1 = bn - 64;
+        // columns of a short block: every block of a sliding head whose tile has fewer than 128
+        // tokens, else the last block of the sequence
+        const int32_t tail_valid = w_mode == MODE_TILES ? bn : w_kv_len - (w_kv_count - 1) * kBlockM;
+        const bool tail_partial = tail_valid < kBlockM;
+        uint32_t tail_mask[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int32_t v = min(max(tail_valid - 32 * i, 0), 32);
+            tail_mask[i] = v == 32 ? 0xffffffffu : ((1u << v) - 1u);
+        }
         float row_max = -INFINITY, row_sum = 0.f;
 
-        for (int32_t j = 0; j < w.kv_count; ++j) {
-            // which columns of this block are real keys
-            uint32_t mask[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
-            bool whole = true;
-            if (w.mode == MODE_TILES) {
-                const uint32_t mask_id = p.kv_list[w.kv_begin + j].mask_id;
-                if (mask_id) {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) mask[i] = __ldg(p.colmasks + mask_id * 4 + i);
-                    whole = false;
-                } else if (bn < kBlockM) {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        int32_t v = min(max(bn - 32 * i, 0), 32);
-                        mask[i] = v == 32 ? 0xffffffffu : ((1u << v) - 1u);
-                    }
-                    whole = false;
-                }
-            } else {
-                const int32_t valid = w.kv_len - j * kBlockM;
-                if (valid < kBlockM) {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        int32_t v = min(max(valid - 32 * i, 0), 32);
-                        mask[i] = v == 32 ? 0xffffffffu : ((1u << v) - 1u);
-                    }
-                    whole = false;
-                }
-            }
-
-            if (row == 0) TRACE(2 + m, j, 0);
-            if (!mbar_wait(bars + 8 * (BAR_S_FULL + m), s_cnt & 1, ctl, p.status, 301 + m)) return;
-            ++s_cnt;
+        // wait for S(u) and read this thread's row of it (all 64 columns, or `width` of them)
+        auto load_sub = [&](auto full, int32_t u, uint32_t(&s)[64]) -> bool {
+            const int32_t b = u & 1;
+            if (!mbar_wait(bars + 8 * (BAR_S_FULL + 2 * m + b), (s_par >> b) & 1, ctl, p.status, 301 + m)) return false;
+            s_par ^= 1u << b;
             tc_fence_after();
-            if (row == 0) TRACE(2 + m, j, 1);
-            // the whole score row of this thread, one TMEM read
-            uint32_t s[128];
+            const int32_t width = decltype(full)::value ? 64 : ((u & sh) ? width1 : width0);
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < 2; ++c) {
                 uint32_t(&chunk)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[32 * c]);
-                if (c * 32 < bn) ptx::tcgen05_ld_32x32b(chunk, t_s + c * 32);
+                if (decltype(full)::value || c * 32 < width) ptx::tcgen05_ld_32x32b(chunk, t_s + b * 64 + c * 32);
             }
             tc_wait_ld();
-            if (row == 0) TRACE(2 + m, j, 2);
-            if (!whole) {
+            return true;
+        };
+        // strike the columns of sub-block u that are not keys (mask class `id` of its block,
+        // fetched ahead by the caller)
+        auto apply_mask = [&](int32_t u, uint32_t id, uint32_t(&s)[64]) {
+            const int32_t h = u & sh;
+            uint32_t m0 = 0, m1 = 0;
+            bool partial = false;
+            if (id) {
+                m0 = ctl->colmasks[id * 4 + 2 * h];
+                m1 = ctl->colmasks[id * 4 + 2 * h + 1];
+                partial = true;
+            } else if (tail_partial && (w_mode == MODE_TILES || (u >> sh) == w_kv_count - 1)) {
+                m0 = h ? tail_mask[2] : tail_mask[0];
+                m1 = h ? tail_mask[3] : tail_mask[1];
+                partial = true;
+            }
+            if (partial) {
 #pragma unroll
-                for (int c = 0; c < 128; ++c)
-                    if (!((mask[c >> 5] >> (c & 31)) & 1u)) s[c] = 0xff800000u;  // -inf: not a key
+                for (int c = 0; c < 64; ++c)
+                    if (!(((c < 32 ? m0 : m1) >> (c & 31)) & 1u)) s[c] = 0xff800000u;  // -inf: not a key
             }
-            // P = exp2(S * scale - max) as packed bf16 over the first bn/2 columns of S, in two
-            // halves: keys [0, 64) -> columns [0, 32), then keys [64, 128) -> columns [32, 64)
-            // (the whole row is already in registers).  The first half is handed to the MMA
-            // warp as soon as it is written, so that its PV MMAs run under the second half.
+        };
+        // One sub-block: s holds the scores of u and row_max covers them.  Writes P(u), then
+        // reads S(u+1) and moves row_max over it.  full: u and u+1 are both whole 64-key
+        // sub-blocks of unmasked blocks, so nothing about widths or masks is looked at.
+        auto step = [&](auto full, int32_t u, uint32_t(&s)[64]) -> bool {
+            constexpr bool kFull = decltype(full)::value;
+            const int32_t b = u & 1;
+            const bool has_next = kFull || u + 1 < n_sub;
+            // mask class of the next sub-block's KV block, in flight under the exponentials
+            const uint32_t next_id =
+                (!kFull && has_next && w_mode == MODE_TILES) ? kv_entries[(u + 1) >> sh].mask_id : 0u;
+            if (row == 0) TRACE(2 + m, u, 0);
+            // P = exp2(S * scale - max) as packed bf16 over the first half of the buffer
             float2 sum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-            const float m_new = fmaxf(row_max, row_max128(s) * scale);
-            if (j == 0) {
-                row_max = m_new;
-            } else if (__any_sync(0xffffffffu, m_new - row_max > kRescaleThreshold)) {
-                // Lazy rescale: O and the row sum move to the new maximum only when it grew by
-                // more than the threshold; until then P may reach 2^threshold.  The previous PV
-                // of this tile has completed (it was issued before the QK whose completion we
-                // just waited for), so O may be rescaled in place.
-                const float a = ex2(row_max - m_new);
-                row_sum *= a;
-                row_max = m_new;
-                rescale_o<D>(t_o, a);
-            }
-            if (row == 0) TRACE(2 + m, j, 3);
-            exp_half<0>(s, scale, -row_max, sum);
-            store_p_half<0>(t_s, bn, s);
+            exp_block(s, scale, -row_max, sum);
+            if (row == 0) TRACE(2 + m, u, 1);
+            store_p(t_s + b * 64, kFull ? 64 : ((u & sh) ? width1 : width0), s);
             tc_fence_before();
-            mbar_arrive(bars + 8 * (BAR_P_LO + m));
-            if (row == 0) TRACE(2 + m, j, 4);
-            if (bn > 64) {
-                exp_half<64>(s, scale, -row_max, sum);
-                store_p_half<1>(t_s, bn, s);
-            }
-            tc_fence_before();
-            mbar_arrive(bars + 8 * (BAR_P_HI + m));
-            if (row == 0) TRACE(2 + m, j, 5);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bars + 8 * (BAR_P_READY + 2 * m + b));
+            if (row == 0) TRACE(2 + m, u, 2);
             row_sum += (sum[0].x + sum[0].y) + (sum[1].x + sum[1].y);
-        }
+            if (has_next) {
+                if (!load_sub(full, u + 1, s)) return false;
+                if (row == 0) TRACE(2 + m, u, 3);
+                if (!kFull) apply_mask(u + 1, next_id, s);
+                const float m_new = fmaxf(row_max, row_max64(s) * scale);
+                if (__any_sync(0xffffffffu, m_new - row_max > kRescaleThreshold)) {
+                    // Lazy rescale: O and the row sum move to the new maximum only when it grew by
+                    // more than the threshold; until then P may reach 2^threshold.  O may be touched
+                    // once PV(u) has completed: the commit that follows it is the next phase of
+                    // this buffer's barrier (looked at here, consumed at sub-block u+2 or in the tail).
+                    if (!mbar_wait(bars + 8 * (BAR_S_FULL + 2 * m + b), (s_par >> b) & 1, ctl, p.status, 321 + m)) return false;
+                    tc_fence_after();
+                    const float a = ex2(row_max - m_new);
+                    row_sum *= a;
+                    row_max = m_new;
+                    rescale_o<D>(t_o, a);
+                }
+                if (row == 0) TRACE(2 + m, u, 4);
+            }
+            return true;
+        };
 
-        // epilogue: O / row_sum -> bf16 -> global memory
-        if (!mbar_wait(bars + 8 * (BAR_PV_DONE + m), part & 1, ctl, p.status, 311 + m)) return;
-        ++part;
+        uint32_t s[64];
+        if (!load_sub(std::false_type{}, 0, s)) return;
+        apply_mask(0, w_mode == MODE_TILES ? kv_entries[0].mask_id : 0u, s);
+        row_max = row_max64(s) * scale;
+        // the leading unmasked blocks, then whatever is cut, short or last
+        const int32_t n_full = min(2 * wp->kv_fast, n_sub) - 1;  // steps whose u and u+1 are both whole
+        int32_t u = 0;
+        for (; u < n_full; ++u)
+            if (!step(std::true_type{}, u, s)) return;
+        for (; u < n_sub; ++u)
+            if (!step(std::false_type{}, u, s)) return;
+
+        // the commits that follow the last two PV MMAs: O is complete
+        for (int32_t u = max(n_sub - 2, 0); u < n_sub; ++u) {
+            if (!mbar_wait(bars + 8 * (BAR_S_FULL + 2 * m + (u & 1)), (s_par >> (u & 1)) & 1, ctl, p.status, 311 + m)) return;
+            s_par ^= 1u << (u & 1);
+        }
         tc_fence_after();
+        // epilogue: O / row_sum -> bf16 -> global memory
         int32_t token = 0;
-        const bool valid = block_row_token(p.g, w.mode, w.q_org[m], w.kv_len, row, &token);
-        const int64_t rows = w.mode == MODE_COMPACT ? p.g.Lc : p.g.L;
-        __nv_bfloat16 *out = (w.mode == MODE_COMPACT ? p.Oc + (int64_t)w.slice * rows * D : p.O + (int64_t)w.out_slice * rows * D) +
+        const int32_t q_org[3] = {wp->q_org[m][0], wp->q_org[m][1], wp->q_org[m][2]};
+        const bool valid = block_row_token(p.g, w_mode, q_org, w_kv_len, row, &token);
+        const int64_t rows = w_mode == MODE_COMPACT ? p.g.Lc : p.g.L;
+        __nv_bfloat16 *out = (w_mode == MODE_COMPACT ? p.Oc + (int64_t)wp->slice * rows * D : p.O + (int64_t)wp->out_slice * rows * D) +
                              (int64_t)token * D;
         const float inv = 1.f / row_sum;
 #pragma unroll
@@ -652,16 +670,17 @@ attention_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_consta
     if (threadIdx.x == 0) {
         const uint32_t bars = smem_u32(ctl->bars);
         for (int i = 0; i < BAR_COUNT; ++i) {
-            const bool many = (i >= BAR_P_LO && i < BAR_P_HI + 2) || (i >= BAR_O_FREE && i < BAR_O_FREE + 2);
-            mbar_init(bars + 8 * i, many ? 128 : 1);
+            // P_READY: one arrival per softmax warp; O_FREE: one per softmax thread
+            mbar_init(bars + 8 * i, i >= BAR_O_FREE && i < BAR_O_FREE + 2 ? 128 : (i >= BAR_P_READY && i < BAR_O_FREE ? 4 : 1));
         }
         ctl->abort = 0;
         ctl->tmem_base = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (threadIdx.x < kMaxMasks * 4) ctl->colmasks[threadIdx.x] = p.colmasks[threadIdx.x];
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
-    if (warp == 2) {
+    if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&ctl->tmem_base))
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -672,13 +691,12 @@ attention_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_consta
     const uint32_t tmem = ctl->tmem_base;
 
     const int32_t begin = p.cta_begin[blockIdx.x], count = p.cta_count[blockIdx.x];
-    if (warp < 4) {
-        reg_dec<64>();
-        if (warp == 0) producer_role<D>(p, maps, ctl, smem_base, begin, count, lane);
-        else if (warp == 1) mma_role<D>(p, ctl, smem_base, tmem, begin, count);
+    if (warp == 0) {
+        producer_role<D>(p, maps, ctl, smem_base, begin, count, lane);
+    } else if (warp == 1) {
+        mma_role<D>(p, ctl, smem_base, tmem, begin, count);
     } else {
-        reg_inc<216>();
-        const int m = (warp - 4) >> 2;
+        const int m = (warp - 2) >> 2;
         softmax_role<D>(p, ctl, tmem, begin, count, m, (warp & 3) * 32 + lane, warp & 3);
     }
 
@@ -688,7 +706,7 @@ attention_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_consta
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 2) {
+    if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
     }

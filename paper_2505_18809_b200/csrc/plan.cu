@@ -20,7 +20,7 @@ struct vorta_plan {
     int sm_count = 0;
     std::vector<uint8_t> routes;
     std::vector<int32_t> seg_start;   // per bucket: first slot of its core_idx segment
-    std::vector<int32_t> kv_count;    // per query tile (read back from the device)
+    std::vector<int32_t> kv_count;    // per query tile (read back from the device), then the leading unmasked ones
     std::vector<int32_t> core_heads;  // heads routed to core-set, ascending
     // device tables
     uint8_t *d_bm = nullptr;
@@ -192,6 +192,7 @@ int build_list(vorta_plan *p, vorta_plan::WorkList &wl, const std::vector<uint8_
         for (int32_t b0 = 0; b0 < nblk; b0 += 2) {
             WorkItem w{};
             w.mode = mode; w.slice = slice; w.out_slice = out_slice; w.kv_count = kv; w.kv_len = len;
+            w.kv_fast = len % kBlockM ? kv - 1 : kv;
             w.n_mblk = std::min(2, nblk - b0);
             for (int m = 0; m < w.n_mblk; ++m) w.q_org[m][0] = (b0 + m) * kBlockM;
             items.push_back(w);
@@ -210,6 +211,7 @@ int build_list(vorta_plan *p, vorta_plan::WorkList &wl, const std::vector<uint8_
                     w.mode = MODE_TILES; w.slice = slice;
                     w.out_slice = by_branch ? VORTA_ROUTE_SLIDING * BH + slice : slice;
                     w.kv_count = p->kv_count[qt];
+                    w.kv_fast = g.bn_tile == kBlockM ? p->kv_count[g.n_tiles + qt] : 0;
                     w.kv_begin = qt * g.max_kv_per_tile;
                     w.kv_len = 0;
                     int32_t t0 = q[0] * g.tile[0];
@@ -482,7 +484,7 @@ int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
     int64_t nt2 = (int64_t)g.n_tiles * g.n_tiles;
     ok = ok && cudaMalloc(&p->d_bm, (size_t)nt2) == cudaSuccess;
     ok = ok && cudaMalloc(&p->d_kv_list, sizeof(KvEntry) * (size_t)g.n_tiles * g.max_kv_per_tile) == cudaSuccess;
-    ok = ok && cudaMalloc(&p->d_kv_count, sizeof(int32_t) * g.n_tiles) == cudaSuccess;
+    ok = ok && cudaMalloc(&p->d_kv_count, sizeof(int32_t) * 2 * g.n_tiles) == cudaSuccess;
     ok = ok && cudaMalloc(&p->d_colmasks, sizeof(uint32_t) * masks.size()) == cudaSuccess;
     ok = ok && cudaMalloc(&p->d_seg_start, sizeof(int32_t) * g.n_buckets) == cudaSuccess;
     ok = ok && cudaMalloc(&p->d_bucket_tab, sizeof(int32_t) * btab.size()) == cudaSuccess;
@@ -497,8 +499,8 @@ int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
         for (auto &e : set) ok = ok && cudaEventCreate(&e) == cudaSuccess;
     // the mask builder runs once per shape; its per-tile counts come back for the work list
     ok = ok && launch_block_mask(g, p->d_bm, p->d_kv_list, p->d_kv_count, nullptr) == cudaSuccess;
-    p->kv_count.resize(g.n_tiles);
-    ok = ok && cudaMemcpy(p->kv_count.data(), p->d_kv_count, sizeof(int32_t) * g.n_tiles, cudaMemcpyDeviceToHost) == cudaSuccess;
+    p->kv_count.resize(2 * (size_t)g.n_tiles);
+    ok = ok && cudaMemcpy(p->kv_count.data(), p->d_kv_count, sizeof(int32_t) * 2 * g.n_tiles, cudaMemcpyDeviceToHost) == cudaSuccess;
     ok = ok && attention_sm100_prepare() == cudaSuccess;
     if (!ok) { cudaGetLastError(); free_device(p); delete p; return VORTA_ERR_CUDA; }
     // self-check: the lists must hold exactly the blocks the window arithmetic predicts

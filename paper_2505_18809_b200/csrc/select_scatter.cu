@@ -45,29 +45,37 @@ __global__ void kv_list_kernel(Geometry g, const uint8_t *__restrict__ bm, KvEnt
     int32_t qt = blockIdx.x * blockDim.x + threadIdx.x;
     if (qt >= g.n_tiles) return;
     KvEntry *out = list + (int64_t)qt * g.max_kv_per_tile;
-    int32_t n = 0;
-    for (int32_t kt = 0; kt < g.n_tiles; ++kt) {
-        if (!bm[(int64_t)qt * g.n_tiles + kt]) continue;
-        int32_t k[3];
-        tile_triple(g, kt, k);
-        int32_t t0 = k[0] * g.tile[0], h0 = k[1] * g.tile[1], w0 = k[2] * g.tile[2];
-        int32_t pt = (g.T - t0 < g.tile[0]), ph = (g.H - h0 < g.tile[1]), pw = (g.W - w0 < g.tile[2]);
-        for (int32_t bx = 0; bx < g.boxes_per_tile; ++bx) {
-            int32_t tb = t0 + bx * g.box[0];
-            if (tb >= g.T) break;
+    // Two passes: the boxes that lie wholly inside the grid (mask class 0) first, the cut
+    // ones after them, so that the attention kernel can run the leading blocks without
+    // any masking.  count[n_tiles + qt] is the number of leading whole boxes.
+    int32_t n = 0, n_whole = 0;
+    for (int pass = 0; pass < 2; ++pass) {
+        for (int32_t kt = 0; kt < g.n_tiles; ++kt) {
+            if (!bm[(int64_t)qt * g.n_tiles + kt]) continue;
+            int32_t k[3];
+            tile_triple(g, kt, k);
+            int32_t t0 = k[0] * g.tile[0], h0 = k[1] * g.tile[1], w0 = k[2] * g.tile[2];
+            int32_t pt = (g.T - t0 < g.tile[0]), ph = (g.H - h0 < g.tile[1]), pw = (g.W - w0 < g.tile[2]);
             bool whole = !pt && !ph && !pw && g.box_rows == g.bn_tile;
-            if (n < g.max_kv_per_tile) {
-                KvEntry e;
-                e.w0 = (int16_t)w0;
-                e.h0 = (int16_t)h0;
-                e.t0 = (int16_t)tb;
-                e.mask_id = whole ? 0 : (uint16_t)(1 + ((pt * 2 + ph) * 2 + pw) * 2 + bx);
-                out[n] = e;
+            if (whole != (pass == 0)) continue;
+            for (int32_t bx = 0; bx < g.boxes_per_tile; ++bx) {
+                int32_t tb = t0 + bx * g.box[0];
+                if (tb >= g.T) break;
+                if (n < g.max_kv_per_tile) {
+                    KvEntry e;
+                    e.w0 = (int16_t)w0;
+                    e.h0 = (int16_t)h0;
+                    e.t0 = (int16_t)tb;
+                    e.mask_id = whole ? 0 : (uint16_t)(1 + ((pt * 2 + ph) * 2 + pw) * 2 + bx);
+                    out[n] = e;
+                }
+                ++n;
             }
-            ++n;
         }
+        if (pass == 0) n_whole = n;
     }
     count[qt] = n;
+    count[g.n_tiles + qt] = n_whole;
 }
 
 cudaError_t launch_block_mask(const Geometry &g, uint8_t *bm, KvEntry *kv_list, int32_t *kv_count,

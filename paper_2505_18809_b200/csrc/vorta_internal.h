@@ -21,7 +21,7 @@ enum : int32_t {
 
 constexpr int kBlockM = 128;       // query rows per M-block (one MMA M)
 constexpr int kMaxMasks = 17;      // column-mask classes of the sliding branch (0 = none)
-constexpr int kAttnThreads = 384;  // tcgen05 kernel: 4 control warps + 2 softmax warpgroups
+constexpr int kAttnThreads = 320;  // tcgen05 kernel: 2 control warps + 2 x 4 softmax warps
 constexpr int kBucketTabStride = 34;  // per bucket shape class: token count, centre, 32 token offsets
 
 // Plain geometry, passed to kernels by value.
@@ -54,7 +54,8 @@ struct WorkItem {
     int32_t kv_len;       // linear modes: number of keys (L or Lc)
     int32_t q_org[2][3];  // per M-block: (w0, h0, t0) of the box, or (row0, 0, 0)
     int32_t out_slice;    // slice of the output tensor the rows are written to (non-compact modes)
-    int32_t pad[3];
+    int32_t kv_fast;      // the first kv_fast blocks are 128 real keys each: no column needs masking
+    int32_t pad[2];
 };
 static_assert(sizeof(WorkItem) == 64, "WorkItem must stay 64 bytes");
 
