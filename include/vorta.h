@@ -178,11 +178,19 @@ VORTA_API int vorta_routed_attention(const vorta_plan *plan, const void *Q, cons
                                      void *workspace, size_t workspace_bytes, void *stream);
 
 /*
- * The same layer with HOST buffers (bf16 [B, heads, L, d], ideally pinned):
- * copies Q, K, V to dev_scratch, runs vorta_routed_attention there, copies O
- * back, all on `stream`; returns after enqueueing (synchronise the stream before
- * reading O_host).  dev_scratch: device memory of at least
- * vorta_plan_info().host_call_scratch_bytes, 256-byte aligned.
+ * The same layer with HOST buffers (bf16 [B, heads, L, d]; pinned memory, or the
+ * copies neither overlap nor return early).  The heads are worked through in up to
+ * eight groups, most expensive first: the plan's own copy-in stream brings a group's
+ * Q, K, V into dev_scratch, the layer's kernels for that group run on `stream`, and
+ * the plan's copy-out stream returns its O, so that copies and kernels of different
+ * groups overlap.  The call starts after the work already enqueued on `stream` and
+ * `stream` ends up waiting for the last copy out: to the caller it is one operation
+ * on `stream`.  Returns after enqueueing (synchronise `stream` before reading
+ * O_host or reusing dev_scratch from another stream).  The result is the one
+ * vorta_routed_attention gives.  dev_scratch: device memory of at least
+ * vorta_plan_info().host_call_scratch_bytes, 256-byte aligned.  Two calls on the
+ * same plan must not be in flight on different streams at once (they share the
+ * plan's copy streams and events).
  */
 VORTA_API int vorta_routed_attention_host(const vorta_plan *plan, const void *Q_host,
                                           const void *K_host, const void *V_host, void *O_host,

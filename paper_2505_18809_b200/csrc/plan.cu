@@ -40,6 +40,19 @@ struct vorta_plan {
         bool built = false;
     };
     WorkList routed, mixture;
+    // The host-buffer entry point works through the heads in groups, so that the copies
+    // of one group run under the kernels of another: each group has its own work list
+    // and core-set problem tables, built with the routes.
+    struct HostChunk {
+        WorkList wl;
+        std::vector<int32_t> heads;
+        int32_t n_core = 0;
+        int32_t *d_core_slice = nullptr, *d_core_xslice = nullptr;
+        cudaEvent_t ev_in = nullptr, ev_done = nullptr;
+    };
+    std::vector<HostChunk> chunks;
+    cudaStream_t s_in = nullptr, s_out = nullptr;  // copy-in and copy-out streams of that entry point
+    cudaEvent_t ev_start = nullptr, ev_out = nullptr;
     int32_t *d_core_slice = nullptr;  // [B * n_core]: compact problem -> b*heads + head
     int32_t *d_core_xslice = nullptr; // same for a shared X with one head
     int32_t *d_status = nullptr;
@@ -137,6 +150,17 @@ void free_device(vorta_plan *p)
         cudaFree(wl->d_items); cudaFree(wl->d_cta_begin); cudaFree(wl->d_cta_count);
     }
     cudaFree(p->d_core_slice); cudaFree(p->d_core_xslice);
+    for (auto &c : p->chunks) {
+        cudaFree(c.wl.d_items); cudaFree(c.wl.d_cta_begin); cudaFree(c.wl.d_cta_count);
+        cudaFree(c.d_core_slice); cudaFree(c.d_core_xslice);
+        if (c.ev_in) cudaEventDestroy(c.ev_in);
+        if (c.ev_done) cudaEventDestroy(c.ev_done);
+    }
+    p->chunks.clear();
+    if (p->s_in) cudaStreamDestroy(p->s_in);
+    if (p->s_out) cudaStreamDestroy(p->s_out);
+    if (p->ev_start) cudaEventDestroy(p->ev_start);
+    if (p->ev_out) cudaEventDestroy(p->ev_out);
     cudaFree(p->d_status);
     for (auto &set : p->ev)
         for (auto &e : set)
@@ -287,6 +311,63 @@ int build_list(vorta_plan *p, vorta_plan::WorkList &wl, const std::vector<uint8_
     return VORTA_OK;
 }
 
+// Groups of heads for the host-buffer entry point.  Heads are taken in descending order of
+// attention work and cut into at most kHostChunks groups of equal head count (equal copy
+// time): the expensive groups run first, so the kernels always have a group to work on
+// while the copy engine brings in the cheap ones.
+constexpr int kHostChunks = 8;
+
+int build_host_chunks(vorta_plan *p)
+{
+    const Geometry &g = p->g;
+    std::vector<double> cost(g.heads);
+    for (int32_t h = 0; h < g.heads; ++h) {
+        const uint8_t r = p->routes[h];
+        cost[h] = r == VORTA_ROUTE_FULL ? (double)g.L * g.L
+                  : r == VORTA_ROUTE_SLIDING ? p->sliding_pairs : (double)g.Lc * g.Lc;
+    }
+    std::vector<int32_t> order(g.heads);
+    for (int32_t h = 0; h < g.heads; ++h) order[h] = h;
+    std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return cost[a] > cost[b]; });
+    const int32_t n_chunks = std::min<int32_t>(kHostChunks, g.heads);
+    const int32_t per = (g.heads + n_chunks - 1) / n_chunks;
+    const size_t want = (size_t)((g.heads + per - 1) / per);
+    while (p->chunks.size() < want) {
+        p->chunks.emplace_back();
+        vorta_plan::HostChunk &c = p->chunks.back();
+        if (cudaEventCreateWithFlags(&c.ev_in, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c.ev_done, cudaEventDisableTiming) != cudaSuccess ||
+            cudaMalloc(&c.d_core_slice, sizeof(int32_t) * g.B * per) != cudaSuccess ||
+            cudaMalloc(&c.d_core_xslice, sizeof(int32_t) * g.B * per) != cudaSuccess)
+            return VORTA_ERR_CUDA;
+    }
+    for (size_t ci = 0; ci < want; ++ci) {
+        vorta_plan::HostChunk &c = p->chunks[ci];
+        c.heads.assign(order.begin() + ci * per, order.begin() + std::min<size_t>((ci + 1) * per, g.heads));
+        std::sort(c.heads.begin(), c.heads.end());
+        std::vector<uint8_t> branches(g.heads, 0);
+        std::vector<int32_t> core;
+        for (int32_t h : c.heads) {
+            branches[h] = (uint8_t)(1u << p->routes[h]);
+            if (p->routes[h] == VORTA_ROUTE_CORESET) core.push_back(h);
+        }
+        int rc = build_list(p, c.wl, branches, false);
+        if (rc != VORTA_OK) return rc;
+        c.n_core = (int32_t)core.size();
+        std::vector<int32_t> cs((size_t)g.B * std::max(c.n_core, 1)), cx(cs.size());
+        for (int32_t b = 0; b < g.B; ++b)
+            for (int32_t k = 0; k < c.n_core; ++k) {
+                cs[(size_t)b * c.n_core + k] = b * g.heads + core[k];
+                cx[(size_t)b * c.n_core + k] = b;
+            }
+        if (c.n_core &&
+            (cudaMemcpy(c.d_core_slice, cs.data(), sizeof(int32_t) * g.B * c.n_core, cudaMemcpyHostToDevice) != cudaSuccess ||
+             cudaMemcpy(c.d_core_xslice, cx.data(), sizeof(int32_t) * g.B * c.n_core, cudaMemcpyHostToDevice) != cudaSuccess))
+            return VORTA_ERR_CUDA;
+    }
+    return VORTA_OK;
+}
+
 // (Re)build the work list for the current routes.
 int build_work(vorta_plan *p)
 {
@@ -310,7 +391,7 @@ int build_work(vorta_plan *p)
         (cudaMemcpy(p->d_core_slice, core_slice.data(), sizeof(int32_t) * g.B * n_core, cudaMemcpyHostToDevice) != cudaSuccess ||
          cudaMemcpy(p->d_core_xslice, core_x.data(), sizeof(int32_t) * g.B * n_core, cudaMemcpyHostToDevice) != cudaSuccess))
         return VORTA_ERR_CUDA;
-    return VORTA_OK;
+    return build_host_chunks(p);
 }
 
 struct DeviceGuard {
@@ -497,6 +578,10 @@ int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
     ok = ok && cudaMemcpy(p->d_seg_start, p->seg_start.data(), sizeof(int32_t) * g.n_buckets, cudaMemcpyHostToDevice) == cudaSuccess;
     for (auto &set : p->ev)
         for (auto &e : set) ok = ok && cudaEventCreate(&e) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&p->s_in, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&p->s_out, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&p->ev_start, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&p->ev_out, cudaEventDisableTiming) == cudaSuccess;
     // the mask builder runs once per shape; its per-tile counts come back for the work list
     ok = ok && launch_block_mask(g, p->d_bm, p->d_kv_list, p->d_kv_count, nullptr) == cudaSuccess;
     p->kv_count.resize(2 * (size_t)g.n_tiles);
@@ -818,17 +903,51 @@ int vorta_routed_attention_host(const vorta_plan *p, const void *Qh, const void 
     DeviceGuard guard(p->device);
     if (!guard.ok) return VORTA_ERR_CUDA;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const int64_t tb = tensor_bytes(p->g), tba = align_up(tb, 256);
+    const Geometry &g = p->g;
+    const int64_t tb = tensor_bytes(g), tba = align_up(tb, 256);
     char *base = static_cast<char *>(scratch);
-    void *dq = base, *dk = base + tba, *dv = base + 2 * tba, *dO = base + 3 * tba, *ws = base + 4 * tba;
-    if (cudaMemcpyAsync(dq, Qh, tb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(dk, Kh, tb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(dv, Vh, tb, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    char *dq = base, *dk = base + tba, *dv = base + 2 * tba, *dO = base + 3 * tba;
+    void *ws = info.workspace_bytes ? base + 4 * tba : nullptr;
+    const char *hq = static_cast<const char *>(Qh), *hk = static_cast<const char *>(Kh),
+               *hv = static_cast<const char *>(Vh);
+    char *ho = static_cast<char *>(Oh);
+    const int64_t hb = (int64_t)g.L * g.d * (int64_t)sizeof(__nv_bfloat16);  // one head of one tensor
+
+    // Three queues: copies in (own stream), kernels (the caller's stream), copies out (own
+    // stream).  Group c's kernels wait for its copies in; its copy out waits for its kernels.
+    // Everything starts after the work already in the caller's stream and the caller's stream
+    // ends up waiting for the last copy out, so the call as a whole behaves as one operation
+    // enqueued on `stream`.
+    if (cudaEventRecord(p->ev_start, s) != cudaSuccess || cudaStreamWaitEvent(p->s_in, p->ev_start, 0) != cudaSuccess ||
+        cudaStreamWaitEvent(p->s_out, p->ev_start, 0) != cudaSuccess)
         return VORTA_ERR_CUDA;
-    int rc = vorta_routed_attention(p, dq, dk, dv, dO, nullptr, 0, info.workspace_bytes ? ws : nullptr,
-                                    (size_t)info.workspace_bytes, stream);
-    if (rc != VORTA_OK) return rc;
-    if (cudaMemcpyAsync(Oh, dO, tb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return VORTA_ERR_CUDA;
+    for (const vorta_plan::HostChunk &c : p->chunks) {
+        for (int32_t b = 0; b < g.B; ++b)
+            for (int32_t h : c.heads) {
+                const int64_t off = ((int64_t)b * g.heads + h) * hb;
+                if (cudaMemcpyAsync(dq + off, hq + off, hb, cudaMemcpyHostToDevice, p->s_in) != cudaSuccess ||
+                    cudaMemcpyAsync(dk + off, hk + off, hb, cudaMemcpyHostToDevice, p->s_in) != cudaSuccess ||
+                    cudaMemcpyAsync(dv + off, hv + off, hb, cudaMemcpyHostToDevice, p->s_in) != cudaSuccess)
+                    return VORTA_ERR_CUDA;
+            }
+        if (cudaEventRecord(c.ev_in, p->s_in) != cudaSuccess || cudaStreamWaitEvent(s, c.ev_in, 0) != cudaSuccess)
+            return VORTA_ERR_CUDA;
+        __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(dO);
+        int rc = run_layer(p, c.wl, c.n_core, c.d_core_slice, c.d_core_xslice, reinterpret_cast<const __nv_bfloat16 *>(dq),
+                           reinterpret_cast<const __nv_bfloat16 *>(dk), reinterpret_cast<const __nv_bfloat16 *>(dv), o, o,
+                           nullptr, 0, ws, s, false);
+        if (rc != VORTA_OK) return rc;
+        if (cudaEventRecord(c.ev_done, s) != cudaSuccess || cudaStreamWaitEvent(p->s_out, c.ev_done, 0) != cudaSuccess)
+            return VORTA_ERR_CUDA;
+        for (int32_t b = 0; b < g.B; ++b)
+            for (int32_t h : c.heads) {
+                const int64_t off = ((int64_t)b * g.heads + h) * hb;
+                if (cudaMemcpyAsync(ho + off, dO + off, hb, cudaMemcpyDeviceToHost, p->s_out) != cudaSuccess)
+                    return VORTA_ERR_CUDA;
+            }
+    }
+    if (cudaEventRecord(p->ev_out, p->s_out) != cudaSuccess || cudaStreamWaitEvent(s, p->ev_out, 0) != cudaSuccess)
+        return VORTA_ERR_CUDA;
     return VORTA_OK;
 }
 

@@ -263,6 +263,29 @@ def test_host_buffer_entry_point_matches_device_path():
     p.close()
 
 
+def test_host_buffer_entry_point_many_heads_batch_and_route_change():
+    """More heads than groups (several heads per group, uneven last group), a batch of two,
+    two calls in a row on the same scratch, then new routes: always the device path's bits."""
+    routes = (0, 1, 2, 1, 2, 2, 1, 0, 1, 1, 2)
+    wl = Workload("host-groups", (5, 9, 11), len(routes), 128, (2, 4, 4), (3, 3, 3), 0.5, routes, 31, False, 2)
+    Q, K, V = workloads.make_qkv(wl, DEV)
+    p = vb.Plan.from_workload(wl)
+    Qh, Kh, Vh = (t.cpu().pin_memory() for t in (Q, K, V))
+    scratch = torch.empty(p.info.host_call_scratch_bytes, dtype=torch.uint8, device=DEV)
+    for step in range(3):
+        if step == 2:
+            routes = tuple((r + 1) % 3 for r in routes)
+            p.set_routes(routes)
+            wl = Workload("host-groups", wl.grid, wl.heads, wl.d, wl.tile, wl.window, wl.ratio, routes, 31, False, 2)
+            scratch = torch.empty(p.info.host_call_scratch_bytes, dtype=torch.uint8, device=DEV)
+        O = run_layer(p, wl, Q, K, V, vb.VORTA_KERNEL_TCGEN05)
+        Oh = torch.full_like(Qh, float("nan")).pin_memory()
+        p.routed_attention_host(Qh, Kh, Vh, Oh, scratch)
+        assert p.device_status() == 0
+        assert torch.equal(Oh.view(torch.int16), O.cpu().view(torch.int16)), step
+    p.close()
+
+
 # --------------------------------------------------------------------------- the named configurations
 def check_config(wl, rows_per_head, kernels=(vb.VORTA_KERNEL_TCGEN05,)):
     Q, K, V = workloads.make_qkv(wl, DEV)
