@@ -37,9 +37,9 @@ UNIT = "TFLOP/s"
 DEFAULT_WORKLOAD = "hunyuan-720p"
 FALLBACK_PEAK_TFLOPS = 1590.0   # used only if MEASURED_PEAKS.json is absent
 # DRAM traffic of the attention kernel: the ncu capture of the three-head profiling case
-# (profiles/attention_sm100_kernel__hunyuan-720p-3h.md) read 477.2 MB and wrote 81.4 MB for 304.0 MB of
+# (profiles/attention_sm100_kernel__hunyuan-720p-3h.md) read 441.5 MB and wrote 62.6 MB for 304.1 MB of
 # algorithmic bytes; a launch of another workload is estimated by the same ratio.
-ATTENTION_TRAFFIC_PER_ALGORITHMIC_BYTE = 558.6 / 304.0
+ATTENTION_TRAFFIC_PER_ALGORITHMIC_BYTE = 504.1 / 304.1
 
 
 def attention_algorithmic_bytes(info, wl) -> float:
