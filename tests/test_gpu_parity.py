@@ -42,6 +42,18 @@ def small_workloads():
         W("ratio-one", (4, 6, 8), 2, 64, (2, 3, 4), (3, 3, 3), 1.0, (2, 2), 26, False),
         # bucket other than the default, grid smaller than one tile on T
         W("bucket-133", (1, 14, 15), 2, 128, (2, 4, 4), (3, 3, 3), 0.34, (2, 1), 27, False, 1, (1, 3, 3)),
+        # the attention kernel's sub-block pipeline at its shortest: window of one tile, so an item has
+        # one KV block: 1 sub-block (32- and 64-token tiles), 2 (128-token tile), 4 (256-token tile)
+        W("one-sub-32", (4, 8, 8), 2, 128, (2, 4, 4), (1, 1, 1), 0.5, (1, 1), 41, False),
+        W("one-sub-64", (8, 8, 8), 2, 64, (4, 4, 4), (1, 1, 1), 0.5, (1, 2), 42, False),
+        W("two-sub-128", (4, 8, 16), 2, 128, (2, 8, 8), (1, 1, 1), 0.5, (1, 0), 43, False),
+        W("four-sub-256", (8, 8, 16), 2, 128, (4, 8, 8), (1, 1, 1), 0.5, (1, 2), 44, False),
+        # odd numbers of sub-blocks (3 KV tiles of 64 tokens in a window) and a cut last tile
+        W("three-sub-64", (4, 4, 11), 2, 128, (4, 4, 4), (1, 1, 3), 0.5, (1, 1), 45, False),
+        # linear heads shorter than one block: 40 tokens (second sub-block all masked), 70 and 129 tokens
+        W("linear-40", (2, 4, 5), 2, 128, (2, 4, 4), (3, 3, 3), 1.0, (0, 2), 46, False),
+        W("linear-70", (2, 5, 7), 2, 64, (2, 4, 4), (3, 3, 3), 0.6, (0, 2), 47, False),
+        W("linear-129", (1, 3, 43), 2, 128, (1, 4, 4), (3, 3, 3), 0.5, (0, 2), 48, False),
     ]
 
 
