@@ -254,6 +254,18 @@ def run_ours(args):
 
     wl = get_workload(args.workload)
     pk = peaks()
+    full_layer_flops = None
+    if args.shard_heads:
+        # strong scaling: ONE layer, its heads split over the ranks by the library's partition
+        # (head-sharded Q, K, V, no collective on the data path); every rank makes only its heads
+        from paper_2505_18809_b200 import sharding
+        if world > wl.heads:
+            raise SystemExit("--shard-heads needs at least one head per rank")
+        host_plan = vb.Plan.from_workload(wl, host_only=True)
+        full_layer_flops = host_plan.info.flops_layer
+        host_plan.close()
+        rank_of_head, _ = sharding.shard_heads(wl, world)
+        wl = sharding.local_workload(wl, sharding.heads_of_rank(rank_of_head, rank))
     # every rank holds its own layer (heads are independent: no exchange inside the op)
     Q, K, V = workloads.make_qkv(wl, dev)
     O = torch.empty_like(Q)
@@ -310,6 +322,8 @@ def run_ours(args):
     ms_total = reduce_max_ms(ms_total, world, dev)
     ms_step = ms_total / args.steps
     value = whole_job_tflops(flops_step, world, ms_step)
+    if full_layer_flops is not None:
+        value = full_layer_flops / (ms_step * 1e-3) / 1e12   # the whole layer over the slowest rank's time
 
     # stage times of the timed steps (CUDA events recorded by the library on the same stream)
     n_hist = min(args.steps, 64)
@@ -344,7 +358,8 @@ def run_ours(args):
                  "hbm_peak_gbs": pk["hbm"]}
         out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "ms_per_layer": ms_step,
-               "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+               "higher_is_better": True, "scaling": "strong" if args.shard_heads else "weak", "vs_baseline": None,
+               "dtype": "bf16",
                "data": "synthetic",
                "config": {"workload": wl.name + ("+soft-mixture" if args.mixture else ""), "grid": list(wl.grid),
                           "tokens": wl.L, "heads": wl.heads,
@@ -354,7 +369,9 @@ def run_ours(args):
                           "algorithmic_tflop_per_layer": info.flops_layer / 1e12,
                           "issued_tflop_per_layer": info.flops_issued_layer / 1e12,
                           "l2": "inputs (3 x %.0f MB) larger than L2" % (Q.numel() * 2 / 1e6),
-                          "per_rank": "one layer per GPU, no collective on the data path"},
+                          "per_rank": ("heads of one layer split over the GPUs (vorta_shard_heads), no collective on the "
+                                       "data path; roofline and stages are rank 0's share") if args.shard_heads
+                          else "one layer per GPU, no collective on the data path"},
                "frac_of_bf16_peak": value / world / pk["bf16"],
                "roofline": roofline, "stages": stage, "gpu_launches": launches, "clocks": clocks}
 
@@ -375,7 +392,9 @@ def run_ours(args):
         barrier()
         ms_e2e = reduce_max_ms(e0.elapsed_time(e1) / n_e2e, world, dev)
         tb = Q.numel() * 2
-        e2e = {"value": whole_job_tflops(info.flops_layer, world, ms_e2e), "unit": UNIT,
+        e2e_value = (full_layer_flops / (ms_e2e * 1e-3) / 1e12 if full_layer_flops is not None
+                     else whole_job_tflops(info.flops_layer, world, ms_e2e))
+        e2e = {"value": e2e_value, "unit": UNIT,
                "ms_per_step": ms_e2e, "steps": n_e2e, "h2d_bytes_per_step": 3 * tb, "d2h_bytes_per_step": tb,
                "api": "vorta_routed_attention_host (pinned host Q, K, V in; O out)"}
         del scratch, Qh, Kh, Vh
@@ -413,6 +432,8 @@ def main():
     ap.add_argument("--reference-rows", type=int, default=16, help="oracle rows per head per step (--impl reference)")
     ap.add_argument("--kernel", type=int, default=-1, help="attention kernel id (see vorta.h); -1 = library default")
     ap.add_argument("--mixture", action="store_true", help="time vorta_soft_mixture (all three branches per head)")
+    ap.add_argument("--shard-heads", action="store_true",
+                    help="strong scaling: one layer, heads split over the ranks (default: one layer per rank)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -134,6 +134,23 @@ VORTA_API int vorta_plan_destroy(vorta_plan *plan);
 VORTA_API int vorta_plan_info(const vorta_plan *plan, vorta_plan_info_t *out);
 
 /*
+ * Head-sharded multi-GPU use (heads are independent units: no exchange inside the
+ * op): split the heads of the current routes over n_ranks devices so that the most
+ * loaded rank is as light as longest-processing-time-first packing makes it.  The
+ * cost of a head is its attention work under its route (flops_full_head,
+ * flops_sliding_head or flops_coreset_head of vorta_plan_info).  Heads are taken in
+ * descending cost (ties: ascending head index) and each goes to the rank with the
+ * least work so far (ties: lowest rank).  Host arrays:
+ *   rank_of_head   out, [heads]: rank in [0, n_ranks) of every head
+ *   rank_flops     out, [n_ranks] or NULL: attention FLOPs per batch entry of each rank
+ * Works on host-only plans.  The paper runs on one GPU; this is the partition a
+ * caller with head-sharded Q, K, V (e.g. after an all-to-all upstream) needs, each
+ * rank then creating a plan over its own heads.
+ */
+VORTA_API int vorta_shard_heads(const vorta_plan *plan, int32_t n_ranks, int32_t *rank_of_head,
+                                double *rank_flops);
+
+/*
  * Copy the canonical block mask to host memory: out_host is uint8
  * [n_tiles * n_tiles], BM[qt*n_tiles + kt] = 1 iff key tile kt lies in the window
  * of query tile qt (Algorithm 1 applied to tile ids, the query tile first moved

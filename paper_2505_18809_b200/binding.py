@@ -30,7 +30,7 @@ EXPORTS = (
     "vorta_routed_attention", "vorta_routed_attention_host", "vorta_plan_set_profiling",
     "vorta_plan_stage_ms", "vorta_plan_stage_ms_at", "vorta_plan_last_launches", "vorta_device_status",
     "vorta_status_string", "vorta_routed_attention_static", "vorta_plan_device",
-    "vorta_router_gates", "vorta_soft_mixture",
+    "vorta_router_gates", "vorta_soft_mixture", "vorta_shard_heads",
 )
 VORTA_STATIC_WORKSPACE_BYTES = 16 * 1024 * 1024
 
@@ -136,6 +136,15 @@ def vorta_plan_info(plan: int) -> vorta_plan_info_t:
     info = vorta_plan_info_t()
     _check(lib().vorta_plan_info(plan, ctypes.byref(info)), "vorta_plan_info")
     return info
+
+
+def vorta_shard_heads(plan: int, heads: int, n_ranks: int):
+    """(rank_of_head int32 [heads], rank_flops float64 [n_ranks]) of the current routes."""
+    rank_of_head = np.zeros(heads, dtype=np.int32)
+    rank_flops = np.zeros(n_ranks, dtype=np.float64)
+    _check(lib().vorta_shard_heads(plan, int(n_ranks), rank_of_head.ctypes.data_as(ctypes.c_void_p),
+                                   rank_flops.ctypes.data_as(ctypes.c_void_p)), "vorta_shard_heads")
+    return rank_of_head, rank_flops
 
 
 def vorta_plan_block_mask(plan: int, n_tiles: int) -> np.ndarray:

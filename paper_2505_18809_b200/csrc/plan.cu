@@ -659,6 +659,33 @@ int vorta_plan_device(const vorta_plan *p, int32_t *device)
     return VORTA_OK;
 }
 
+int vorta_shard_heads(const vorta_plan *p, int32_t n_ranks, int32_t *rank_of_head, double *rank_flops)
+{
+    if (!p || !rank_of_head || n_ranks < 1) return VORTA_ERR_INVALID_ARG;
+    const Geometry &g = p->g;
+    vorta_plan_info_t info;
+    int rc = vorta_plan_info(p, &info);
+    if (rc != VORTA_OK) return rc;
+    std::vector<double> cost(g.heads);
+    for (int32_t h = 0; h < g.heads; ++h)
+        cost[h] = p->routes[h] == VORTA_ROUTE_FULL ? info.flops_full_head
+                  : p->routes[h] == VORTA_ROUTE_SLIDING ? info.flops_sliding_head : info.flops_coreset_head;
+    std::vector<int32_t> order(g.heads);
+    for (int32_t h = 0; h < g.heads; ++h) order[h] = h;
+    std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return cost[a] > cost[b]; });
+    std::vector<double> load((size_t)n_ranks, 0.0);
+    for (int32_t h : order) {
+        int32_t best = 0;
+        for (int32_t r = 1; r < n_ranks; ++r)
+            if (load[r] < load[best]) best = r;
+        rank_of_head[h] = best;
+        load[best] += cost[h];
+    }
+    if (rank_flops)
+        for (int32_t r = 0; r < n_ranks; ++r) rank_flops[r] = load[r];
+    return VORTA_OK;
+}
+
 int vorta_plan_block_mask(const vorta_plan *p, uint8_t *out_host)
 {
     if (!p || !out_host) return VORTA_ERR_INVALID_ARG;
