@@ -18,7 +18,11 @@
  *   - the similarity of bucketed core-set selection is the cosine;
  *   - keep(n) = max(1, floor(r*n + 1/2)) tokens survive in a bucket of n tokens;
  *   - by default pruned tokens are NOT merged into the centre: they only receive
- *     the centre's output row at unpool time; the optional merge is the plain mean.
+ *     the centre's output row at unpool time; the optional merge is the plain mean;
+ *   - joint sequences of MMDiT models (video tokens followed by Lt text tokens; the
+ *     paper runs HunyuanVideo, Section 4, but does not say how its branches treat the
+ *     text tokens): a text key is visible to every query, a text query sees every
+ *     key, and core-set selection prunes video tokens only.
  *
  * Pinned by tests/test_oracle_pins.py against: brute-force dense attention with
  * explicit masks built a different way (numpy), torch's fp64
@@ -221,17 +225,22 @@ VO_API int vo_attn_full(int64_t L, int32_t d, const double *Q, const double *K, 
  * Sliding tile attention: Eq. 2 with scores outside Algorithm 1's mask removed.
  * For each query row the mask row is evaluated pair by pair, exactly as the
  * double loop of Algorithm 1 does, and the row attends to the keys it keeps.
+ *
+ * Joint sequence: Q, K, V hold the L = T*H*W video tokens followed by Lt text
+ * tokens.  A video query keeps the video keys of Algorithm 1's mask and every
+ * text key; a text query keeps every key.  P, if not NULL, is [nq, L + Lt].
  */
-VO_API int vo_attn_sliding(const int32_t v[3], const int32_t t[3], const int32_t w[3], int32_t d,
-                           const double *Q, const double *K, const double *V, double scale,
-                           int64_t nq, const int64_t *q_rows, double *O, double *P)
+VO_API int vo_attn_sliding_joint(const int32_t v[3], const int32_t t[3], const int32_t w[3], int64_t Lt,
+                                 int32_t d, const double *Q, const double *K, const double *V, double scale,
+                                 int64_t nq, const int64_t *q_rows, double *O, double *P)
 {
     int64_t L = (int64_t)v[0] * v[1] * v[2];
+    int64_t Ltot = L + Lt;
     int err = 0;
 #pragma omp parallel
     {
-        double *s = (double *)malloc(sizeof(double) * (size_t)L);
-        int64_t *keys = (int64_t *)malloc(sizeof(int64_t) * (size_t)L);
+        double *s = (double *)malloc(sizeof(double) * (size_t)Ltot);
+        int64_t *keys = (int64_t *)malloc(sizeof(int64_t) * (size_t)Ltot);
         if (!s || !keys) {
 #pragma omp atomic write
             err = 1;
@@ -243,11 +252,12 @@ VO_API int vo_attn_sliding(const int32_t v[3], const int32_t t[3], const int32_t
                 int64_t i = q_rows ? q_rows[r] : r;
                 int64_t nk = 0;
                 for (int64_t j = 0; j < L; ++j)
-                    if (sta_mask_pair(i, j, v, t, w)) keys[nk++] = j;
+                    if (i >= L || sta_mask_pair(i, j, v, t, w)) keys[nk++] = j;
+                for (int64_t j = L; j < Ltot; ++j) keys[nk++] = j;
                 attend_row(Q + i * d, K, V, d, keys, nk, scale, O + r * d, s);
                 if (P) {
-                    double *prow = P + r * L;
-                    for (int64_t j = 0; j < L; ++j) prow[j] = 0.0;
+                    double *prow = P + r * Ltot;
+                    for (int64_t j = 0; j < Ltot; ++j) prow[j] = 0.0;
                     for (int64_t jj = 0; jj < nk; ++jj) prow[keys[jj]] = s[jj];
                 }
             }
@@ -256,6 +266,13 @@ VO_API int vo_attn_sliding(const int32_t v[3], const int32_t t[3], const int32_t
         free(keys);
     }
     return err;
+}
+
+VO_API int vo_attn_sliding(const int32_t v[3], const int32_t t[3], const int32_t w[3], int32_t d,
+                           const double *Q, const double *K, const double *V, double scale,
+                           int64_t nq, const int64_t *q_rows, double *O, double *P)
+{
+    return vo_attn_sliding_joint(v, t, w, 0, d, Q, K, V, scale, nq, q_rows, O, P);
 }
 
 /* ------------------------------------------------------------------------- */
@@ -411,14 +428,21 @@ VO_API int64_t vo_coreset_select(const int32_t v[3], const int32_t b[3], double 
  * become the mean over the centre and the tokens pruned from its bucket.  With a bucket
  * that keeps one token this is average pooling (the AP variants of Section 4.2).
  */
-VO_API int64_t vo_attn_coreset_ex(const int32_t v[3], const int32_t b[3], double r, int32_t d,
-                                  const double *Q, const double *K, const double *V, const double *X,
-                                  int32_t dx, double scale, int64_t nq, const int64_t *q_rows,
-                                  double *O, int32_t *core_idx, int32_t *src_slot, int merge)
+/*
+ * Joint sequence (Lt text tokens after the L video tokens in Q, K, V; X holds at least
+ * the L video rows): selection runs on the video tokens only, every text token is kept.
+ * The compact sequences are the Lc kept video tokens followed by the Lt text tokens; a
+ * text query row i >= L reads compact row Lc + (i - L).  Returns Lc (video tokens kept).
+ */
+VO_API int64_t vo_attn_coreset_joint(const int32_t v[3], const int32_t b[3], double r, int64_t Lt, int32_t d,
+                                     const double *Q, const double *K, const double *V, const double *X,
+                                     int32_t dx, double scale, int64_t nq, const int64_t *q_rows,
+                                     double *O, int32_t *core_idx, int32_t *src_slot, int merge)
 {
     int64_t L = (int64_t)v[0] * v[1] * v[2];
-    int64_t Lc = vo_coreset_select(v, b, r, X, dx, core_idx, src_slot, NULL);
-    if (Lc < 0) return -1;
+    int64_t Lv = vo_coreset_select(v, b, r, X, dx, core_idx, src_slot, NULL);
+    if (Lv < 0) return -1;
+    int64_t Lc = Lv + Lt; /* rows of the compact sequences */
 
     /* pool: the compact sequences */
     double *Qc = (double *)malloc(sizeof(double) * (size_t)(Lc * d));
@@ -431,9 +455,10 @@ VO_API int64_t vo_attn_coreset_ex(const int32_t v[3], const int32_t b[3], double
     int64_t *need = (int64_t *)malloc(sizeof(int64_t) * (size_t)Lc); /* slot -> dense id or -1 */
     if (!Kc || !Vc || !slot_of_row || !need) return -1;
     for (int64_t s = 0; s < Lc; ++s) {
-        memcpy(Qc + s * d, Q + (int64_t)core_idx[s] * d, sizeof(double) * (size_t)d);
-        memcpy(Kc + s * d, K + (int64_t)core_idx[s] * d, sizeof(double) * (size_t)d);
-        memcpy(Vc + s * d, V + (int64_t)core_idx[s] * d, sizeof(double) * (size_t)d);
+        int64_t src = s < Lv ? (int64_t)core_idx[s] : L + (s - Lv); /* kept video token, or text token */
+        memcpy(Qc + s * d, Q + src * d, sizeof(double) * (size_t)d);
+        memcpy(Kc + s * d, K + src * d, sizeof(double) * (size_t)d);
+        memcpy(Vc + s * d, V + src * d, sizeof(double) * (size_t)d);
         need[s] = -1;
         members[s] = 1;
     }
@@ -449,7 +474,7 @@ VO_API int64_t vo_attn_coreset_ex(const int32_t v[3], const int32_t b[3], double
             }
             members[s] += 1;
         }
-        for (int64_t s = 0; s < Lc; ++s)
+        for (int64_t s = 0; s < Lv; ++s)
             if (members[s] > 1)
                 for (int32_t c = 0; c < d; ++c) {
                     Qc[s * d + c] /= (double)members[s];
@@ -460,8 +485,8 @@ VO_API int64_t vo_attn_coreset_ex(const int32_t v[3], const int32_t b[3], double
     int64_t n_need = 0;
     for (int64_t rr = 0; rr < nq; ++rr) {
         int64_t i = q_rows ? q_rows[rr] : rr;
-        if (i < 0 || i >= L) return -1;
-        int64_t s = src_slot[i];
+        if (i < 0 || i >= L + Lt) return -1;
+        int64_t s = i < L ? (int64_t)src_slot[i] : Lv + (i - L);
         if (need[s] < 0) need[s] = n_need++;
         slot_of_row[rr] = s;
     }
@@ -502,7 +527,15 @@ VO_API int64_t vo_attn_coreset_ex(const int32_t v[3], const int32_t b[3], double
     free(need);
     free(slots);
     free(Oc);
-    return err ? -1 : Lc;
+    return err ? -1 : Lv;
+}
+
+VO_API int64_t vo_attn_coreset_ex(const int32_t v[3], const int32_t b[3], double r, int32_t d,
+                                  const double *Q, const double *K, const double *V, const double *X,
+                                  int32_t dx, double scale, int64_t nq, const int64_t *q_rows,
+                                  double *O, int32_t *core_idx, int32_t *src_slot, int merge)
+{
+    return vo_attn_coreset_joint(v, b, r, 0, d, Q, K, V, X, dx, scale, nq, q_rows, O, core_idx, src_slot, merge);
 }
 
 VO_API int64_t vo_attn_coreset(const int32_t v[3], const int32_t b[3], double r, int32_t d,

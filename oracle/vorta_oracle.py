@@ -53,6 +53,9 @@ def _load() -> ctypes.CDLL:
     lib.vo_attn_sliding.argtypes = [_i32p, _i32p, _i32p, ctypes.c_int32, _f64p, _f64p, _f64p,
                                     ctypes.c_double, ctypes.c_int64, _i64p, _f64p, _f64p]
     lib.vo_attn_sliding.restype = ctypes.c_int
+    lib.vo_attn_sliding_joint.argtypes = [_i32p, _i32p, _i32p, ctypes.c_int64, ctypes.c_int32, _f64p, _f64p,
+                                          _f64p, ctypes.c_double, ctypes.c_int64, _i64p, _f64p, _f64p]
+    lib.vo_attn_sliding_joint.restype = ctypes.c_int
     lib.vo_coreset_len.argtypes = [_i32p, _i32p, ctypes.c_double]
     lib.vo_coreset_len.restype = ctypes.c_int64
     lib.vo_coreset_select.argtypes = [_i32p, _i32p, ctypes.c_double, _f64p, ctypes.c_int32,
@@ -64,6 +67,10 @@ def _load() -> ctypes.CDLL:
     lib.vo_attn_coreset.restype = ctypes.c_int64
     lib.vo_attn_coreset_ex.argtypes = lib.vo_attn_coreset.argtypes + [ctypes.c_int]
     lib.vo_attn_coreset_ex.restype = ctypes.c_int64
+    lib.vo_attn_coreset_joint.argtypes = [_i32p, _i32p, ctypes.c_double, ctypes.c_int64, ctypes.c_int32, _f64p,
+                                          _f64p, _f64p, _f64p, ctypes.c_int32, ctypes.c_double, ctypes.c_int64,
+                                          _i64p, _f64p, _i32p, _i32p, ctypes.c_int]
+    lib.vo_attn_coreset_joint.restype = ctypes.c_int64
     lib.vo_num_threads.argtypes = []
     lib.vo_num_threads.restype = ctypes.c_int
     _lib = lib
@@ -126,17 +133,20 @@ def attn_full(Q, K, V, scale: float, q_rows=None, return_probs: bool = False):
 
 
 def attn_sliding(grid, tile, window, Q, K, V, scale: float, q_rows=None,
-                 return_probs: bool = False):
-    """Sliding tile attention (Algorithm 1's mask on Eq. 2) for one head."""
+                 return_probs: bool = False, text: int = 0):
+    """Sliding tile attention (Algorithm 1's mask on Eq. 2) for one head.
+
+    text: Q, K, V hold that many text tokens after the video tokens (joint sequence): text
+    keys are visible to every query and text queries see every key."""
     Q, K, V = _f64(Q), _f64(K), _f64(V)
     L, d = Q.shape
-    assert L == int(grid[0]) * int(grid[1]) * int(grid[2])
+    assert L == int(grid[0]) * int(grid[1]) * int(grid[2]) + int(text)
     rows, nq = _rows(q_rows, L)
     O = np.zeros((nq, d), dtype=np.float64)
     P = np.zeros((nq, L), dtype=np.float64) if return_probs else None
-    rc = _load().vo_attn_sliding(_triple(grid), _triple(tile), _triple(window), d, _ptr(Q, _f64p),
-                                 _ptr(K, _f64p), _ptr(V, _f64p), float(scale), nq,
-                                 _ptr(rows, _i64p), _ptr(O, _f64p), _ptr(P, _f64p))
+    rc = _load().vo_attn_sliding_joint(_triple(grid), _triple(tile), _triple(window), int(text), d,
+                                       _ptr(Q, _f64p), _ptr(K, _f64p), _ptr(V, _f64p), float(scale), nq,
+                                       _ptr(rows, _i64p), _ptr(O, _f64p), _ptr(P, _f64p))
     if rc != 0:
         raise MemoryError("vo_attn_sliding")
     return (O, P) if return_probs else O
@@ -168,25 +178,28 @@ def coreset_select(grid, bucket, ratio: float, X, return_gap: bool = False):
 
 
 def attn_coreset(grid, bucket, ratio: float, Q, K, V, scale: float, X=None, q_rows=None,
-                 merge: bool = False):
+                 merge: bool = False, text: int = 0):
     """Core-set attention (unpool . attn . pool) for one head.
 
     X defaults to K.  merge: the centre's Q, K, V rows become the mean over the centre and
-    the tokens pruned from its bucket.  Returns (O [nq, d], core_idx, src_slot).
+    the tokens pruned from its bucket.  text: Q, K, V (and X) hold that many text tokens after
+    the video tokens; selection prunes video tokens only and every text token is kept.
+    Returns (O [nq, d], core_idx [kept video tokens], src_slot [video tokens]).
     """
     Q, K, V = _f64(Q), _f64(K), _f64(V)
     X = K if X is None else _f64(X)
-    L, d = Q.shape
-    assert X.shape[0] == L
-    rows, nq = _rows(q_rows, L)
+    Ltot, d = Q.shape
+    L = Ltot - int(text)
+    assert L == int(grid[0]) * int(grid[1]) * int(grid[2]) and X.shape[0] >= L
+    rows, nq = _rows(q_rows, Ltot)
     Lc = coreset_len(grid, bucket, ratio)
     O = np.zeros((nq, d), dtype=np.float64)
     core_idx = np.zeros(Lc, dtype=np.int32)
     src_slot = np.zeros(L, dtype=np.int32)
-    got = _load().vo_attn_coreset_ex(_triple(grid), _triple(bucket), float(ratio), d, _ptr(Q, _f64p),
-                                     _ptr(K, _f64p), _ptr(V, _f64p), _ptr(X, _f64p), X.shape[1],
-                                     float(scale), nq, _ptr(rows, _i64p), _ptr(O, _f64p),
-                                     _ptr(core_idx, _i32p), _ptr(src_slot, _i32p), int(bool(merge)))
+    got = _load().vo_attn_coreset_joint(_triple(grid), _triple(bucket), float(ratio), int(text), d,
+                                        _ptr(Q, _f64p), _ptr(K, _f64p), _ptr(V, _f64p), _ptr(X, _f64p),
+                                        X.shape[1], float(scale), nq, _ptr(rows, _i64p), _ptr(O, _f64p),
+                                        _ptr(core_idx, _i32p), _ptr(src_slot, _i32p), int(bool(merge)))
     if got != Lc:
         raise RuntimeError(f"vo_attn_coreset returned {got}, expected {Lc}")
     return O, core_idx, src_slot
@@ -212,10 +225,10 @@ def router_gates(T, WR):
     return gates, routes
 
 
-def soft_mixture(grid, tile, window, bucket, ratio, Q, K, V, scale, gates, q_rows=None):
+def soft_mixture(grid, tile, window, bucket, ratio, Q, K, V, scale, gates, q_rows=None, text: int = 0):
     """Eq. 5 for one head: gates[0] attn + gates[1] sliding-attn + gates[2] coreset-attn."""
     g = np.asarray(gates, dtype=np.float64)
     o_full = attn_full(Q, K, V, scale, q_rows=q_rows)
-    o_sld = attn_sliding(grid, tile, window, Q, K, V, scale, q_rows=q_rows)
-    o_core, _, _ = attn_coreset(grid, bucket, ratio, Q, K, V, scale, q_rows=q_rows)
+    o_sld = attn_sliding(grid, tile, window, Q, K, V, scale, q_rows=q_rows, text=text)
+    o_core, _, _ = attn_coreset(grid, bucket, ratio, Q, K, V, scale, q_rows=q_rows, text=text)
     return g[0] * o_full + g[1] * o_sld + g[2] * o_core

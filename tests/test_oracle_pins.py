@@ -433,3 +433,91 @@ def test_merge_vs_explicit_numpy():
     assert np.abs(O - Oc[bs]).max() < 1e-12
     plain, _, _ = oracle.attn_coreset(grid, bucket, r, Q, K, V, 0.35)
     assert np.abs(O - plain).max() > 1e-3
+
+
+# --------------------------------------------------------------------------- joint sequences (video + text tokens)
+def joint_mask(grid, tile, window, text):
+    """[L + text, L + text] mask written out directly: the coordinate-range video mask, every
+    text column allowed, every text row allowed."""
+    Mv = brute_mask(grid, tile, window)
+    L = Mv.shape[0]
+    M = np.ones((L + text, L + text), dtype=bool)
+    M[:L, :L] = Mv
+    return M
+
+
+@pytest.mark.parametrize("grid,tile,window,text", [((10, 4, 6), (2, 2, 2), (3, 3, 3), 5),
+                                                   ((9, 5, 7), (2, 2, 3), (3, 1, 3), 1),
+                                                   ((4, 4, 12), (1, 2, 4), (3, 3, 1), 17)])
+def test_joint_sliding_attention_vs_explicit_mask(grid, tile, window, text):
+    L = grid[0] * grid[1] * grid[2]
+    Q, K, V = rand_qkv(L + text, 8, 21)
+    O, P = oracle.attn_sliding(grid, tile, window, Q, K, V, 0.4, return_probs=True, text=text)
+    M = joint_mask(grid, tile, window, text)
+    Ob, Pb = dense_attention(Q, K, V, 0.4, M)
+    assert np.abs(O - Ob).max() < 1e-12 and np.abs(P - Pb).max() < 1e-12
+    # every query gives every text key some weight; outside its window a video query gives none
+    assert (P[:, L:] > 0).all()
+    assert (P[:L, :L][~M[:L, :L]] == 0).all() and (~M[:L, :L]).any()
+    # a text query is a full-attention row
+    Of = oracle.attn_full(Q, K, V, 0.4, q_rows=np.arange(L, L + text))
+    assert np.abs(O[L:] - Of).max() < 1e-12
+    # no text tokens: the video-only function
+    O0 = oracle.attn_sliding(grid, tile, window, Q[:L], K[:L], V[:L], 0.4, text=0)
+    assert np.array_equal(O0, oracle.attn_sliding(grid, tile, window, Q[:L], K[:L], V[:L], 0.4))
+    # row subsets, text rows included
+    rows = [L + text - 1, 0, L, L - 1]
+    assert np.array_equal(oracle.attn_sliding(grid, tile, window, Q, K, V, 0.4, q_rows=rows, text=text), O[rows])
+
+
+def test_joint_window_covering_the_grid_is_full_attention_over_all_tokens():
+    grid, text = (3, 4, 5), 7
+    L = 60
+    Q, K, V = rand_qkv(L + text, 8, 22)
+    O = oracle.attn_sliding(grid, (1, 2, 2), (3, 3, 3), Q, K, V, 0.3, text=text)
+    assert np.abs(O - oracle.attn_full(Q, K, V, 0.3)).max() < 1e-12
+
+
+def test_joint_coreset_keeps_every_text_token_and_prunes_video_only():
+    grid, bucket, r, text = (4, 6, 6), (2, 3, 2), 0.5, 9
+    L, d = 144, 8
+    Q, K, V = rand_qkv(L + text, d, 23)
+    O, core, src = oracle.attn_coreset(grid, bucket, r, Q, K, V, 0.35, text=text)
+    # selection saw the video rows of K only
+    bc, bs = brute_select(grid, bucket, r, K[:L])
+    assert np.array_equal(core, bc) and np.array_equal(src, bs)
+    # explicit pool / attend / unpool: kept video tokens, then the text tokens
+    keep = np.concatenate([bc, np.arange(L, L + text)])
+    Oc, _ = dense_attention(Q[keep], K[keep], V[keep], 0.35)
+    assert np.abs(O[:L] - Oc[bs]).max() < 1e-12
+    assert np.abs(O[L:] - Oc[len(bc):]).max() < 1e-12
+    pruned = np.setdiff1d(np.arange(L), core)
+    assert np.array_equal(O[pruned], O[core[src[pruned]]])
+    # ratio 1: nothing pruned, so full attention over all tokens (a permutation of the keys)
+    O1, _, _ = oracle.attn_coreset(grid, bucket, 1.0, Q, K, V, 0.35, text=text)
+    assert np.abs(O1 - oracle.attn_full(Q, K, V, 0.35)).max() < 1e-12
+    # an X of its own, with or without rows for the text tokens
+    X = np.random.default_rng(24).standard_normal((L + text, 5))
+    Oa, ca, _ = oracle.attn_coreset(grid, bucket, r, Q, K, V, 0.35, X=X, text=text)
+    Ob, cb, _ = oracle.attn_coreset(grid, bucket, r, Q, K, V, 0.35, X=X[:L], text=text)
+    assert np.array_equal(ca, cb) and np.array_equal(Oa, Ob)
+    # merge averages video rows only: text rows of the compact sequences are untouched
+    Om, _, _ = oracle.attn_coreset(grid, bucket, r, Q, K, V, 0.35, text=text, merge=True)
+    Qm, Km, Vm = Q.copy(), K.copy(), V.copy()
+    for s_, c_ in enumerate(bc):
+        mem = [c_] + [i for i in pruned if bs[i] == s_]
+        for A, Am in ((Q, Qm), (K, Km), (V, Vm)):
+            Am[c_] = A[mem].mean(axis=0)
+    Ocm, _ = dense_attention(Qm[keep], Km[keep], Vm[keep], 0.35)
+    assert np.abs(Om[:L] - Ocm[bs]).max() < 1e-12 and np.abs(Om[L:] - Ocm[len(bc):]).max() < 1e-12
+
+
+def test_joint_soft_mixture_one_hot_gates_give_the_joint_branches():
+    grid, tile, window, bucket, r, text = (4, 6, 4), (2, 3, 2), (1, 1, 3), (2, 3, 2), 0.5, 3
+    Q, K, V = rand_qkv(96 + text, 8, 25)
+    want = [oracle.attn_full(Q, K, V, 0.3), oracle.attn_sliding(grid, tile, window, Q, K, V, 0.3, text=text),
+            oracle.attn_coreset(grid, bucket, r, Q, K, V, 0.3, text=text)[0]]
+    for b in range(3):
+        gates = np.eye(3)[b]
+        got = oracle.soft_mixture(grid, tile, window, bucket, r, Q, K, V, 0.3, gates, text=text)
+        assert np.abs(got - want[b]).max() < 1e-15
