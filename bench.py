@@ -59,7 +59,7 @@ def peaks():
 
 def get_workload(name):
     from paper_2505_18809_b200 import workloads
-    if name in workloads.CONFIG_NAMES or name in workloads.PROFILE_NAMES:
+    if name in workloads.CONFIG_NAMES or name in workloads.PROFILE_NAMES or name in workloads.JOINT_NAMES:
         return workloads.config(name)
     for w in workloads.route_mix_sweep():
         if w.name == name:
@@ -153,22 +153,26 @@ def time_oracle(wl, Q, K, V, rows_per_head: int, budget_s: float, seed: int = 0)
     Lc = oracle.coreset_len(wl.grid, wl.bucket, float(np.float32(wl.ratio)))
     g = np.random.default_rng(seed)
     flops, t_total, heads_done = 0.0, 0.0, 0
+    text = getattr(wl, "text", 0)
+    n_rows = wl.L + text
     for h in range(wl.heads):
         if t_total > budget_s:
             break
         q, k, v = (x[0, h].to("cpu", torch.float64).numpy() for x in (Q, K, V))
-        rows = np.sort(g.choice(wl.L, size=min(rows_per_head, wl.L), replace=False)).astype(np.int64)
+        rows = np.sort(g.choice(n_rows, size=min(rows_per_head, n_rows), replace=False)).astype(np.int64)
         t0 = time.perf_counter()
         if wl.routes[h] == 0:
             oracle.attn_full(q, k, v, scale, q_rows=rows)
-            f = 4.0 * wl.d * wl.L * len(rows)
+            f = 4.0 * wl.d * n_rows * len(rows)
         elif wl.routes[h] == 1:
-            oracle.attn_sliding(wl.grid, wl.tile, wl.window, q, k, v, scale, q_rows=rows)
-            f = 4.0 * wl.d * sum(_window_keys(wl, int(r)) for r in rows)
+            oracle.attn_sliding(wl.grid, wl.tile, wl.window, q, k, v, scale, q_rows=rows, text=text)
+            # a video query: its window and every text key; a text query: every key
+            f = 4.0 * wl.d * sum(_window_keys(wl, int(r)) + text if r < wl.L else n_rows for r in rows)
         else:
             _, _, src = oracle.attn_coreset(wl.grid, wl.bucket, float(np.float32(wl.ratio)), q, k, v, scale,
-                                            q_rows=rows)
-            f = 4.0 * wl.d * Lc * len(set(src[rows].tolist()))
+                                            q_rows=rows, text=text)
+            slots = set(src[rows[rows < wl.L]].tolist()) | set((Lc + (rows[rows >= wl.L] - wl.L)).tolist())
+            f = 4.0 * wl.d * (Lc + text) * len(slots)
         t_total += time.perf_counter() - t0
         flops += f
         heads_done += 1
@@ -362,7 +366,7 @@ def run_ours(args):
                "dtype": "bf16",
                "data": "synthetic",
                "config": {"workload": wl.name + ("+soft-mixture" if args.mixture else ""), "grid": list(wl.grid),
-                          "tokens": wl.L, "heads": wl.heads,
+                          "tokens": wl.L, "text_tokens": getattr(wl, "text", 0), "heads": wl.heads,
                           "d": wl.d, "tile": list(wl.tile), "window_tiles": list(wl.window),
                           "coreset_ratio": wl.ratio, "routes": list(wl.routes),
                           "heads_full_sliding_coreset": [info.n_full, info.n_sliding, info.n_coreset],

@@ -10,7 +10,9 @@
  *
  * Conventions shared by all entry points
  *   - Tokens are 0-based and frame-major: i = (t*H + h)*W + w, L = T*H*W.
- *   - Q, K, V, O are bf16, contiguous [B, heads, L, d]; d is 64 or 128.
+ *   - Q, K, V, O are bf16, contiguous [B, heads, L, d]; d is 64 or 128.  With text tokens
+ *     (vorta_plan_desc.text_tokens > 0) every "L" row count of a tensor argument below is
+ *     L + text_tokens: the video tokens of a head, then its text tokens.
  *   - "dev" pointers are CUDA device memory, "host" pointers ordinary host
  *     memory.  The caller owns every buffer it passes and the stream; the library
  *     owns the plan and the small device tables inside it.
@@ -84,10 +86,16 @@ typedef struct {
     const uint8_t *routes;/* host, [heads]: branch of each head (same for every batch entry) */
     int32_t flags;        /* bit set of VORTA_PLAN_* */
     int32_t device;       /* CUDA device ordinal; -1 = the calling thread's current device */
+    int32_t text_tokens;  /* joint sequence of an MMDiT model: this many text tokens follow the T*H*W video
+                             tokens in every head of Q, K, V, O (and X); 0 = video tokens only.  A text key
+                             is visible to every query of every branch, a text query sees every key, and
+                             core-set selection prunes video tokens only (every text token is kept).  The
+                             paper runs HunyuanVideo (Section 4) without saying how its branches treat the
+                             text tokens: this is this library's reading. */
 } vorta_plan_desc;
 
 typedef struct {
-    int64_t L;                   /* tokens per head */
+    int64_t L;                   /* video tokens per head (T*H*W); rows per head = L + text_tokens */
     int64_t Lc;                  /* core-set tokens per head (geometry only, data independent) */
     int32_t tiles_per_axis[3];   /* ceil(dim / tile) */
     int32_t n_tiles;
@@ -99,17 +107,19 @@ typedef struct {
     int64_t host_call_scratch_bytes; /* device scratch vorta_routed_attention_host needs */
     int64_t mixture_workspace_bytes; /* device workspace vorta_soft_mixture needs */
     /* Algorithmic work: 4*d*(query, key) pairs the method itself attends, per (batch, head). */
-    double flops_full_head;      /* 4 d L^2 */
-    double flops_sliding_head;   /* 4 d * sum over tile pairs in the window of valid tokens products */
-    double flops_coreset_head;   /* 4 d Lc^2 */
+    double flops_full_head;      /* 4 d (L + Lt)^2, Lt = text_tokens */
+    double flops_sliding_head;   /* 4 d * (sum over tile pairs in the window of valid tokens products
+                                    + L Lt [video queries x text keys] + Lt (L + Lt) [text queries]) */
+    double flops_coreset_head;   /* 4 d (Lc + Lt)^2 */
     double flops_layer;          /* B * sum over heads, current routes */
     double flops_issued_layer;   /* what the tensor cores are really given (padding to 128-row blocks
                                     and partial tiles included); 0 for a host-only plan */
     int64_t n_work_items;        /* (head, query block) items in one launch; 0 for a host-only plan */
     /* Algorithmic bytes of the memory-bound stages, per core-set (batch, head). */
     int64_t select_bytes_head;   /* L*dx*2 read + (Lc + L)*4 written, with dx = d */
-    int64_t gather_bytes_head;   /* 3 * Lc*d*2 read and written */
-    int64_t scatter_bytes_head;  /* Lc*d*2 read + L*d*2 written */
+    int64_t gather_bytes_head;   /* 3 * (Lc + Lt)*d*2 read and written */
+    int64_t scatter_bytes_head;  /* (Lc + Lt)*d*2 read + (L + Lt)*d*2 written */
+    int64_t text_tokens;         /* Lt of the plan (0 = video tokens only) */
 } vorta_plan_info_t;
 
 /*
@@ -183,8 +193,9 @@ VORTA_API int vorta_coreset_select(const vorta_plan *plan, const void *X_dev, in
  * [B, Hx, L, d] with Hx == 1, shared by all heads, or Hx == heads), gather the
  * kept rows of Q, K, V, attend, scatter back (Section 3.2, last paragraph).
  * Sliding heads: Algorithm 1's mask, only the listed tile pairs are computed.
- *   Q, K, V      device bf16 [B, heads, L, d], 16-byte aligned
- *   O            device bf16 [B, heads, L, d] out; every element is written
+ *   Q, K, V      device bf16 [B, heads, L + text_tokens, d], 16-byte aligned (per head: the
+ *                L = T*H*W video tokens, then the text tokens)
+ *   O            same shape, out; every element is written
  *   workspace    device, >= vorta_plan_info().workspace_bytes, 256-byte aligned
  *                (may be NULL when no head is routed to core-set); contents are
  *                scratch and undefined afterwards

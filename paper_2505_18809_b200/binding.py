@@ -41,7 +41,7 @@ class vorta_plan_desc(ctypes.Structure):
                 ("tile", ctypes.c_int32 * 3), ("window", ctypes.c_int32 * 3),
                 ("bucket", ctypes.c_int32 * 3), ("coreset_ratio", ctypes.c_float),
                 ("softmax_scale", ctypes.c_float), ("routes", ctypes.POINTER(ctypes.c_uint8)),
-                ("flags", ctypes.c_int32), ("device", ctypes.c_int32)]
+                ("flags", ctypes.c_int32), ("device", ctypes.c_int32), ("text_tokens", ctypes.c_int32)]
 
 
 class vorta_plan_info_t(ctypes.Structure):
@@ -57,7 +57,7 @@ class vorta_plan_info_t(ctypes.Structure):
                 ("flops_coreset_head", ctypes.c_double), ("flops_layer", ctypes.c_double),
                 ("flops_issued_layer", ctypes.c_double), ("n_work_items", ctypes.c_int64),
                 ("select_bytes_head", ctypes.c_int64), ("gather_bytes_head", ctypes.c_int64),
-                ("scatter_bytes_head", ctypes.c_int64)]
+                ("scatter_bytes_head", ctypes.c_int64), ("text_tokens", ctypes.c_int64)]
 
 
 _lib: Optional[ctypes.CDLL] = None
@@ -236,7 +236,7 @@ def vorta_device_status(plan: int, stream: int = 0) -> int:
 
 
 def make_desc(B, heads, grid, d, tile, window, ratio, routes, bucket=(0, 0, 0), scale=0.0,
-              flags=0, device=-1):
+              flags=0, device=-1, text=0):
     """Fill a vorta_plan_desc; keeps the routes array alive on the returned object."""
     desc = vorta_plan_desc()
     desc.B, desc.heads = int(B), int(heads)
@@ -251,6 +251,7 @@ def make_desc(B, heads, grid, d, tile, window, ratio, routes, bucket=(0, 0, 0), 
     desc._routes_keepalive = arr
     desc.routes = ctypes.cast(arr, ctypes.POINTER(ctypes.c_uint8))
     desc.flags, desc.device = int(flags), int(device)
+    desc.text_tokens = int(text)
     return desc
 
 
@@ -259,9 +260,9 @@ class Plan:
     """Owns one vorta_plan; methods take torch CUDA tensors and pass their pointers on."""
 
     def __init__(self, B, heads, grid, d, tile, window, ratio, routes, bucket=(0, 0, 0),
-                 scale=0.0, host_only=False, device=-1, merge=False):
+                 scale=0.0, host_only=False, device=-1, merge=False, text=0):
         flags = (VORTA_PLAN_HOST_ONLY if host_only else 0) | (VORTA_PLAN_POOL_MERGE if merge else 0)
-        self.desc = make_desc(B, heads, grid, d, tile, window, ratio, routes, bucket, scale, flags, device)
+        self.desc = make_desc(B, heads, grid, d, tile, window, ratio, routes, bucket, scale, flags, device, text)
         self.handle = vorta_plan_create(self.desc)
         self.B, self.heads, self.grid, self.d = B, heads, tuple(grid), d
         self._workspace = None
@@ -269,7 +270,7 @@ class Plan:
     @classmethod
     def from_workload(cls, wl, host_only=False, device=-1):
         return cls(wl.B, wl.heads, wl.grid, wl.d, wl.tile, wl.window, wl.ratio, wl.routes,
-                   wl.bucket, 0.0, host_only, device, getattr(wl, "merge", False))
+                   wl.bucket, 0.0, host_only, device, getattr(wl, "merge", False), getattr(wl, "text", 0))
 
     def close(self):
         if getattr(self, "handle", None):
@@ -314,14 +315,15 @@ class Plan:
         return int(torch.cuda.current_stream().cuda_stream)
 
     def coreset_select(self, X):
-        """X: bf16 CUDA [B, Hx, L, dx] -> (core_idx int32 [B, Hx, Lc], src_slot int32 [B, Hx, L])."""
+        """X: bf16 CUDA [B, Hx, L + text, dx] -> (core_idx int32 [B, Hx, Lc], src_slot int32 [B, Hx, L]);
+        only the L video rows of X are looked at."""
         import torch
         assert X.is_cuda and X.dtype == torch.bfloat16 and X.is_contiguous()
-        B, Hx, L, dx = X.shape
+        B, Hx, rows, dx = X.shape
         info = self.info
-        assert B == self.B and L == info.L
+        assert B == self.B and rows == info.L + info.text_tokens
         core_idx = torch.empty((B, Hx, info.Lc), dtype=torch.int32, device=X.device)
-        src_slot = torch.empty((B, Hx, L), dtype=torch.int32, device=X.device)
+        src_slot = torch.empty((B, Hx, info.L), dtype=torch.int32, device=X.device)
         vorta_coreset_select(self.handle, X.data_ptr(), Hx, dx, core_idx.data_ptr(),
                              src_slot.data_ptr(), self._stream())
         return core_idx, src_slot
@@ -337,11 +339,12 @@ class Plan:
         return self._workspace
 
     def routed_attention(self, Q, K, V, O=None, X=None, workspace=None):
-        """Q, K, V: bf16 CUDA [B, heads, L, d] -> O (same shape)."""
+        """Q, K, V: bf16 CUDA [B, heads, L + text, d] -> O (same shape)."""
         import torch
+        info = self.info
         for t in (Q, K, V):
             assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
-            assert tuple(t.shape) == (self.B, self.heads, self.info.L, self.d)
+            assert tuple(t.shape) == (self.B, self.heads, info.L + info.text_tokens, self.d)
         if O is None:
             O = torch.empty_like(Q)
         ws = workspace if workspace is not None else self.workspace(Q.device)

@@ -23,7 +23,7 @@ attention_simt_kernel(AttnParams p)
     const bool compact = w.mode == MODE_COMPACT;
     const __nv_bfloat16 *Q = compact ? p.Qc : p.Q, *K = compact ? p.Kc : p.K, *V = compact ? p.Vc : p.V;
     __nv_bfloat16 *O = compact ? p.Oc : p.O;
-    const int64_t rows = compact ? g.Lc : g.L;
+    const int64_t rows = compact ? g.Lct : g.Ltot;
     const int64_t base = (int64_t)w.slice * rows * D;
     const float scale = p.scale_log2 * 0.6931471805599453f;
 
@@ -44,7 +44,14 @@ attention_simt_kernel(AttnParams p)
     for (int32_t j = 0; j < w.kv_count; ++j) {
         int32_t org[3];
         uint32_t mask[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
-        if (w.mode == MODE_TILES) {
+        // the last kv_text blocks of a sliding item are runs of bn_tile text tokens (rows L + ...)
+        const bool text = w.mode == MODE_TILES && j >= w.kv_count - w.kv_text;
+        int32_t kv_mode = w.mode, kv_len = w.kv_len;
+        if (text) {
+            kv_mode = MODE_LINEAR;
+            kv_len = g.Ltot;
+            org[0] = g.L + (j - (w.kv_count - w.kv_text)) * g.bn_tile; org[1] = 0; org[2] = 0;
+        } else if (w.mode == MODE_TILES) {
             KvEntry e = p.kv_list[w.kv_begin + j];
             org[0] = e.w0; org[1] = e.h0; org[2] = e.t0;
             if (e.mask_id)
@@ -57,7 +64,7 @@ attention_simt_kernel(AttnParams p)
             if (threadIdx.x < kKvChunk) {
                 int32_t n = c0 + threadIdx.x, tok = -1, t;
                 if (n < bn && ((mask[n >> 5] >> (n & 31)) & 1u) &&
-                    block_row_token(g, w.mode, org, w.kv_len, n, &t))
+                    block_row_token(g, kv_mode, org, kv_len, n, &t))
                     tok = t;
                 sTok[threadIdx.x] = tok;
             }

@@ -268,11 +268,16 @@ __device__ __forceinline__ float max3(float a, float b, float c)
     return r;
 }
 
-// Coordinates of block `j` of the item's KV sequence and its column-mask class.
+// Coordinates of block `j` of the item's KV sequence and its column-mask class.  text: the
+// block is a run of bn_tile text tokens (the last kv_text blocks of a sliding item), fetched
+// through the text-row tensor maps.
 __device__ __forceinline__ void kv_block_coords(const AttnParams &p, const WorkItem &w, int32_t j, int32_t &c1,
-                                                int32_t &c2, int32_t &c3, uint32_t &mask_id)
+                                                int32_t &c2, int32_t &c3, uint32_t &mask_id, bool &text)
 {
-    if (w.mode == MODE_TILES) {
+    text = w.mode == MODE_TILES && j >= w.kv_count - w.kv_text;
+    if (text) {
+        c1 = (j - (w.kv_count - w.kv_text)) * p.g.bn_tile; c2 = 0; c3 = 0; mask_id = 0;
+    } else if (w.mode == MODE_TILES) {
         const KvEntry e = p.kv_list[w.kv_begin + j];
         c1 = e.w0; c2 = e.h0; c3 = e.t0; mask_id = e.mask_id;
     } else {
@@ -370,15 +375,18 @@ __device__ __forceinline__ void producer_role(const AttnParams &p, const AttnMap
         for (int32_t j = 0; j < w.kv_count; ++j) {
             int32_t c1, c2, c3;
             uint32_t mask_id;
-            kv_block_coords(p, w, j, c1, c2, c3, mask_id);
+            bool text;
+            kv_block_coords(p, w, j, c1, c2, c3, mask_id, text);
+            const uint32_t kv_bytes = (text ? (uint32_t)p.g.bn_tile * 128u : half_bytes) * kHalves;
 #pragma unroll
             for (int kv = 0; kv < 2; ++kv) {
                 const uint32_t slot = kv_it % kStages;
                 if (!mbar_wait(bars + 8 * (BAR_KV_EMPTY + slot), ((kv_it / kStages) & 1) ^ 1, ctl, p.status, 102)) return;
                 if (lane == 0) {
                     const uint32_t full = bars + 8 * (BAR_KV_FULL + slot);
-                    mbar_expect_tx(full, half_bytes * kHalves);
-                    const CUtensorMap *map = kv == 0 ? &maps.k[w.mode] : &maps.v[w.mode];
+                    mbar_expect_tx(full, kv_bytes);
+                    const CUtensorMap *map = text ? (kv == 0 ? &maps.kt : &maps.vt)
+                                                  : (kv == 0 ? &maps.k[w.mode] : &maps.v[w.mode]);
                     for (int h = 0; h < kHalves; ++h)
                         tma_load_5d(smem_base + kSmemKV + slot * kTileBytes + h * kHalfBytes, map, full, h * 64, c1,
                                     c2, c3, w.slice);
@@ -510,6 +518,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
         if (m >= wp->n_mblk) continue;
         const int32_t w_mode = wp->mode, w_kv_len = wp->kv_len, w_kv_count = wp->kv_count;
         const KvEntry *kv_entries = p.kv_list + wp->kv_begin;
+        const int32_t n_boxes = w_mode == MODE_TILES ? w_kv_count - wp->kv_text : w_kv_count;  // the rest: text-token blocks
         const int32_t bn = w_mode == MODE_TILES ? p.g.bn_tile : kBlockM;
         const int32_t sh = bn > 64 ? 1 : 0;  // log2 of the sub-blocks per KV block
         const int32_t n_sub = w_kv_count << sh;
@@ -542,12 +551,21 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
             return true;
         };
         // strike the columns of sub-block u that are not keys (mask class `id` of its block,
-        // fetched ahead by the caller)
+        // fetched ahead by the caller; blocks of text tokens have none: their last one is cut at Lt)
         auto apply_mask = [&](int32_t u, uint32_t id, uint32_t(&s)[64]) {
             const int32_t h = u & sh;
             uint32_t m0 = 0, m1 = 0;
             bool partial = false;
-            if (id) {
+            if ((u >> sh) >= n_boxes) {
+                // text keys of this sub-block: what is left of Lt, at most the block's bn columns
+                const int32_t valid = min(p.g.Lt - ((u >> sh) - n_boxes) * bn, bn) - 64 * h;
+                if (valid < 64) {
+                    const int32_t v0 = min(max(valid, 0), 32), v1 = min(max(valid - 32, 0), 32);
+                    m0 = v0 == 32 ? 0xffffffffu : ((1u << v0) - 1u);
+                    m1 = v1 == 32 ? 0xffffffffu : ((1u << v1) - 1u);
+                    partial = true;
+                }
+            } else if (id) {
                 m0 = ctl->colmasks[id * 4 + 2 * h];
                 m1 = ctl->colmasks[id * 4 + 2 * h + 1];
                 partial = true;
@@ -571,7 +589,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
             const bool has_next = kFull || u + 1 < n_sub;
             // mask class of the next sub-block's KV block, in flight under the exponentials
             const uint32_t next_id =
-                (!kFull && has_next && w_mode == MODE_TILES) ? kv_entries[(u + 1) >> sh].mask_id : 0u;
+                (!kFull && has_next && w_mode == MODE_TILES && ((u + 1) >> sh) < n_boxes) ? kv_entries[(u + 1) >> sh].mask_id : 0u;
             if (row == 0) TRACE(2 + m, u, 0);
             // P = exp2(S * scale - max) as packed bf16 over the first half of the buffer
             float2 sum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
@@ -607,7 +625,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
 
         uint32_t s[64];
         if (!load_sub(std::false_type{}, 0, s)) return;
-        apply_mask(0, w_mode == MODE_TILES ? kv_entries[0].mask_id : 0u, s);
+        apply_mask(0, (w_mode == MODE_TILES && n_boxes > 0) ? kv_entries[0].mask_id : 0u, s);
         row_max = row_max64(s) * scale;
         // the leading unmasked blocks, then whatever is cut, short or last
         const int32_t n_full = min(2 * wp->kv_fast, n_sub) - 1;  // steps whose u and u+1 are both whole
@@ -627,7 +645,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
         int32_t token = 0;
         const int32_t q_org[3] = {wp->q_org[m][0], wp->q_org[m][1], wp->q_org[m][2]};
         const bool valid = block_row_token(p.g, w_mode, q_org, w_kv_len, row, &token);
-        const int64_t rows = w_mode == MODE_COMPACT ? p.g.Lc : p.g.L;
+        const int64_t rows = w_mode == MODE_COMPACT ? p.g.Lct : p.g.Ltot;
         __nv_bfloat16 *out = (w_mode == MODE_COMPACT ? p.Oc + (int64_t)wp->slice * rows * D : p.O + (int64_t)wp->out_slice * rows * D) +
                              (int64_t)token * D;
         const float inv = 1.f / row_sum;

@@ -90,15 +90,17 @@ EncodeTiledFn encode_fn()
 
 // 5-D bf16 map (d, n1, n2, n3, slices) over a contiguous [slices, n3, n2, n1, d]
 // tensor with a (64, b1, b2, b3, 1) box and the 128-byte swizzle.
+// slice_rows: rows of d elements between consecutive slices (>= n1*n2*n3; the map may cover only the
+// leading or, with an offset base, the trailing rows of a slice).
 bool make_map(CUtensorMap *m, const void *base, int32_t d, int64_t n1, int64_t n2, int64_t n3,
-              int64_t slices, int32_t b1, int32_t b2, int32_t b3)
+              int64_t slices, int32_t b1, int32_t b2, int32_t b3, int64_t slice_rows = 0)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[5] = {(cuuint64_t)d, (cuuint64_t)n1, (cuuint64_t)n2, (cuuint64_t)n3,
                           (cuuint64_t)slices};
     cuuint64_t row = (cuuint64_t)d * 2;
-    cuuint64_t strides[4] = {row, row * n1, row * n1 * n2, row * n1 * n2 * n3};
+    cuuint64_t strides[4] = {row, row * n1, row * n1 * n2, row * (slice_rows ? slice_rows : n1 * n2 * n3)};
     cuuint32_t box[5] = {64, (cuuint32_t)b1, (cuuint32_t)b2, (cuuint32_t)b3, 1};
     cuuint32_t estr[5] = {1, 1, 1, 1, 1};
     CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(base), dims, strides,
@@ -125,7 +127,7 @@ Workspace workspace_layout(const Geometry &g, int64_t n_prob)
     int64_t off = 0;
     w.core_idx = off; off = align_up(off + n_prob * g.Lc * 4, 256);
     w.src_slot = off; off = align_up(off + n_prob * g.L * 4, 256);
-    int64_t rows = align_up(n_prob * (int64_t)g.Lc * g.d * 2, 256);
+    int64_t rows = align_up(n_prob * (int64_t)g.Lct * g.d * 2, 256);
     w.Qc = off; off += rows;
     w.Kc = off; off += rows;
     w.Vc = off; off += rows;
@@ -134,7 +136,7 @@ Workspace workspace_layout(const Geometry &g, int64_t n_prob)
     return w;
 }
 
-int64_t tensor_bytes(const Geometry &g) { return (int64_t)g.B * g.heads * g.L * g.d * 2; }
+int64_t tensor_bytes(const Geometry &g) { return (int64_t)g.B * g.heads * g.Ltot * g.d * 2; }
 
 // Bytes of the three branch outputs and of the all-heads core-set scratch of a mixture call.
 int64_t mixture_workspace_bytes(const Geometry &g)
@@ -210,15 +212,16 @@ int build_list(vorta_plan *p, vorta_plan::WorkList &wl, const std::vector<uint8_
     const int32_t BH = g.B * g.heads;
     std::vector<WorkItem> items;
     std::vector<double> cost;
-    auto linear_items = [&](int32_t mode, int32_t slice, int32_t out_slice, int32_t len) {
-        int32_t nblk = (len + kBlockM - 1) / kBlockM;
-        int32_t kv = nblk;
+    // query rows [q0, q1) of a sequence of `len` keys, two 128-row blocks per item
+    auto linear_items = [&](int32_t mode, int32_t slice, int32_t out_slice, int32_t len, int32_t q0, int32_t q1) {
+        int32_t nblk = (q1 - q0 + kBlockM - 1) / kBlockM;
+        int32_t kv = (len + kBlockM - 1) / kBlockM;
         for (int32_t b0 = 0; b0 < nblk; b0 += 2) {
             WorkItem w{};
             w.mode = mode; w.slice = slice; w.out_slice = out_slice; w.kv_count = kv; w.kv_len = len;
             w.kv_fast = len % kBlockM ? kv - 1 : kv;
             w.n_mblk = std::min(2, nblk - b0);
-            for (int m = 0; m < w.n_mblk; ++m) w.q_org[m][0] = (b0 + m) * kBlockM;
+            for (int m = 0; m < w.n_mblk; ++m) w.q_org[m][0] = q0 + (b0 + m) * kBlockM;
             items.push_back(w);
             cost.push_back((double)w.n_mblk * kv + 2.0);
         }
@@ -227,14 +230,16 @@ int build_list(vorta_plan *p, vorta_plan::WorkList &wl, const std::vector<uint8_
         for (int32_t h = 0; h < g.heads; ++h) {
             const int32_t slice = b * g.heads + h;
             if (branches[h] & (1u << VORTA_ROUTE_FULL))
-                linear_items(MODE_LINEAR, slice, by_branch ? VORTA_ROUTE_FULL * BH + slice : slice, g.L);
+                linear_items(MODE_LINEAR, slice, by_branch ? VORTA_ROUTE_FULL * BH + slice : slice, g.Ltot, 0, g.Ltot);
             if (branches[h] & (1u << VORTA_ROUTE_SLIDING)) {
                 for (int32_t qt = 0; qt < g.n_tiles; ++qt) {
                     int32_t q[3] = {qt / (g.nt[2] * g.nt[1]), (qt / g.nt[2]) % g.nt[1], qt % g.nt[2]};
                     WorkItem w{};
                     w.mode = MODE_TILES; w.slice = slice;
                     w.out_slice = by_branch ? VORTA_ROUTE_SLIDING * BH + slice : slice;
-                    w.kv_count = p->kv_count[qt];
+                    // the boxes of the window, then every text key in blocks of bn_tile
+                    w.kv_text = g.text_blocks;
+                    w.kv_count = p->kv_count[qt] + w.kv_text;
                     w.kv_fast = g.bn_tile == kBlockM ? p->kv_count[g.n_tiles + qt] : 0;
                     w.kv_begin = qt * g.max_kv_per_tile;
                     w.kv_len = 0;
@@ -249,10 +254,14 @@ int build_list(vorta_plan *p, vorta_plan::WorkList &wl, const std::vector<uint8_
                     items.push_back(w);
                     cost.push_back((double)w.n_mblk * w.kv_count * g.bn_tile / 128.0 + 2.0);
                 }
+                // the text queries of a sliding head see every key: linear items over rows [L, L + Lt)
+                if (g.Lt > 0)
+                    linear_items(MODE_LINEAR, slice, by_branch ? VORTA_ROUTE_SLIDING * BH + slice : slice, g.Ltot,
+                                 g.L, g.Ltot);
             }
             if (branches[h] & (1u << VORTA_ROUTE_CORESET)) {
                 int32_t k = (int32_t)(std::find(core_heads.begin(), core_heads.end(), h) - core_heads.begin());
-                linear_items(MODE_COMPACT, b * n_core + k, 0, g.Lc);
+                linear_items(MODE_COMPACT, b * n_core + k, 0, g.Lct, 0, g.Lct);
             }
         }
     }
@@ -323,8 +332,9 @@ int build_host_chunks(vorta_plan *p)
     std::vector<double> cost(g.heads);
     for (int32_t h = 0; h < g.heads; ++h) {
         const uint8_t r = p->routes[h];
-        cost[h] = r == VORTA_ROUTE_FULL ? (double)g.L * g.L
-                  : r == VORTA_ROUTE_SLIDING ? p->sliding_pairs : (double)g.Lc * g.Lc;
+        cost[h] = r == VORTA_ROUTE_FULL ? (double)g.Ltot * g.Ltot
+                  : r == VORTA_ROUTE_SLIDING ? p->sliding_pairs + (double)g.L * g.Lt + (double)g.Lt * g.Ltot
+                                             : (double)g.Lct * g.Lct;
     }
     std::vector<int32_t> order(g.heads);
     for (int32_t h = 0; h < g.heads; ++h) order[h] = h;
@@ -447,7 +457,7 @@ int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
     if (!D.routes || D.B < 1 || D.heads < 1 || D.T < 1 || D.H < 1 || D.W < 1) return VORTA_ERR_INVALID_ARG;
     if (D.T > 32767 || D.H > 32767 || D.W > 32767) return VORTA_ERR_INVALID_ARG;
     int64_t L64 = (int64_t)D.T * D.H * D.W;
-    if (L64 >= (int64_t)1 << 31) return VORTA_ERR_INVALID_ARG;
+    if (D.text_tokens < 0 || L64 + D.text_tokens >= (int64_t)1 << 31) return VORTA_ERR_INVALID_ARG;
     if ((int64_t)D.B * D.heads > 65535) return VORTA_ERR_INVALID_ARG;
     if (!(D.coreset_ratio > 0.f) || !(D.coreset_ratio <= 1.f)) return VORTA_ERR_INVALID_ARG;
     if (!(D.softmax_scale >= 0.f) || !std::isfinite(D.softmax_scale)) return VORTA_ERR_INVALID_ARG;
@@ -497,6 +507,9 @@ int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
         Lc += keep_count(n, g.ratio);
     }
     g.Lc = (int32_t)Lc;
+    g.Lt = D.text_tokens;
+    g.Ltot = g.L + g.Lt;
+    g.Lct = g.Lc + g.Lt;
 
     // sliding branch blocking
     g.boxes_per_tile = tile_tokens > 128 ? 2 : 1;
@@ -506,6 +519,7 @@ int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
     int32_t kv_tiles = 1;
     for (int a = 0; a < 3; ++a) kv_tiles *= std::min(g.nt[a], 2 * g.half[a] + 1);
     g.max_kv_per_tile = kv_tiles * g.boxes_per_tile;
+    g.text_blocks = (g.Lt + g.bn_tile - 1) / g.bn_tile;
     p->sliding_pairs = sliding_valid_pairs(g);
 
     if (p->host_only) {
@@ -639,16 +653,17 @@ int vorta_plan_info(const vorta_plan *p, vorta_plan_info_t *o)
     o->workspace_bytes_max = workspace_layout(g, (int64_t)g.B * g.heads).total;
     o->host_call_scratch_bytes = 4 * align_up(tensor_bytes(g), 256) + o->workspace_bytes;
     o->mixture_workspace_bytes = mixture_workspace_bytes(g);
-    o->flops_full_head = 4.0 * g.d * (double)g.L * (double)g.L;
-    o->flops_sliding_head = 4.0 * g.d * p->sliding_pairs;
-    o->flops_coreset_head = 4.0 * g.d * (double)g.Lc * (double)g.Lc;
+    o->text_tokens = g.Lt;
+    o->flops_full_head = 4.0 * g.d * (double)g.Ltot * (double)g.Ltot;
+    o->flops_sliding_head = 4.0 * g.d * (p->sliding_pairs + (double)g.L * g.Lt + (double)g.Lt * g.Ltot);
+    o->flops_coreset_head = 4.0 * g.d * (double)g.Lct * (double)g.Lct;
     o->flops_layer = g.B * (o->n_full * o->flops_full_head + o->n_sliding * o->flops_sliding_head +
                             o->n_coreset * o->flops_coreset_head);
     o->flops_issued_layer = p->host_only ? 0.0 : p->routed.flops_issued;
     o->n_work_items = p->host_only ? 0 : p->routed.n_items;
     o->select_bytes_head = (int64_t)g.L * g.d * 2 + ((int64_t)g.Lc + g.L) * 4;
-    o->gather_bytes_head = 3 * 2 * (int64_t)g.Lc * g.d * 2;
-    o->scatter_bytes_head = ((int64_t)g.Lc + g.L) * g.d * 2;
+    o->gather_bytes_head = 3 * 2 * (int64_t)g.Lct * g.d * 2;
+    o->scatter_bytes_head = ((int64_t)g.Lct + g.Ltot) * g.d * 2;
     return VORTA_OK;
 }
 
@@ -794,12 +809,23 @@ static int run_layer(const vorta_plan *p, const vorta_plan::WorkList &wl, int32_
         const void *src[3] = {q, k, v};
         CUtensorMap *dst[3] = {maps.q, maps.k, maps.v};
         for (int t = 0; t < 3 && ok; ++t) {
-            ok = ok && make_map(&dst[t][MODE_LINEAR], src[t], g.d, g.L, 1, 1, BH, kBlockM, 1, 1);
-            ok = ok && make_map(&dst[t][MODE_TILES], src[t], g.d, g.W, g.H, g.T, BH, g.box[2], g.box[1], g.box[0]);
+            ok = ok && make_map(&dst[t][MODE_LINEAR], src[t], g.d, g.Ltot, 1, 1, BH, kBlockM, 1, 1);
+            // the video rows of a head as a T x H x W grid; heads are L + Lt rows apart
+            ok = ok && make_map(&dst[t][MODE_TILES], src[t], g.d, g.W, g.H, g.T, BH, g.box[2], g.box[1], g.box[0],
+                                g.Ltot);
+        }
+        if (g.Lt > 0) {
+            // the text rows of K and V: Lt rows starting L rows into every head, in boxes of bn_tile rows
+            const __nv_bfloat16 *kt = k + (int64_t)g.L * g.d, *vt = v + (int64_t)g.L * g.d;
+            ok = ok && make_map(&maps.kt, kt, g.d, g.Lt, 1, 1, BH, g.bn_tile, 1, 1, g.Ltot);
+            ok = ok && make_map(&maps.vt, vt, g.d, g.Lt, 1, 1, BH, g.bn_tile, 1, 1, g.Ltot);
+        } else {
+            maps.kt = maps.k[MODE_LINEAR];
+            maps.vt = maps.v[MODE_LINEAR];
         }
         const void *csrc[3] = {Qc, Kc, Vc};
         for (int t = 0; t < 3 && ok; ++t) {
-            if (n_prob) ok = ok && make_map(&dst[t][MODE_COMPACT], csrc[t], g.d, g.Lc, 1, 1, n_prob, kBlockM, 1, 1);
+            if (n_prob) ok = ok && make_map(&dst[t][MODE_COMPACT], csrc[t], g.d, g.Lct, 1, 1, n_prob, kBlockM, 1, 1);
             else dst[t][MODE_COMPACT] = dst[t][MODE_LINEAR];
         }
         if (!ok) return VORTA_ERR_CUDA;
@@ -938,7 +964,7 @@ int vorta_routed_attention_host(const vorta_plan *p, const void *Qh, const void 
     const char *hq = static_cast<const char *>(Qh), *hk = static_cast<const char *>(Kh),
                *hv = static_cast<const char *>(Vh);
     char *ho = static_cast<char *>(Oh);
-    const int64_t hb = (int64_t)g.L * g.d * (int64_t)sizeof(__nv_bfloat16);  // one head of one tensor
+    const int64_t hb = (int64_t)g.Ltot * g.d * (int64_t)sizeof(__nv_bfloat16);  // one head of one tensor
 
     // Three queues: copies in (own stream), kernels (the caller's stream), copies out (own
     // stream).  Group c's kernels wait for its copies in; its copy out waits for its kernels.

@@ -134,7 +134,7 @@ coreset_select_kernel(Geometry g, const __nv_bfloat16 *__restrict__ X, int32_t d
     const int32_t p = (int32_t)(warp / g.n_buckets);
     const int32_t bkt = (int32_t)(warp % g.n_buckets);
     const int32_t slice = prob_slice ? prob_slice[p] : p;
-    const __nv_bfloat16 *Xs = X + (int64_t)slice * g.L * dx;
+    const __nv_bfloat16 *Xs = X + (int64_t)slice * g.Ltot * dx;  // video rows of the slice
 
     // the bucket: id, extents cut by the grid, token count, centre
     int32_t id[3] = {bkt / (g.nb[2] * g.nb[1]), (bkt / g.nb[2]) % g.nb[1], bkt % g.nb[2]};
@@ -247,7 +247,7 @@ coreset_select_d128_kernel(Geometry g, const __nv_bfloat16 *__restrict__ X, cons
     if (bkt >= g.n_buckets) return;
     const int32_t p = blockIdx.y;
     const int32_t slice = prob_slice ? prob_slice[p] : p;
-    const __nv_bfloat16 *Xs = X + (int64_t)slice * g.L * dx;
+    const __nv_bfloat16 *Xs = X + (int64_t)slice * g.Ltot * dx;  // video rows of the slice
 
     const int32_t bt = bkt / (g.nb[2] * g.nb[1]), bhw = bkt - bt * (g.nb[2] * g.nb[1]);
     const int32_t bh = bhw / g.nb[2], bw = bhw - bh * g.nb[2];
@@ -424,17 +424,19 @@ gather_rows_kernel(Geometry g, int32_t n_prob, const int32_t *__restrict__ prob_
                    uint4 *__restrict__ Kc, uint4 *__restrict__ Vc)
 {
     const int32_t cpr = g.d >> 3;  // 16-byte chunks per row
-    const int64_t total = (int64_t)n_prob * g.Lc * cpr;
+    // compact row r of a problem: kept video token core_idx[r] for r < Lc, text token r - Lc after that
+    const int64_t total = (int64_t)n_prob * g.Lct * cpr;
     const uint4 *src = blockIdx.y == 0 ? Q : (blockIdx.y == 1 ? K : V);
     uint4 *dst = blockIdx.y == 0 ? Qc : (blockIdx.y == 1 ? Kc : Vc);
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
          i += (int64_t)gridDim.x * blockDim.x) {
         int64_t row = i / cpr;
         int32_t c = (int32_t)(i % cpr);
-        int32_t p = (int32_t)(row / g.Lc);
-        int32_t tok = __ldg(core_idx + row);
+        int32_t p = (int32_t)(row / g.Lct);
+        int32_t r = (int32_t)(row % g.Lct);
+        int32_t tok = r < g.Lc ? __ldg(core_idx + (int64_t)p * g.Lc + r) : g.L + (r - g.Lc);
         const int32_t slice = prob_slice ? prob_slice[p] : p;
-        dst[i] = __ldg(src + ((int64_t)slice * g.L + tok) * cpr + c);
+        dst[i] = __ldg(src + ((int64_t)slice * g.Ltot + tok) * cpr + c);
     }
 }
 
@@ -444,7 +446,7 @@ cudaError_t launch_gather(const Geometry &g, int32_t n_prob, const int32_t *prob
                           __nv_bfloat16 *Vc, cudaStream_t s)
 {
     if (n_prob == 0) return cudaSuccess;
-    int64_t total = (int64_t)n_prob * g.Lc * (g.d >> 3);
+    int64_t total = (int64_t)n_prob * g.Lct * (g.d >> 3);
     unsigned blocks = (unsigned)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
     gather_rows_kernel<<<dim3(blocks, 3), 256, 0, s>>>(
         g, n_prob, prob_slice, core_idx, reinterpret_cast<const uint4 *>(Q),
@@ -497,7 +499,7 @@ merge_centres_kernel(Geometry g, const int32_t *__restrict__ prob_slice, const i
         for (uint32_t m = members; m; m &= m - 1) {
             const int32_t l = __ffs(m) - 1;
             const int32_t tok = origin + t[2 + l];
-            const uint4 u = __ldg(src + ((int64_t)slice * g.L + tok) * cpr + c);
+            const uint4 u = __ldg(src + ((int64_t)slice * g.Ltot + tok) * cpr + c);
             const uint32_t w[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -511,7 +513,7 @@ merge_centres_kernel(Geometry g, const int32_t *__restrict__ prob_slice, const i
             __nv_bfloat162 v = __floats2bfloat162_rn(acc[2 * i] * inv, acc[2 * i + 1] * inv);
             r[i] = *reinterpret_cast<uint32_t *>(&v);
         }
-        dst[((int64_t)p * g.Lc + seg) * cpr + c] = make_uint4(r[0], r[1], r[2], r[3]);
+        dst[((int64_t)p * g.Lct + seg) * cpr + c] = make_uint4(r[0], r[1], r[2], r[3]);
     }
 }
 
@@ -539,16 +541,17 @@ scatter_rows_kernel(Geometry g, int32_t n_prob, const int32_t *__restrict__ prob
                     uint4 *__restrict__ O)
 {
     const int32_t cpr = g.d >> 3;
-    const int64_t total = (int64_t)n_prob * g.L * cpr;
+    // a video token takes the row of its slot, a text token its own compact row
+    const int64_t total = (int64_t)n_prob * g.Ltot * cpr;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
          i += (int64_t)gridDim.x * blockDim.x) {
         int64_t row = i / cpr;
         int32_t c = (int32_t)(i % cpr);
-        int32_t p = (int32_t)(row / g.L);
-        int32_t tok = (int32_t)(row % g.L);
-        int32_t slot = __ldg(src_slot + row);
+        int32_t p = (int32_t)(row / g.Ltot);
+        int32_t tok = (int32_t)(row % g.Ltot);
+        int32_t slot = tok < g.L ? __ldg(src_slot + (int64_t)p * g.L + tok) : g.Lc + (tok - g.L);
         const int32_t slice = prob_slice ? prob_slice[p] : p;
-        O[((int64_t)slice * g.L + tok) * cpr + c] = __ldg(Oc + ((int64_t)p * g.Lc + slot) * cpr + c);
+        O[((int64_t)slice * g.Ltot + tok) * cpr + c] = __ldg(Oc + ((int64_t)p * g.Lct + slot) * cpr + c);
     }
 }
 
@@ -557,7 +560,7 @@ cudaError_t launch_scatter(const Geometry &g, int32_t n_prob, const int32_t *pro
                            cudaStream_t s)
 {
     if (n_prob == 0) return cudaSuccess;
-    int64_t total = (int64_t)n_prob * g.L * (g.d >> 3);
+    int64_t total = (int64_t)n_prob * g.Ltot * (g.d >> 3);
     unsigned blocks = (unsigned)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
     scatter_rows_kernel<<<blocks, 256, 0, s>>>(g, n_prob, prob_slice, src_slot,
                                                reinterpret_cast<const uint4 *>(Oc),
@@ -616,7 +619,7 @@ mix_combine_kernel(Geometry g, const float *__restrict__ gates, const uint4 *__r
                    uint4 *__restrict__ O)
 {
     const int32_t cpr = g.d >> 3;
-    const int64_t per_slice = (int64_t)g.L * cpr, total = (int64_t)g.B * g.heads * per_slice;
+    const int64_t per_slice = (int64_t)g.Ltot * cpr, total = (int64_t)g.B * g.heads * per_slice;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
          i += (int64_t)gridDim.x * blockDim.x) {
         const int32_t h = (int32_t)((i / per_slice) % g.heads);
@@ -640,7 +643,7 @@ mix_combine_kernel(Geometry g, const float *__restrict__ gates, const uint4 *__r
 cudaError_t launch_mix_combine(const Geometry &g, const float *gates, const __nv_bfloat16 *branches,
                                __nv_bfloat16 *O, cudaStream_t s)
 {
-    int64_t total = (int64_t)g.B * g.heads * g.L * (g.d >> 3);
+    int64_t total = (int64_t)g.B * g.heads * g.Ltot * (g.d >> 3);
     unsigned blocks = (unsigned)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
     mix_combine_kernel<<<blocks, 256, 0, s>>>(g, gates, reinterpret_cast<const uint4 *>(branches),
                                               reinterpret_cast<uint4 *>(O));

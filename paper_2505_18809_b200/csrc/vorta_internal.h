@@ -32,6 +32,9 @@ struct Geometry {
     int32_t half[3], restricted[3];       // floor(w/2); 0 when the window covers the axis
     int32_t bucket[3], nb[3], n_buckets;  // core-set buckets
     int32_t Lc;
+    int32_t Lt;                           // text tokens after the video tokens of every head (joint sequence)
+    int32_t Ltot, Lct;                    // rows per head of Q, K, V, O (L + Lt) and of the compact tensors (Lc + Lt)
+    int32_t text_blocks;                  // KV blocks of bn_tile text keys a sliding item appends: ceil(Lt / bn_tile)
     double ratio;
     // sliding branch blocking: one block = a TMA box of box[0] x box[1] x box[2] tokens
     int32_t box[3], box_rows, bn_tile, boxes_per_tile, max_kv_per_tile;
@@ -55,13 +58,15 @@ struct WorkItem {
     int32_t q_org[2][3];  // per M-block: (w0, h0, t0) of the box, or (row0, 0, 0)
     int32_t out_slice;    // slice of the output tensor the rows are written to (non-compact modes)
     int32_t kv_fast;      // the first kv_fast blocks are 128 real keys each: no column needs masking
-    int32_t pad[2];
+    int32_t kv_text;      // MODE_TILES: blocks [kv_count - kv_text, kv_count) are bn_tile-key blocks of text tokens
+    int32_t pad[1];
 };
 static_assert(sizeof(WorkItem) == 64, "WorkItem must stay 64 bytes");
 
 // Tensor maps of one attention launch (all 5-D: d, W|rows, H, T, slice).
 struct AttnMaps {
     CUtensorMap q[3], k[3], v[3];  // indexed by mode
+    CUtensorMap kt, vt;            // text rows [L, L + Lt) of K and V in boxes of bn_tile rows (sliding items)
 };
 
 struct AttnParams {
@@ -72,8 +77,8 @@ struct AttnParams {
     const int32_t *cta_count;      // [grid]
     const KvEntry *kv_list;
     const uint32_t *colmasks;      // [kMaxMasks][4]
-    __nv_bfloat16 *O;              // [B*heads, L, d]
-    __nv_bfloat16 *Oc;             // [n_compact, Lc, d]
+    __nv_bfloat16 *O;              // [B*heads, L + Lt, d]
+    __nv_bfloat16 *Oc;             // [n_compact, Lc + Lt, d]
     const __nv_bfloat16 *Q, *K, *V;     // originals (SIMT kernel)
     const __nv_bfloat16 *Qc, *Kc, *Vc;  // gathered (SIMT kernel)
     int32_t *status;               // device word: 0 or the code of an expired wait

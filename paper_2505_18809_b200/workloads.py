@@ -35,10 +35,17 @@ class Workload:
     B: int = 1
     bucket: Tuple[int, int, int] = (2, 3, 2)
     merge: bool = False                 # core-set heads merge pruned tokens into the centre (mean)
+    text: int = 0                       # text tokens after the video tokens of every head (MMDiT joint sequence)
 
     @property
     def L(self) -> int:
+        """Video tokens per head."""
         return self.grid[0] * self.grid[1] * self.grid[2]
+
+    @property
+    def rows(self) -> int:
+        """Rows per head of Q, K, V, O: video tokens, then text tokens."""
+        return self.L + self.text
 
 
 def apportion_routes(heads: int, fractions: Sequence[float], seed: int) -> Tuple[int, ...]:
@@ -69,6 +76,10 @@ def config(name: str) -> Workload:
     if name == "wan14b-720p":
         return Workload(name, (21, 45, 80), 40, 128, (4, 8, 8), (3, 3, 3), 0.25,
                         apportion_routes(40, (0.0, 0.8, 0.2), 3), 3, True)
+    if name == "hunyuan-720p-text256":
+        # second workload: the MMDiT joint sequence of HunyuanVideo, 256 text tokens after the video tokens
+        return Workload(name, (33, 45, 80), 24, 128, (4, 8, 8), (3, 3, 3), 0.5,
+                        apportion_routes(24, (0.2, 0.5, 0.3), 2), 2, True, 1, (2, 3, 2), False, 256)
     if name == "hunyuan-720p-3h":
         # profiling case: the HunyuanVideo-720p grid with one head per route, so that a
         # counter capture of one launch stays short while the inputs still exceed L2
@@ -82,6 +93,7 @@ def config(name: str) -> Workload:
 
 
 CONFIG_NAMES = ("tiny", "wan1.3b-480p", "hunyuan-720p", "wan14b-720p")
+JOINT_NAMES = ("hunyuan-720p-text256",)
 PROFILE_NAMES = ("hunyuan-720p-3h", "hunyuan-720p-8c")
 
 
@@ -113,7 +125,8 @@ def _smooth_field(n_chan: int, grid, g: torch.Generator, device) -> torch.Tensor
 
 
 def make_qkv(wl: Workload, device="cpu", heads: Optional[Sequence[int]] = None):
-    """Q, K, V as bf16 [B, heads, L, d] on `device`, token order i = (t*H + h)*W + w.
+    """Q, K, V as bf16 [B, heads, L + text, d] on `device`, video token order i = (t*H + h)*W + w,
+    text tokens (plain N(0,1)) after them.
 
     One generator per (tensor, batch, head), seeded from the workload seed, so a
     subset of heads can be made without the rest (`heads`: which heads to fill; the
@@ -125,7 +138,7 @@ def make_qkv(wl: Workload, device="cpu", heads: Optional[Sequence[int]] = None):
     L = wl.L
     out = []
     for ti in range(3):
-        x = torch.zeros((wl.B, wl.heads, L, wl.d), dtype=torch.bfloat16, device=dev)
+        x = torch.zeros((wl.B, wl.heads, L + wl.text, wl.d), dtype=torch.bfloat16, device=dev)
         for b in range(wl.B):
             for h in (range(wl.heads) if heads is None else heads):
                 g = torch.Generator(device=dev)
@@ -135,6 +148,9 @@ def make_qkv(wl: Workload, device="cpu", heads: Optional[Sequence[int]] = None):
                     f = f.reshape(wl.d, L).t()
                 else:
                     f = torch.randn((L, wl.d), generator=g, device=dev, dtype=torch.float32)
-                x[b, h] = f.to(torch.bfloat16)
+                x[b, h, :L] = f.to(torch.bfloat16)
+                if wl.text:
+                    x[b, h, L:] = torch.randn((wl.text, wl.d), generator=g, device=dev,
+                                              dtype=torch.float32).to(torch.bfloat16)
         out.append(x)
     return tuple(out)

@@ -23,15 +23,16 @@ def oracle_head_rows(wl, Q, K, V, b, h, rows, scale=None, X=None, route=None):
     q, k, v = head_f64(Q, b, h), head_f64(K, b, h), head_f64(V, b, h)
     scale = 1.0 / math.sqrt(wl.d) if scale is None else scale
     route = wl.routes[h] if route is None else route
+    text = getattr(wl, "text", 0)
     if route == 0:
         return oracle.attn_full(q, k, v, scale, q_rows=rows)
     if route == 1:
-        return oracle.attn_sliding(wl.grid, wl.tile, wl.window, q, k, v, scale, q_rows=rows)
+        return oracle.attn_sliding(wl.grid, wl.tile, wl.window, q, k, v, scale, q_rows=rows, text=text)
     x = None if X is None else X
     # the float ratio is what the library sees (the ABI carries a float)
     r = float(np.float32(wl.ratio))
     O, _, _ = oracle.attn_coreset(wl.grid, wl.bucket, r, q, k, v, scale, X=x, q_rows=rows,
-                                  merge=getattr(wl, "merge", False))
+                                  merge=getattr(wl, "merge", False), text=text)
     return O
 
 
@@ -52,10 +53,13 @@ def sample_rows(wl, n: int, seed: int) -> np.ndarray:
         hh2 = hh if pick == 1 else int(g.integers(0, H))
         ww = w if pick == 2 else int(g.integers(0, W))
         forced.add((tt * H + hh2) * W + ww)
+    text = getattr(wl, "text", 0)
+    if text:  # first, last and a few random text tokens
+        forced |= {L, L + text - 1} | {L + int(e) for e in g.integers(0, text, size=4)}
     rows = list(sorted(forced))[:n]
     rest = n - len(rows)
     if rest > 0:
-        extra = g.choice(L, size=min(rest, L), replace=False)
+        extra = g.choice(L + text, size=min(rest, L + text), replace=False)
         rows = sorted(set(rows) | set(int(e) for e in extra))
     return np.asarray(rows, dtype=np.int64)
 

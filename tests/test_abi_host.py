@@ -145,3 +145,23 @@ def test_default_bucket_is_the_papers():
     assert a.info.Lc == b.info.Lc == 64 and a.info.n_buckets == b.info.n_buckets == 2 * 3 * 4
     a.close()
     b.close()
+
+
+def test_joint_sequence_accounting_host_only():
+    """Text tokens: FLOPs per head from the definitions (pairs attended), against the oracle's masks."""
+    from paper_2505_18809_b200.workloads import Workload
+    wl = Workload("j", (5, 6, 7), 3, 64, (2, 2, 3), (3, 1, 3), 0.5, (0, 1, 2), 1, False, 1, (2, 3, 2), False, 19)
+    p = vb.Plan.from_workload(wl, host_only=True)
+    info = p.info
+    p.close()
+    L, Lt, d = wl.L, wl.text, wl.d
+    assert info.L == L and info.text_tokens == Lt
+    assert info.flops_full_head == pytest.approx(4.0 * d * (L + Lt) ** 2, rel=1e-12)
+    M = oracle.sta_token_mask(wl.grid, wl.tile, wl.window)
+    pairs = float(M.sum()) + L * Lt + Lt * (L + Lt)
+    assert info.flops_sliding_head == pytest.approx(4.0 * d * pairs, rel=1e-12)
+    Lc = oracle.coreset_len(wl.grid, wl.bucket, float(np.float32(wl.ratio)))
+    assert info.Lc == Lc
+    assert info.flops_coreset_head == pytest.approx(4.0 * d * (Lc + Lt) ** 2, rel=1e-12)
+    with pytest.raises(vb.VortaError):
+        vb.Plan(1, 1, (2, 2, 2), 64, (1, 1, 1), (1, 1, 1), 0.5, (0,), host_only=True, text=-1)

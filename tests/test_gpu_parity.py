@@ -298,6 +298,71 @@ def test_host_buffer_entry_point_many_heads_batch_and_route_change():
     p.close()
 
 
+# --------------------------------------------------------------------------- joint sequences (video + text tokens)
+def joint_workloads():
+    W = Workload
+    #  name, grid, heads, d, tile, window, ratio, routes, seed, smooth, B, bucket, merge, text
+    return [
+        # 256-token tiles, real windows, ragged H and W; 77 text tokens (one cut text block per item)
+        W("joint-256tile", (9, 21, 27), 3, 128, (4, 8, 8), (3, 3, 3), 0.5, (1, 0, 2), 51, True, 1, (2, 3, 2), False, 77),
+        # 64-token tiles: text keys in blocks of 64, 130 of them (three blocks, the last of 2); batch of 2
+        W("joint-tile64", (10, 12, 20), 4, 128, (4, 4, 4), (3, 3, 3), 0.25, (1, 1, 2, 0), 52, False, 2, (2, 3, 2), False, 130),
+        # 27-token tiles (blocks of 32 columns, 27 real): one text token; d = 64
+        W("joint-tile27-one-text", (7, 9, 12), 3, 64, (3, 3, 3), (1, 3, 5), 0.5, (1, 2, 1), 53, False, 1, (2, 3, 2), False, 1),
+        # exactly two whole text blocks of 128; merged core-set heads
+        W("joint-2x128-merge", (4, 8, 16), 3, 128, (2, 8, 8), (3, 3, 3), 0.5, (2, 1, 0), 54, False, 1, (2, 3, 2), True, 256),
+        # more text tokens than video tokens
+        W("joint-text-heavy", (2, 4, 6), 3, 128, (1, 2, 2), (1, 1, 3), 0.5, (0, 1, 2), 55, False, 1, (2, 3, 2), False, 300),
+    ]
+
+
+@pytest.mark.parametrize("kernel", [vb.VORTA_KERNEL_SIMT, vb.VORTA_KERNEL_TCGEN05], ids=["simt", "tcgen05"])
+@pytest.mark.parametrize("wl", joint_workloads(), ids=lambda w: w.name)
+def test_joint_sequence_all_rows(wl, kernel):
+    """Video tokens followed by text tokens: text keys visible to every query, text queries see
+    every key, core-set selection prunes video tokens only."""
+    Q, K, V = workloads.make_qkv(wl, DEV)
+    assert Q.shape[2] == wl.L + wl.text
+    p = vb.Plan.from_workload(wl)
+    assert p.info.text_tokens == wl.text
+    core_heads = [h for h in range(wl.heads) if wl.routes[h] == 2]
+    if core_heads:
+        core, src = p.coreset_select(K)
+        r = float(np.float32(wl.ratio))
+        for h in core_heads:
+            c, s_ = oracle.coreset_select(wl.grid, wl.bucket, r, head_f64(K, 0, h)[: wl.L])
+            assert np.array_equal(core[0, h].cpu().numpy(), c) and np.array_equal(src[0, h].cpu().numpy(), s_)
+    O = run_layer(p, wl, Q, K, V, kernel)
+    for b in range(wl.B):
+        for h in range(wl.heads):
+            want = oracle_head_rows(wl, Q, K, V, b, h, None)
+            assert_close(O[b, h], want, f"{wl.name} b{b} h{h} route {wl.routes[h]}")
+    p.close()
+
+
+def test_joint_sequence_host_entry_and_soft_mixture():
+    wl = joint_workloads()[0]
+    Q, K, V = workloads.make_qkv(wl, DEV)
+    p = vb.Plan.from_workload(wl)
+    O = run_layer(p, wl, Q, K, V, vb.VORTA_KERNEL_TCGEN05)
+    Qh, Kh, Vh = (t.cpu().pin_memory() for t in (Q, K, V))
+    Oh = torch.full_like(Qh, float("nan")).pin_memory()
+    scratch = torch.empty(p.info.host_call_scratch_bytes, dtype=torch.uint8, device=DEV)
+    p.routed_attention_host(Qh, Kh, Vh, Oh, scratch)
+    assert p.device_status() == 0
+    assert torch.equal(Oh.view(torch.int16), O.cpu().view(torch.int16))
+    gates = torch.tensor([[0.2, 0.5, 0.3], [1.0, 0.0, 0.0], [0.1, 0.1, 0.8]], device=DEV)
+    Om = p.soft_mixture(Q, K, V, gates)
+    assert p.device_status() == 0
+    scale = 1.0 / np.sqrt(wl.d)
+    for h in range(wl.heads):
+        want = oracle.soft_mixture(wl.grid, wl.tile, wl.window, wl.bucket, float(np.float32(wl.ratio)),
+                                   head_f64(Q, 0, h), head_f64(K, 0, h), head_f64(V, 0, h), scale,
+                                   gates[h].double().cpu().numpy(), text=wl.text)
+        assert_close(Om[0, h], want, f"mixture h{h}")
+    p.close()
+
+
 # --------------------------------------------------------------------------- the named configurations
 def check_config(wl, rows_per_head, kernels=(vb.VORTA_KERNEL_TCGEN05,)):
     Q, K, V = workloads.make_qkv(wl, DEV)
@@ -308,7 +373,7 @@ def check_config(wl, rows_per_head, kernels=(vb.VORTA_KERNEL_TCGEN05,)):
     if core_heads:
         core, src = p.coreset_select(K)
         for h in core_heads:
-            c, s = oracle.coreset_select(wl.grid, wl.bucket, float(np.float32(wl.ratio)), head_f64(K, 0, h))
+            c, s = oracle.coreset_select(wl.grid, wl.bucket, float(np.float32(wl.ratio)), head_f64(K, 0, h)[: wl.L])
             assert np.array_equal(core[0, h].cpu().numpy(), c), h
             assert np.array_equal(src[0, h].cpu().numpy(), s), h
         del core, src
@@ -340,6 +405,10 @@ def test_config_hunyuan_720p_sampled_rows():
 
 def test_config_wan14b_720p_sampled_rows():
     check_config(workloads.config("wan14b-720p"), 32)
+
+
+def test_config_hunyuan_720p_with_256_text_tokens_sampled_rows():
+    check_config(workloads.config("hunyuan-720p-text256"), 40)
 
 
 def test_config_route_mix_sweep_sampled_rows():
