@@ -518,7 +518,8 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
         if (m >= wp->n_mblk) continue;
         const int32_t w_mode = wp->mode, w_kv_len = wp->kv_len, w_kv_count = wp->kv_count;
         const KvEntry *kv_entries = p.kv_list + wp->kv_begin;
-        const int32_t n_boxes = w_mode == MODE_TILES ? w_kv_count - wp->kv_text : w_kv_count;  // the rest: text-token blocks
+        const bool has_text = w_mode == MODE_TILES && wp->kv_text > 0;
+        const int32_t n_boxes = has_text ? w_kv_count - wp->kv_text : w_kv_count;  // the rest: text-token blocks
         const int32_t bn = w_mode == MODE_TILES ? p.g.bn_tile : kBlockM;
         const int32_t sh = bn > 64 ? 1 : 0;  // log2 of the sub-blocks per KV block
         const int32_t n_sub = w_kv_count << sh;
@@ -552,11 +553,11 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
         };
         // strike the columns of sub-block u that are not keys (mask class `id` of its block,
         // fetched ahead by the caller; blocks of text tokens have none: their last one is cut at Lt)
-        auto apply_mask = [&](int32_t u, uint32_t id, uint32_t(&s)[64]) {
+        auto apply_mask = [&](auto with_text, int32_t u, uint32_t id, uint32_t(&s)[64]) {
             const int32_t h = u & sh;
             uint32_t m0 = 0, m1 = 0;
             bool partial = false;
-            if ((u >> sh) >= n_boxes) {
+            if (decltype(with_text)::value && (u >> sh) >= n_boxes) {
                 // text keys of this sub-block: what is left of Lt, at most the block's bn columns
                 const int32_t valid = min(p.g.Lt - ((u >> sh) - n_boxes) * bn, bn) - 64 * h;
                 if (valid < 64) {
@@ -583,13 +584,16 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
         // One sub-block: s holds the scores of u and row_max covers them.  Writes P(u), then
         // reads S(u+1) and moves row_max over it.  full: u and u+1 are both whole 64-key
         // sub-blocks of unmasked blocks, so nothing about widths or masks is looked at.
-        auto step = [&](auto full, int32_t u, uint32_t(&s)[64]) -> bool {
+        // with_text: the item ends in blocks of text tokens (looked at only then)
+        auto step = [&](auto full, auto with_text, int32_t u, uint32_t(&s)[64]) -> bool {
             constexpr bool kFull = decltype(full)::value;
+            constexpr bool kText = decltype(with_text)::value;
             const int32_t b = u & 1;
             const bool has_next = kFull || u + 1 < n_sub;
             // mask class of the next sub-block's KV block, in flight under the exponentials
             const uint32_t next_id =
-                (!kFull && has_next && w_mode == MODE_TILES && ((u + 1) >> sh) < n_boxes) ? kv_entries[(u + 1) >> sh].mask_id : 0u;
+                (!kFull && has_next && w_mode == MODE_TILES && (!kText || ((u + 1) >> sh) < n_boxes))
+                    ? kv_entries[(u + 1) >> sh].mask_id : 0u;
             if (row == 0) TRACE(2 + m, u, 0);
             // P = exp2(S * scale - max) as packed bf16 over the first half of the buffer
             float2 sum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
@@ -604,7 +608,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
             if (has_next) {
                 if (!load_sub(full, u + 1, s)) return false;
                 if (row == 0) TRACE(2 + m, u, 3);
-                if (!kFull) apply_mask(u + 1, next_id, s);
+                if (!kFull) apply_mask(with_text, u + 1, next_id, s);
                 const float m_new = fmaxf(row_max, row_max64(s) * scale);
                 if (__any_sync(0xffffffffu, m_new - row_max > kRescaleThreshold)) {
                     // Lazy rescale: O and the row sum move to the new maximum only when it grew by
@@ -625,15 +629,20 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
 
         uint32_t s[64];
         if (!load_sub(std::false_type{}, 0, s)) return;
-        apply_mask(0, (w_mode == MODE_TILES && n_boxes > 0) ? kv_entries[0].mask_id : 0u, s);
+        apply_mask(std::true_type{}, 0, (w_mode == MODE_TILES && n_boxes > 0) ? kv_entries[0].mask_id : 0u, s);
         row_max = row_max64(s) * scale;
         // the leading unmasked blocks, then whatever is cut, short or last
         const int32_t n_full = min(2 * wp->kv_fast, n_sub) - 1;  // steps whose u and u+1 are both whole
         int32_t u = 0;
         for (; u < n_full; ++u)
-            if (!step(std::true_type{}, u, s)) return;
-        for (; u < n_sub; ++u)
-            if (!step(std::false_type{}, u, s)) return;
+            if (!step(std::true_type{}, std::false_type{}, u, s)) return;
+        if (has_text) {
+            for (; u < n_sub; ++u)
+                if (!step(std::false_type{}, std::true_type{}, u, s)) return;
+        } else {
+            for (; u < n_sub; ++u)
+                if (!step(std::false_type{}, std::false_type{}, u, s)) return;
+        }
 
         // the commits that follow the last two PV MMAs: O is complete
         for (int32_t u = max(n_sub - 2, 0); u < n_sub; ++u) {
