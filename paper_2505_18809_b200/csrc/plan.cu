@@ -321,10 +321,27 @@ int build_list(vorta_plan *p, vorta_plan::WorkList &wl, const std::vector<uint8_
 }
 
 // Groups of heads for the host-buffer entry point.  Heads are taken in descending order of
-// attention work and cut into at most kHostChunks groups of equal head count (equal copy
-// time): the expensive groups run first, so the kernels always have a group to work on
-// while the copy engine brings in the cheap ones.
+// attention work and cut into at most kHostChunks groups: the expensive groups run first, so
+// the kernels always have a group to work on while the copy engine brings in the cheap ones.
+// The first group's copy in and the last group's copy out are the only transfers nothing
+// overlaps, so the first groups are small (1, then 2 heads) and so is the last (1 head); the
+// heads between are split evenly.
 constexpr int kHostChunks = 8;
+
+std::vector<int32_t> host_chunk_sizes(int32_t heads)
+{
+    std::vector<int32_t> sizes;
+    if (heads < 2 * kHostChunks) {  // few heads: equal groups
+        const int32_t n = std::min<int32_t>(kHostChunks, heads), per = (heads + n - 1) / n;
+        for (int32_t left = heads; left > 0; left -= per) sizes.push_back(std::min(per, left));
+        return sizes;
+    }
+    sizes = {1, 2};
+    const int32_t mid = heads - 4, n_mid = kHostChunks - 3;
+    for (int32_t i = 0; i < n_mid; ++i) sizes.push_back(mid / n_mid + (i < mid % n_mid ? 1 : 0));
+    sizes.push_back(1);
+    return sizes;
+}
 
 int build_host_chunks(vorta_plan *p)
 {
@@ -339,9 +356,9 @@ int build_host_chunks(vorta_plan *p)
     std::vector<int32_t> order(g.heads);
     for (int32_t h = 0; h < g.heads; ++h) order[h] = h;
     std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return cost[a] > cost[b]; });
-    const int32_t n_chunks = std::min<int32_t>(kHostChunks, g.heads);
-    const int32_t per = (g.heads + n_chunks - 1) / n_chunks;
-    const size_t want = (size_t)((g.heads + per - 1) / per);
+    const std::vector<int32_t> sizes = host_chunk_sizes(g.heads);
+    const int32_t per = *std::max_element(sizes.begin(), sizes.end());
+    const size_t want = sizes.size();
     while (p->chunks.size() < want) {
         p->chunks.emplace_back();
         vorta_plan::HostChunk &c = p->chunks.back();
@@ -351,9 +368,10 @@ int build_host_chunks(vorta_plan *p)
             cudaMalloc(&c.d_core_xslice, sizeof(int32_t) * g.B * per) != cudaSuccess)
             return VORTA_ERR_CUDA;
     }
-    for (size_t ci = 0; ci < want; ++ci) {
+    size_t first = 0;
+    for (size_t ci = 0; ci < want; first += (size_t)sizes[ci], ++ci) {
         vorta_plan::HostChunk &c = p->chunks[ci];
-        c.heads.assign(order.begin() + ci * per, order.begin() + std::min<size_t>((ci + 1) * per, g.heads));
+        c.heads.assign(order.begin() + first, order.begin() + first + sizes[ci]);
         std::sort(c.heads.begin(), c.heads.end());
         std::vector<uint8_t> branches(g.heads, 0);
         std::vector<int32_t> core;
