@@ -126,6 +126,22 @@ def test_routed_attention_small_all_rows(wl, kernel):
     p.close()
 
 
+def test_many_slices_small_heads():
+    """Batch 3 x 70 heads of 48 tokens: slice indexing of every stage (the 5th TMA coordinate,
+    compact problem numbering, per-batch core-set tables) with far more heads than SMs' items."""
+    routes = tuple((h * 7 + 3) % 3 for h in range(70))
+    wl = Workload("many-slices", (2, 4, 6), 70, 64, (1, 2, 2), (3, 3, 3), 0.5, routes, 61, False, 3)
+    Q, K, V = workloads.make_qkv(wl, DEV)
+    p = vb.Plan.from_workload(wl)
+    O = run_layer(p, wl, Q, K, V, vb.VORTA_KERNEL_TCGEN05)
+    for b in range(wl.B):
+        for h in range(0, wl.heads, 3):
+            for hh in (h, min(h + 1 + b, wl.heads - 1)):
+                want = oracle_head_rows(wl, Q, K, V, b, hh, None)
+                assert_close(O[b, hh], want, f"b{b} h{hh} route {wl.routes[hh]}")
+    p.close()
+
+
 def test_pruned_rows_copy_their_centre_and_reruns_are_bitwise_equal():
     wl = small_workloads()[2]
     Q, K, V = workloads.make_qkv(wl, DEV)
