@@ -218,7 +218,9 @@ VORTA_API int vorta_routed_attention(const vorta_plan *plan, const void *Q, cons
  * vorta_routed_attention gives.  dev_scratch: device memory of at least
  * vorta_plan_info().host_call_scratch_bytes, 256-byte aligned.  Two calls on the
  * same plan must not be in flight on different streams at once (they share the
- * plan's copy streams and events).
+ * plan's copy streams and events).  The first call after plan creation or a route
+ * change builds the groups' work lists (small device allocations, synchronous
+ * copies) before it enqueues.
  */
 VORTA_API int vorta_routed_attention_host(const vorta_plan *plan, const void *Q_host,
                                           const void *K_host, const void *V_host, void *O_host,

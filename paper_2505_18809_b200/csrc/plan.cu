@@ -50,7 +50,8 @@ struct vorta_plan {
         int32_t *d_core_slice = nullptr, *d_core_xslice = nullptr;
         cudaEvent_t ev_in = nullptr, ev_done = nullptr;
     };
-    std::vector<HostChunk> chunks;
+    mutable std::vector<HostChunk> chunks;
+    mutable bool chunks_stale = true;  // the groups are rebuilt by the first host-buffer call after a route change
     cudaStream_t s_in = nullptr, s_out = nullptr;  // copy-in and copy-out streams of that entry point
     cudaEvent_t ev_start = nullptr, ev_out = nullptr;
     int32_t *d_core_slice = nullptr;  // [B * n_core]: compact problem -> b*heads + head
@@ -419,7 +420,8 @@ int build_work(vorta_plan *p)
         (cudaMemcpy(p->d_core_slice, core_slice.data(), sizeof(int32_t) * g.B * n_core, cudaMemcpyHostToDevice) != cudaSuccess ||
          cudaMemcpy(p->d_core_xslice, core_x.data(), sizeof(int32_t) * g.B * n_core, cudaMemcpyHostToDevice) != cudaSuccess))
         return VORTA_ERR_CUDA;
-    return build_host_chunks(p);
+    p->chunks_stale = true;
+    return VORTA_OK;
 }
 
 struct DeviceGuard {
@@ -975,6 +977,13 @@ int vorta_routed_attention_host(const vorta_plan *p, const void *Qh, const void 
     if (!guard.ok) return VORTA_ERR_CUDA;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const Geometry &g = p->g;
+    if (p->chunks_stale) {
+        // first call since the routes were set: build the groups' work lists (small device
+        // allocations and synchronous copies; later calls only enqueue)
+        int rc = build_host_chunks(const_cast<vorta_plan *>(p));
+        if (rc != VORTA_OK) return rc;
+        p->chunks_stale = false;
+    }
     const int64_t tb = tensor_bytes(g), tba = align_up(tb, 256);
     char *base = static_cast<char *>(scratch);
     char *dq = base, *dk = base + tba, *dv = base + 2 * tba, *dO = base + 3 * tba;
