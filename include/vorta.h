@@ -209,9 +209,10 @@ VORTA_API int vorta_routed_attention(const vorta_plan *plan, const void *Q, cons
  * The same layer with HOST buffers (bf16 [B, heads, L, d]; pinned memory, or the
  * copies neither overlap nor return early).  The heads are worked through in up to
  * eight groups, most expensive first: the plan's own copy-in stream brings a group's
- * Q, K, V into dev_scratch, the layer's kernels for that group run on `stream`, and
- * the plan's copy-out stream returns its O, so that copies and kernels of different
- * groups overlap.  The call starts after the work already enqueued on `stream` and
+ * Q, K, V into dev_scratch, the layer's kernels for that group run on `stream` or on
+ * a second kernel stream of the plan (groups alternate, so that one group's kernels
+ * start in the SMs the previous group's last blocks leave), and the plan's copy-out
+ * stream returns its O, so that copies and kernels of different groups overlap.  The call starts after the work already enqueued on `stream` and
  * `stream` ends up waiting for the last copy out: to the caller it is one operation
  * on `stream`.  Returns after enqueueing (synchronise `stream` before reading
  * O_host or reusing dev_scratch from another stream).  The result is the one

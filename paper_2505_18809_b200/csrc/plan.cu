@@ -53,6 +53,7 @@ struct vorta_plan {
     mutable std::vector<HostChunk> chunks;
     mutable bool chunks_stale = true;  // the groups are rebuilt by the first host-buffer call after a route change
     cudaStream_t s_in = nullptr, s_out = nullptr;  // copy-in and copy-out streams of that entry point
+    cudaStream_t s_alt = nullptr;                  // second kernel queue: odd groups run here, even ones on the caller's stream
     cudaEvent_t ev_start = nullptr, ev_out = nullptr;
     int32_t *d_core_slice = nullptr;  // [B * n_core]: compact problem -> b*heads + head
     int32_t *d_core_xslice = nullptr; // same for a shared X with one head
@@ -162,6 +163,7 @@ void free_device(vorta_plan *p)
     p->chunks.clear();
     if (p->s_in) cudaStreamDestroy(p->s_in);
     if (p->s_out) cudaStreamDestroy(p->s_out);
+    if (p->s_alt) cudaStreamDestroy(p->s_alt);
     if (p->ev_start) cudaEventDestroy(p->ev_start);
     if (p->ev_out) cudaEventDestroy(p->ev_out);
     cudaFree(p->d_status);
@@ -614,6 +616,7 @@ int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
         for (auto &e : set) ok = ok && cudaEventCreate(&e) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&p->s_in, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&p->s_out, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&p->s_alt, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&p->ev_start, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&p->ev_out, cudaEventDisableTiming) == cudaSuccess;
     // the mask builder runs once per shape; its per-tile counts come back for the work list
@@ -671,7 +674,9 @@ int vorta_plan_info(const vorta_plan *p, vorta_plan_info_t *o)
     }
     o->workspace_bytes = workspace_layout(g, (int64_t)g.B * o->n_coreset).total;
     o->workspace_bytes_max = workspace_layout(g, (int64_t)g.B * g.heads).total;
-    o->host_call_scratch_bytes = 4 * align_up(tensor_bytes(g), 256) + o->workspace_bytes;
+    // four tensors, then one core-set workspace per group of heads (their sizes add up to the layer's,
+    // plus alignment padding per group)
+    o->host_call_scratch_bytes = 4 * align_up(tensor_bytes(g), 256) + o->workspace_bytes + kHostChunks * 8 * 256;
     o->mixture_workspace_bytes = mixture_workspace_bytes(g);
     o->text_tokens = g.Lt;
     o->flops_full_head = 4.0 * g.d * (double)g.Ltot * (double)g.Ltot;
@@ -987,21 +992,28 @@ int vorta_routed_attention_host(const vorta_plan *p, const void *Qh, const void 
     const int64_t tb = tensor_bytes(g), tba = align_up(tb, 256);
     char *base = static_cast<char *>(scratch);
     char *dq = base, *dk = base + tba, *dv = base + 2 * tba, *dO = base + 3 * tba;
-    void *ws = info.workspace_bytes ? base + 4 * tba : nullptr;
+    void *ws = base + 4 * tba;
     const char *hq = static_cast<const char *>(Qh), *hk = static_cast<const char *>(Kh),
                *hv = static_cast<const char *>(Vh);
     char *ho = static_cast<char *>(Oh);
     const int64_t hb = (int64_t)g.Ltot * g.d * (int64_t)sizeof(__nv_bfloat16);  // one head of one tensor
 
-    // Three queues: copies in (own stream), kernels (the caller's stream), copies out (own
-    // stream).  Group c's kernels wait for its copies in; its copy out waits for its kernels.
-    // Everything starts after the work already in the caller's stream and the caller's stream
-    // ends up waiting for the last copy out, so the call as a whole behaves as one operation
-    // enqueued on `stream`.
+    // Four queues: copies in (own stream), kernels (the caller's stream for even groups, a second
+    // stream for odd ones), copies out (own stream).  Group c's kernels wait for its copies in; its
+    // copy out waits for its kernels.  Consecutive groups sit in different kernel queues and use
+    // different slices of the core-set workspace, so the persistent CTAs of the next group move
+    // into the SMs the tail of the current one leaves.  Everything starts after the work already
+    // in the caller's stream and the caller's stream ends up waiting for the last copy out (which
+    // waited for every group's kernels), so the call as a whole behaves as one operation enqueued
+    // on `stream`.
     if (cudaEventRecord(p->ev_start, s) != cudaSuccess || cudaStreamWaitEvent(p->s_in, p->ev_start, 0) != cudaSuccess ||
-        cudaStreamWaitEvent(p->s_out, p->ev_start, 0) != cudaSuccess)
+        cudaStreamWaitEvent(p->s_out, p->ev_start, 0) != cudaSuccess ||
+        cudaStreamWaitEvent(p->s_alt, p->ev_start, 0) != cudaSuccess)
         return VORTA_ERR_CUDA;
+    int64_t ws_off = 0;
+    int32_t ci = 0;
     for (const vorta_plan::HostChunk &c : p->chunks) {
+        cudaStream_t sk = (ci++ & 1) ? p->s_alt : s;
         for (int32_t b = 0; b < g.B; ++b)
             for (int32_t h : c.heads) {
                 const int64_t off = ((int64_t)b * g.heads + h) * hb;
@@ -1010,14 +1022,16 @@ int vorta_routed_attention_host(const vorta_plan *p, const void *Qh, const void 
                     cudaMemcpyAsync(dv + off, hv + off, hb, cudaMemcpyHostToDevice, p->s_in) != cudaSuccess)
                     return VORTA_ERR_CUDA;
             }
-        if (cudaEventRecord(c.ev_in, p->s_in) != cudaSuccess || cudaStreamWaitEvent(s, c.ev_in, 0) != cudaSuccess)
+        if (cudaEventRecord(c.ev_in, p->s_in) != cudaSuccess || cudaStreamWaitEvent(sk, c.ev_in, 0) != cudaSuccess)
             return VORTA_ERR_CUDA;
         __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(dO);
+        void *ws_c = c.n_core ? static_cast<char *>(ws) + ws_off : nullptr;
+        ws_off += align_up(workspace_layout(g, (int64_t)g.B * c.n_core).total, 256);
         int rc = run_layer(p, c.wl, c.n_core, c.d_core_slice, c.d_core_xslice, reinterpret_cast<const __nv_bfloat16 *>(dq),
                            reinterpret_cast<const __nv_bfloat16 *>(dk), reinterpret_cast<const __nv_bfloat16 *>(dv), o, o,
-                           nullptr, 0, ws, s, false);
+                           nullptr, 0, ws_c, sk, false);
         if (rc != VORTA_OK) return rc;
-        if (cudaEventRecord(c.ev_done, s) != cudaSuccess || cudaStreamWaitEvent(p->s_out, c.ev_done, 0) != cudaSuccess)
+        if (cudaEventRecord(c.ev_done, sk) != cudaSuccess || cudaStreamWaitEvent(p->s_out, c.ev_done, 0) != cudaSuccess)
             return VORTA_ERR_CUDA;
         for (int32_t b = 0; b < g.B; ++b)
             for (int32_t h : c.heads) {
