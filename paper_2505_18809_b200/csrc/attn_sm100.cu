@@ -8,7 +8,8 @@
 //                  the row-major [T, H, W, d] layout;
 //   core-set head  like a full head, over the gathered rows.
 //
-// Warp roles (320 threads, so that every thread may hold 200 registers):
+// Warp roles (320 threads; every role is compiled for the launch bound's 168 registers,
+// three warps on an SM sub-partition's 16 K registers; no setmaxnreg):
 //   warp 0        TMA producer: Q once per item, then K_j, V_j into a 4-slot ring
 //   warp 1        TMEM allocation; MMA issuer: S = Q K^T and O += P V as tcgen05.mma,
 //                 accumulators in TMEM
