@@ -257,6 +257,9 @@ def run_ours(args):
     vb.lib()
 
     wl = get_workload(args.workload)
+    if args.merge:
+        import dataclasses
+        wl = dataclasses.replace(wl, name=wl.name + "+merge", merge=True)
     pk = peaks()
     full_layer_flops = None
     if args.shard_heads:
@@ -436,6 +439,8 @@ def main():
     ap.add_argument("--reference-rows", type=int, default=16, help="oracle rows per head per step (--impl reference)")
     ap.add_argument("--kernel", type=int, default=-1, help="attention kernel id (see vorta.h); -1 = library default")
     ap.add_argument("--mixture", action="store_true", help="time vorta_soft_mixture (all three branches per head)")
+    ap.add_argument("--merge", action="store_true",
+                    help="core-set heads merge the pruned tokens into their centre (mean) before attention")
     ap.add_argument("--shard-heads", action="store_true",
                     help="strong scaling: one layer, heads split over the ranks (default: one layer per rank)")
     ap.add_argument("--no-e2e", action="store_true")
