@@ -42,6 +42,9 @@ def small_workloads():
         W("ratio-one", (4, 6, 8), 2, 64, (2, 3, 4), (3, 3, 3), 1.0, (2, 2), 26, False),
         # bucket other than the default, grid smaller than one tile on T
         W("bucket-133", (1, 14, 15), 2, 128, (2, 4, 4), (3, 3, 3), 0.34, (2, 1), 27, False, 1, (1, 3, 3)),
+        # the largest bucket the library takes (32 tokens), cut by the grid on every axis; d = 128 and 64
+        W("bucket-32", (5, 9, 10), 2, 128, (2, 4, 4), (3, 3, 3), 0.3, (2, 2), 28, True, 1, (2, 4, 4)),
+        W("bucket-32-d64", (6, 6, 7), 2, 64, (2, 4, 4), (3, 3, 3), 0.6, (2, 1), 29, False, 2, (4, 2, 4)),
         # the attention kernel's sub-block pipeline at its shortest: window of one tile, so an item has
         # one KV block: 1 sub-block (32- and 64-token tiles), 2 (128-token tile), 4 (256-token tile)
         W("one-sub-32", (4, 8, 8), 2, 128, (2, 4, 4), (1, 1, 1), 0.5, (1, 1), 41, False),
