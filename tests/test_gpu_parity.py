@@ -163,6 +163,25 @@ def test_the_most_slices_the_library_takes():
         vb.Plan(2, 32768, wl.grid, 64, wl.tile, wl.window, 0.5, (0,) * 32768, host_only=True)
 
 
+@pytest.mark.parametrize("grid,tile,bucket", [((1, 1, 32767), (1, 1, 64), (1, 1, 12)), ((32767, 1, 1), (4, 1, 1), (2, 1, 1))],
+                         ids=["W-32767", "T-32767"])
+def test_longest_axis_the_library_takes(grid, tile, bucket):
+    """A grid axis of 32 767 (the limit): tile coordinates at the top of the int16 range, 8 192
+    one-box tiles along T; sampled rows of every route."""
+    wl = Workload("long-axis", grid, 3, 64, tile, (3, 3, 3), 0.5, (0, 1, 2), 63, False, 1, bucket)
+    Q, K, V = workloads.make_qkv(wl, DEV)
+    p = vb.Plan.from_workload(wl)
+    assert np.array_equal(p.block_mask(), oracle.sta_block_mask(wl.grid, wl.tile, wl.window))
+    O = run_layer(p, wl, Q, K, V, vb.VORTA_KERNEL_TCGEN05)
+    for h in range(3):
+        rows = sample_rows(wl, 64, 2000 + h)
+        want = oracle_head_rows(wl, Q, K, V, 0, h, rows)
+        assert_close(O[0, h][torch.from_numpy(rows).to(DEV)], want, f"h{h}")
+    p.close()
+    with pytest.raises(vb.VortaError):
+        vb.Plan(1, 1, (1, 1, 32768), 64, tile, (3, 3, 3), 0.5, (0,), host_only=True)
+
+
 def test_pruned_rows_copy_their_centre_and_reruns_are_bitwise_equal():
     wl = small_workloads()[2]
     Q, K, V = workloads.make_qkv(wl, DEV)
