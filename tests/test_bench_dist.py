@@ -6,6 +6,7 @@ import socket
 import subprocess
 import sys
 
+import pytest
 import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
@@ -68,3 +69,19 @@ def test_window_key_count_matches_the_oracle_mask():
     M = oracle.sta_token_mask(wl.grid, wl.tile, wl.window)
     for tok in (0, 17, 100, wl.L - 1):
         assert bench._window_keys(wl, tok) == int(M[tok].sum())
+
+
+def test_cpu_baseline_flop_accounting_equals_the_plan_accounting_when_every_row_is_sampled():
+    """bench.time_oracle counts 4*d*(pairs attended) of the rows it runs; with all rows of a small
+    joint workload (text tokens included) that must be the plan's flops_layer."""
+    import torch
+    from paper_2505_18809_b200 import binding as vb, workloads
+    from paper_2505_18809_b200.workloads import Workload
+    wl = Workload("acc", (4, 6, 5), 3, 64, (2, 2, 2), (3, 1, 3), 0.5, (0, 1, 2), 3, False, 1, (2, 3, 2), False, 7)
+    Q, K, V = workloads.make_qkv(wl, "cpu")
+    flops, secs, heads, threads = bench.time_oracle(wl, Q, K, V, wl.L + wl.text, 1e9)
+    p = vb.Plan.from_workload(wl, host_only=True)
+    want = p.info.flops_layer
+    p.close()
+    assert heads == wl.heads and threads >= 1 and secs > 0
+    assert flops == pytest.approx(want, rel=1e-12)
