@@ -128,9 +128,11 @@ typedef struct {
  * CUDA kernel) and the ordered work list of the persistent attention kernel.
  * Reads desc and desc->routes (host) during the call only.  *out receives the
  * plan; free it with vorta_plan_destroy.
- * Unsupported (VORTA_ERR_UNSUPPORTED): d not in {64,128}; a tile with more than
- * 256 tokens, or with more than 128 tokens and an odd tT; a tile extent > 256;
- * a bucket with more than 32 tokens.
+ * Unsupported (VORTA_ERR_UNSUPPORTED): d not in {64,128}; a tile that cannot be cut
+ * into at most 8 equal boxes of at most 128 tokens (cuts along any of its axes; a
+ * 6 x 9 x 8 tile is four 3 x 9 x 4 boxes, a tile of more than 1 024 tokens or a
+ * 131-token one has no such cut); a tile extent > 256; a bucket with more than 32
+ * tokens.
  */
 VORTA_API int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out);
 

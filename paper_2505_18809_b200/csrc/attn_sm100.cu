@@ -50,7 +50,8 @@ constexpr uint32_t kTileBytes = 32768;    // two halves (d = 128)
 constexpr uint32_t kSmemQ = 0;
 constexpr uint32_t kSmemKV = 2 * kTileBytes;
 constexpr uint32_t kSmemBars = kSmemKV + kStages * kTileBytes;
-constexpr uint32_t kSmemTotal = kSmemBars + 512;
+constexpr uint32_t kCtlBytes = 2048;  // control block: barriers, flags, the column-mask classes
+constexpr uint32_t kSmemTotal = kSmemBars + kCtlBytes;
 constexpr uint32_t kSmemAlloc = kSmemTotal + 1024;  // slack to align the base to 1024 B
 constexpr float kRescaleThreshold = 8.0f;           // log2 units the row maximum may grow before O is rescaled
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
@@ -74,7 +75,8 @@ struct Ctl {
     volatile int32_t abort;
     uint32_t colmasks[kMaxMasks * 4];  // copy of the plan's column-mask classes
 };
-static_assert(sizeof(Ctl) <= 512, "control block outgrew its reservation");
+static_assert(sizeof(Ctl) <= kCtlBytes, "control block outgrew its reservation");
+static_assert(kMaxMasks * 4 <= kAttnThreads, "one thread copies one word of the column masks");
 
 // Optional cycle trace of one CTA (compiled in only with -DVORTA_TRACE; a debugging aid).
 #ifdef VORTA_TRACE

@@ -111,6 +111,32 @@ bool make_map(CUtensorMap *m, const void *base, int32_t d, int64_t n1, int64_t n
     return r == CUDA_SUCCESS;
 }
 
+// Cut a tile into equal boxes of at most 128 tokens (one MMA block of rows or keys): the fewest
+// boxes, at most kMaxBoxes; among equals the split that cuts T before H before W (long rows along
+// W keep the TMA boxes contiguous).  false if the tile has no such split.
+bool choose_boxes(const int32_t tile[3], int32_t nbox[3])
+{
+    int32_t best = kMaxBoxes + 1;
+    for (int32_t n2 = 1; n2 <= kMaxBoxes; ++n2) {
+        if (tile[2] % n2) continue;
+        for (int32_t n1 = 1; n1 * n2 <= kMaxBoxes; ++n1) {
+            if (tile[1] % n1) continue;
+            for (int32_t n0 = 1; n0 * n1 * n2 <= kMaxBoxes; ++n0) {
+                if (tile[0] % n0) continue;
+                const int64_t rows = (int64_t)(tile[0] / n0) * (tile[1] / n1) * (tile[2] / n2);
+                const int32_t boxes = n0 * n1 * n2;
+                // strict <: with n2 outermost and n0 innermost the first split found of a given
+                // size is the one with the fewest cuts along W, then along H
+                if (rows <= kBlockM && boxes < best) {
+                    best = boxes;
+                    nbox[0] = n0; nbox[1] = n1; nbox[2] = n2;
+                }
+            }
+        }
+    }
+    return best <= kMaxBoxes;
+}
+
 int64_t keep_count(int64_t n, double r)
 {
     int64_t k = (int64_t)std::floor(r * (double)n + 0.5);
@@ -237,25 +263,32 @@ int build_list(vorta_plan *p, vorta_plan::WorkList &wl, const std::vector<uint8_
             if (branches[h] & (1u << VORTA_ROUTE_SLIDING)) {
                 for (int32_t qt = 0; qt < g.n_tiles; ++qt) {
                     int32_t q[3] = {qt / (g.nt[2] * g.nt[1]), (qt / g.nt[2]) % g.nt[1], qt % g.nt[2]};
-                    WorkItem w{};
-                    w.mode = MODE_TILES; w.slice = slice;
-                    w.out_slice = by_branch ? VORTA_ROUTE_SLIDING * BH + slice : slice;
-                    // the boxes of the window, then every text key in blocks of bn_tile
-                    w.kv_text = g.text_blocks;
-                    w.kv_count = p->kv_count[qt] + w.kv_text;
-                    w.kv_fast = g.bn_tile == kBlockM ? p->kv_count[g.n_tiles + qt] : 0;
-                    w.kv_begin = qt * g.max_kv_per_tile;
-                    w.kv_len = 0;
-                    int32_t t0 = q[0] * g.tile[0];
+                    // the boxes of the tile that start inside the grid, two per item
+                    int32_t org[kMaxBoxes][3], nb = 0;
                     for (int32_t bx = 0; bx < g.boxes_per_tile; ++bx) {
-                        if (t0 + bx * g.box[0] >= g.T) break;
-                        w.q_org[bx][0] = q[2] * g.tile[2];
-                        w.q_org[bx][1] = q[1] * g.tile[1];
-                        w.q_org[bx][2] = t0 + bx * g.box[0];
-                        w.n_mblk = bx + 1;
+                        const int32_t bb[3] = {bx / (g.nbox[1] * g.nbox[2]), (bx / g.nbox[2]) % g.nbox[1], bx % g.nbox[2]};
+                        const int32_t o3[3] = {q[0] * g.tile[0] + bb[0] * g.box[0], q[1] * g.tile[1] + bb[1] * g.box[1],
+                                               q[2] * g.tile[2] + bb[2] * g.box[2]};
+                        if (o3[0] >= g.T || o3[1] >= g.H || o3[2] >= g.W) continue;
+                        org[nb][0] = o3[2]; org[nb][1] = o3[1]; org[nb][2] = o3[0];  // (w0, h0, t0)
+                        ++nb;
                     }
-                    items.push_back(w);
-                    cost.push_back((double)w.n_mblk * w.kv_count * g.bn_tile / 128.0 + 2.0);
+                    for (int32_t b0 = 0; b0 < nb; b0 += 2) {
+                        WorkItem w{};
+                        w.mode = MODE_TILES; w.slice = slice;
+                        w.out_slice = by_branch ? VORTA_ROUTE_SLIDING * BH + slice : slice;
+                        // the boxes of the window, then every text key in blocks of bn_tile
+                        w.kv_text = g.text_blocks;
+                        w.kv_count = p->kv_count[qt] + w.kv_text;
+                        w.kv_fast = g.bn_tile == kBlockM ? p->kv_count[g.n_tiles + qt] : 0;
+                        w.kv_begin = qt * g.max_kv_per_tile;
+                        w.kv_len = 0;
+                        w.n_mblk = std::min(2, nb - b0);
+                        for (int m = 0; m < w.n_mblk; ++m)
+                            for (int a = 0; a < 3; ++a) w.q_org[m][a] = org[b0 + m][a];
+                        items.push_back(w);
+                        cost.push_back((double)w.n_mblk * w.kv_count * g.bn_tile / 128.0 + 2.0);
+                    }
                 }
                 // the text queries of a sliding head see every key: linear items over rows [L, L + Lt)
                 if (g.Lt > 0)
@@ -491,9 +524,9 @@ int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
     for (int32_t h = 0; h < D.heads; ++h)
         if (D.routes[h] > VORTA_ROUTE_CORESET) return VORTA_ERR_INVALID_ARG;
     if (D.d != 64 && D.d != 128) return VORTA_ERR_UNSUPPORTED;
-    int64_t tile_tokens = (int64_t)D.tile[0] * D.tile[1] * D.tile[2];
-    if (D.tile[0] > 256 || D.tile[1] > 256 || D.tile[2] > 256 || tile_tokens > 256) return VORTA_ERR_UNSUPPORTED;
-    if (tile_tokens > 128 && (D.tile[0] % 2) != 0) return VORTA_ERR_UNSUPPORTED;
+    if (D.tile[0] > 256 || D.tile[1] > 256 || D.tile[2] > 256) return VORTA_ERR_UNSUPPORTED;
+    int32_t nbox[3];
+    if (!choose_boxes(D.tile, nbox)) return VORTA_ERR_UNSUPPORTED;
     if ((int64_t)bucket[0] * bucket[1] * bucket[2] > 32) return VORTA_ERR_UNSUPPORTED;
 
     vorta_plan *p = new (std::nothrow) vorta_plan();
@@ -533,9 +566,12 @@ int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
     g.Ltot = g.L + g.Lt;
     g.Lct = g.Lc + g.Lt;
 
-    // sliding branch blocking
-    g.boxes_per_tile = tile_tokens > 128 ? 2 : 1;
-    g.box[0] = g.tile[0] / g.boxes_per_tile; g.box[1] = g.tile[1]; g.box[2] = g.tile[2];
+    // sliding branch blocking: equal boxes of at most 128 tokens
+    g.boxes_per_tile = nbox[0] * nbox[1] * nbox[2];
+    for (int a = 0; a < 3; ++a) {
+        g.nbox[a] = nbox[a];
+        g.box[a] = g.tile[a] / nbox[a];
+    }
     g.box_rows = g.box[0] * g.box[1] * g.box[2];
     g.bn_tile = (g.box_rows + 15) / 16 * 16;
     int32_t kv_tiles = 1;
@@ -561,18 +597,23 @@ int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
     if (prop.major != 10) { delete p; return VORTA_ERR_UNSUPPORTED; }
     p->sm_count = prop.multiProcessorCount;
 
-    // column masks of the sliding branch: class -> valid columns of a KV box
+    // column masks of the sliding branch: class -> valid columns of a KV box.  Class
+    // 1 + (4 pt + 2 ph + pw) * boxes_per_tile + bx: box bx of a tile the grid cuts on the axes flagged.
     std::vector<uint32_t> masks((size_t)kMaxMasks * 4, 0u);
-    for (int32_t id = 1; id < kMaxMasks; ++id) {
-        int32_t c = id - 1, bx = c & 1, pw = (c >> 1) & 1, ph = (c >> 2) & 1, pt = (c >> 3) & 1;
-        if (bx >= g.boxes_per_tile) continue;
-        int32_t et = pt ? dim[0] - (g.nt[0] - 1) * g.tile[0] : g.tile[0];
-        int32_t vt = std::min(std::max(et - bx * g.box[0], 0), g.box[0]);
-        int32_t vh = ph ? dim[1] - (g.nt[1] - 1) * g.tile[1] : g.tile[1];
-        int32_t vw = pw ? dim[2] - (g.nt[2] - 1) * g.tile[2] : g.tile[2];
-        for (int32_t r = 0; r < g.box_rows; ++r) {
-            int32_t lw = r % g.box[2], lh = (r / g.box[2]) % g.box[1], lt = r / (g.box[2] * g.box[1]);
-            if (lw < vw && lh < vh && lt < vt) masks[(size_t)id * 4 + r / 32] |= 1u << (r % 32);
+    for (int32_t code = 0; code < 8; ++code) {
+        const int32_t part[3] = {(code >> 2) & 1, (code >> 1) & 1, code & 1};
+        for (int32_t bx = 0; bx < g.boxes_per_tile; ++bx) {
+            const int32_t b[3] = {bx / (g.nbox[1] * g.nbox[2]), (bx / g.nbox[2]) % g.nbox[1], bx % g.nbox[2]};
+            int32_t valid[3];
+            for (int a = 0; a < 3; ++a) {
+                const int32_t extent = part[a] ? dim[a] - (g.nt[a] - 1) * g.tile[a] : g.tile[a];
+                valid[a] = std::min(std::max(extent - b[a] * g.box[a], 0), g.box[a]);
+            }
+            const int32_t id = 1 + code * g.boxes_per_tile + bx;
+            for (int32_t r = 0; r < g.box_rows; ++r) {
+                int32_t lw = r % g.box[2], lh = (r / g.box[2]) % g.box[1], lt = r / (g.box[2] * g.box[1]);
+                if (lw < valid[2] && lh < valid[1] && lt < valid[0]) masks[(size_t)id * 4 + r / 32] |= 1u << (r % 32);
+            }
         }
     }
 

@@ -38,7 +38,7 @@ __global__ void block_mask_kernel(Geometry g, uint8_t *__restrict__ bm)
 
 // One thread per query tile: turn its mask row into the list of KV blocks the
 // attention kernel walks (key tiles ascending; a tile of more than 128 tokens
-// gives two boxes; boxes that lie wholly outside the grid are dropped).
+// gives several boxes; boxes that lie wholly outside the grid are dropped).
 __global__ void kv_list_kernel(Geometry g, const uint8_t *__restrict__ bm, KvEntry *__restrict__ list,
                                int32_t *__restrict__ count)
 {
@@ -59,14 +59,17 @@ __global__ void kv_list_kernel(Geometry g, const uint8_t *__restrict__ bm, KvEnt
             bool whole = !pt && !ph && !pw && g.box_rows == g.bn_tile;
             if (whole != (pass == 0)) continue;
             for (int32_t bx = 0; bx < g.boxes_per_tile; ++bx) {
-                int32_t tb = t0 + bx * g.box[0];
-                if (tb >= g.T) break;
+                // box bx of the tile; boxes that start outside the grid are dropped
+                int32_t tb = t0 + (bx / (g.nbox[1] * g.nbox[2])) * g.box[0];
+                int32_t hb = h0 + ((bx / g.nbox[2]) % g.nbox[1]) * g.box[1];
+                int32_t wb = w0 + (bx % g.nbox[2]) * g.box[2];
+                if (tb >= g.T || hb >= g.H || wb >= g.W) continue;
                 if (n < g.max_kv_per_tile) {
                     KvEntry e;
-                    e.w0 = (int16_t)w0;
-                    e.h0 = (int16_t)h0;
+                    e.w0 = (int16_t)wb;
+                    e.h0 = (int16_t)hb;
                     e.t0 = (int16_t)tb;
-                    e.mask_id = whole ? 0 : (uint16_t)(1 + ((pt * 2 + ph) * 2 + pw) * 2 + bx);
+                    e.mask_id = whole ? 0 : (uint16_t)(1 + ((pt * 2 + ph) * 2 + pw) * g.boxes_per_tile + bx);
                     out[n] = e;
                 }
                 ++n;

@@ -20,7 +20,9 @@ enum : int32_t {
 };
 
 constexpr int kBlockM = 128;       // query rows per M-block (one MMA M)
-constexpr int kMaxMasks = 17;      // column-mask classes of the sliding branch (0 = none)
+constexpr int kMaxBoxes = 8;       // a sliding tile is cut into at most this many TMA boxes of <= 128 tokens
+constexpr int kMaxMasks = 1 + 8 * kMaxBoxes;  // column-mask classes of the sliding branch (0 = none):
+                                              // which axes the grid cuts the tile on x which box of the tile
 constexpr int kAttnThreads = 320;  // tcgen05 kernel: 2 control warps + 2 x 4 softmax warps
 constexpr int kBucketTabStride = 34;  // per bucket shape class: token count, centre, 32 token offsets
 
@@ -37,7 +39,8 @@ struct Geometry {
     int32_t text_blocks;                  // KV blocks of bn_tile text keys a sliding item appends: ceil(Lt / bn_tile)
     double ratio;
     // sliding branch blocking: one block = a TMA box of box[0] x box[1] x box[2] tokens
-    int32_t box[3], box_rows, bn_tile, boxes_per_tile, max_kv_per_tile;
+    // (T, H, W order); a tile is nbox[0] x nbox[1] x nbox[2] boxes, numbered bx = (bt * nbox[1] + bh) * nbox[2] + bw
+    int32_t box[3], nbox[3], box_rows, bn_tile, boxes_per_tile, max_kv_per_tile;
 };
 
 // One KV block of a sliding-tile query: origin of its box and its column-mask class.

@@ -80,6 +80,11 @@ def config(name: str) -> Workload:
         # second workload: the MMDiT joint sequence of HunyuanVideo, 256 text tokens after the video tokens
         return Workload(name, (33, 45, 80), 24, 128, (4, 8, 8), (3, 3, 3), 0.5,
                         apportion_routes(24, (0.2, 0.5, 0.3), 2), 2, True, 1, (2, 3, 2), False, 256)
+    if name == "hunyuan-30x45x80-tile6x9x8":
+        # the window the paper prints for HunyuanVideo (18 x 27 x 24 = 3 tiles of 6 x 9 x 8 on the
+        # 30 x 45 x 80 latent, Appendix A.2): 432-token tiles, cut into four boxes of 108
+        return Workload(name, (30, 45, 80), 24, 128, (6, 9, 8), (3, 3, 3), 0.5,
+                        apportion_routes(24, (0.2, 0.5, 0.3), 2), 2, True)
     if name == "hunyuan-720p-3h":
         # profiling case: the HunyuanVideo-720p grid with one head per route, so that a
         # counter capture of one launch stays short while the inputs still exceed L2
@@ -93,7 +98,7 @@ def config(name: str) -> Workload:
 
 
 CONFIG_NAMES = ("tiny", "wan1.3b-480p", "hunyuan-720p", "wan14b-720p")
-JOINT_NAMES = ("hunyuan-720p-text256",)
+JOINT_NAMES = ("hunyuan-720p-text256", "hunyuan-30x45x80-tile6x9x8")  # further workloads bench.py accepts
 PROFILE_NAMES = ("hunyuan-720p-3h", "hunyuan-720p-8c")
 
 

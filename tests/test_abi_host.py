@@ -50,8 +50,9 @@ def host_plan(**kw):
 
 @pytest.mark.parametrize("kw,status", [
     (dict(d=96), vb.VORTA_ERR_UNSUPPORTED),
-    (dict(tile=(4, 9, 8)), vb.VORTA_ERR_UNSUPPORTED),          # 288 tokens
-    (dict(tile=(3, 8, 8)), vb.VORTA_ERR_UNSUPPORTED),          # 192 tokens, odd tT
+    (dict(tile=(16, 16, 8)), vb.VORTA_ERR_UNSUPPORTED),        # 2 048 tokens: more than 8 boxes of 128
+    (dict(tile=(1, 1, 131)), vb.VORTA_ERR_UNSUPPORTED),        # 131 tokens, prime: no equal boxes of <= 128
+    (dict(tile=(1, 257, 1)), vb.VORTA_ERR_UNSUPPORTED),        # an extent over 256
     (dict(bucket=(4, 3, 3)), vb.VORTA_ERR_UNSUPPORTED),        # 36 tokens
     (dict(ratio=0.0), vb.VORTA_ERR_INVALID_ARG),
     (dict(ratio=1.5), vb.VORTA_ERR_INVALID_ARG),
@@ -165,3 +166,18 @@ def test_joint_sequence_accounting_host_only():
     assert info.flops_coreset_head == pytest.approx(4.0 * d * (Lc + Lt) ** 2, rel=1e-12)
     with pytest.raises(vb.VortaError):
         vb.Plan(1, 1, (2, 2, 2), 64, (1, 1, 1), (1, 1, 1), 0.5, (0,), host_only=True, text=-1)
+
+
+@pytest.mark.parametrize("tile,boxes", [((4, 8, 8), 2), ((6, 9, 8), 4), ((3, 9, 8), 2), ((8, 8, 16), 8),
+                                        ((2, 4, 4), 1), ((3, 8, 8), 2), ((4, 9, 8), 3)])
+def test_tiles_are_cut_into_equal_boxes_of_at_most_128_tokens(tile, boxes):
+    """Accepted tiles: the work list has one item per pair of boxes, so its length gives the box count away
+    (host-only plans have no work list: the FLOP accounting, which does not depend on the cut, is checked)."""
+    grid = tuple(2 * t for t in tile)
+    p = vb.Plan(1, 1, grid, 64, tile, (3, 3, 3), 0.5, (1,), host_only=True)
+    info = p.info
+    p.close()
+    M = oracle.sta_token_mask(grid, tile, (3, 3, 3)) if grid[0] * grid[1] * grid[2] <= 4096 else None
+    if M is not None:
+        assert info.flops_sliding_head == pytest.approx(4.0 * 64 * float(M.sum()), rel=1e-12)
+    assert tile[0] * tile[1] * tile[2] <= boxes * 128

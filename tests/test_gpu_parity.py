@@ -45,6 +45,11 @@ def small_workloads():
         # the largest bucket the library takes (32 tokens), cut by the grid on every axis; d = 128 and 64
         W("bucket-32", (5, 9, 10), 2, 128, (2, 4, 4), (3, 3, 3), 0.3, (2, 2), 28, True, 1, (2, 4, 4)),
         W("bucket-32-d64", (6, 6, 7), 2, 64, (2, 4, 4), (3, 3, 3), 0.6, (2, 1), 29, False, 2, (4, 2, 4)),
+        # tiles cut into more than two boxes, along several axes: the 6x9x8 tile of the paper's window
+        # 18x27x24 (four 3x9x4 boxes of 108 tokens), a 3x9x8 tile (odd T: cut along H and W), eight boxes
+        W("tile-6x9x8", (13, 20, 18), 3, 128, (6, 9, 8), (3, 3, 3), 0.5, (1, 0, 2), 71, False),
+        W("tile-3x9x8", (7, 19, 17), 2, 64, (3, 9, 8), (3, 1, 3), 0.5, (1, 1), 72, False, 2),
+        W("tile-8x8x16", (9, 17, 33), 2, 128, (8, 8, 16), (1, 3, 3), 0.5, (1, 1), 73, False),
         # the attention kernel's sub-block pipeline at its shortest: window of one tile, so an item has
         # one KV block: 1 sub-block (32- and 64-token tiles), 2 (128-token tile), 4 (256-token tile)
         W("one-sub-32", (4, 8, 8), 2, 128, (2, 4, 4), (1, 1, 1), 0.5, (1, 1), 41, False),
@@ -461,6 +466,10 @@ def test_config_hunyuan_720p_sampled_rows():
 
 def test_config_wan14b_720p_sampled_rows():
     check_config(workloads.config("wan14b-720p"), 32)
+
+
+def test_config_paper_window_18x27x24_sampled_rows():
+    check_config(workloads.config("hunyuan-30x45x80-tile6x9x8"), 40)
 
 
 def test_config_hunyuan_720p_with_256_text_tokens_sampled_rows():
