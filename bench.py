@@ -36,10 +36,18 @@ METRIC = "routed_attention_effective_tflops"
 UNIT = "TFLOP/s"
 DEFAULT_WORKLOAD = "hunyuan-720p"
 FALLBACK_PEAK_TFLOPS = 1590.0   # used only if MEASURED_PEAKS.json is absent
-# DRAM traffic of the attention kernel: the ncu capture of the three-head profiling case
-# (profiles/attention_sm100_kernel__hunyuan-720p-3h.md) read 441.5 MB and wrote 62.6 MB for 304.1 MB of
-# algorithmic bytes; a launch of another workload is estimated by the same ratio.
-ATTENTION_TRAFFIC_PER_ALGORITHMIC_BYTE = 504.1 / 304.1
+# DRAM traffic of the attention kernels: ncu captures of the three-head profiling case
+# (profiles/attention_kernels__hunyuan-720p-3h.md), 304.1 MB of algorithmic bytes.  The single-CTA
+# kernel alone read 441.5 MB and wrote 62.6 MB; the pair kernel followed by the single-CTA kernel for
+# the sliding head read 553.2 MB and wrote 110.8 MB.  A launch of another workload is estimated by the
+# same ratio.
+# keys: VORTA_KERNEL_* ids (0 the single-CTA kernel, 2 the pair kernel + single-CTA kernel, 1 the debug kernel)
+ATTENTION_TRAFFIC_PER_ALGORITHMIC_BYTE = {0: 504.1 / 304.1, 2: 664.0 / 304.1}
+ATTENTION_KERNEL_NAMES = {
+    0: "attention_sm100_kernel",
+    2: "attention_sm100_pair_kernel (full and core-set heads) then attention_sm100_kernel (sliding heads)",
+    1: "attention_simt_kernel",
+}
 
 
 def attention_algorithmic_bytes(info, wl) -> float:
@@ -347,7 +355,10 @@ def run_ours(args):
     out = None
     if rank == 0:
         achieved = flops_step / (attn_ms * 1e-3) / 1e12
-        roofline = {"bound": "tensor", "kernel": "attention_sm100_kernel", "achieved": achieved,
+        kernel_used = plan.kernel_in_use()
+        traffic_ratio = ATTENTION_TRAFFIC_PER_ALGORITHMIC_BYTE.get(kernel_used)
+        roofline = {"bound": "tensor", "kernel": ATTENTION_KERNEL_NAMES.get(kernel_used, str(kernel_used)),
+                    "achieved": achieved,
                     "peak": pk["bf16"], "unit": UNIT, "frac": achieved / pk["bf16"],
                     "peak_source": f"{pk['source']} burst bf16",
                     "frac_of_sustained": achieved / pk["bf16_sustained"] if pk["bf16_sustained"] else None,
@@ -355,7 +366,7 @@ def run_ours(args):
                     "issued_tflops": info.flops_issued_layer / (attn_ms * 1e-3) / 1e12,
                     "kernel_ms": attn_ms,
                     "algorithmic_bytes": attention_algorithmic_bytes(info, wl),
-                    "traffic": ATTENTION_TRAFFIC_PER_ALGORITHMIC_BYTE * attention_algorithmic_bytes(info, wl),
+                    "traffic": traffic_ratio * attention_algorithmic_bytes(info, wl) if traffic_ratio else None,
                     "traffic_source": "ncu dram bytes of the 3-head capture scaled by algorithmic bytes"}
         gbs = lambda b, ms: (b / (ms * 1e-3) / 1e9) if ms > 0 else None
         stage = {"select_ms": st[0], "gather_ms": st[1], "attention_ms": st[2], "scatter_ms": st[3],

@@ -67,10 +67,15 @@ enum {
                                  (1,2,1) or (1,1,2) at ratio 0.5 are the AP variants of Section 4.2. */
 };
 
-/* Which attention kernel vorta_routed_attention launches. */
+/* Which attention kernel(s) vorta_routed_attention launches. */
 enum {
-    VORTA_KERNEL_TCGEN05 = 0, /* default: persistent TMA + tcgen05/TMEM kernel */
-    VORTA_KERNEL_SIMT = 1     /* slow CUDA-core kernel over the same work lists (debug aid) */
+    VORTA_KERNEL_TCGEN05 = 0, /* one persistent TMA + tcgen05/TMEM kernel, one CTA per SM, for every head */
+    VORTA_KERNEL_SIMT = 1,    /* slow CUDA-core kernel over the same work lists (debug aid) */
+    VORTA_KERNEL_PAIR = 2,    /* two launches: full and core-set heads in the CTA-pair kernel (cta_group::2
+                                 MMAs, K/V shared by an SM pair), sliding heads in the TCGEN05 kernel after it.
+                                 d = 128 and an even number of SMs; VORTA_ERR_UNSUPPORTED otherwise */
+    VORTA_KERNEL_AUTO = 3     /* default: PAIR where it is supported and the full and core-set heads hold
+                                 at least half of the attention work of the call, else TCGEN05 */
 };
 
 typedef struct {
@@ -171,8 +176,12 @@ VORTA_API int vorta_shard_heads(const vorta_plan *plan, int32_t n_ranks, int32_t
  */
 VORTA_API int vorta_plan_block_mask(const vorta_plan *plan, uint8_t *out_host);
 
-/* Select the attention kernel (VORTA_KERNEL_*).  Default VORTA_KERNEL_TCGEN05. */
+/* Select the attention kernel (VORTA_KERNEL_*).  Default VORTA_KERNEL_AUTO. */
 VORTA_API int vorta_plan_set_kernel(vorta_plan *plan, int32_t kernel);
+
+/* The kernel vorta_routed_attention uses with the current routes and selection: what
+ * VORTA_KERNEL_AUTO resolves to, else the selected one.  Negative on a null or host-only plan. */
+VORTA_API int32_t vorta_plan_kernel_in_use(const vorta_plan *plan);
 
 /*
  * Bucketed core-set selection (Section 3.2; Appendix A.1): for every (b, hx)

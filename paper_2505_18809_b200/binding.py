@@ -22,7 +22,7 @@ VORTA_ERR_WORKSPACE, VORTA_ERR_CUDA, VORTA_ERR_TIMEOUT, VORTA_ERR_INTERNAL = 4, 
 VORTA_ROUTE_FULL, VORTA_ROUTE_SLIDING, VORTA_ROUTE_CORESET = 0, 1, 2
 VORTA_PLAN_HOST_ONLY = 1
 VORTA_PLAN_POOL_MERGE = 2
-VORTA_KERNEL_TCGEN05, VORTA_KERNEL_SIMT = 0, 1
+VORTA_KERNEL_TCGEN05, VORTA_KERNEL_SIMT, VORTA_KERNEL_PAIR, VORTA_KERNEL_AUTO = 0, 1, 2, 3
 
 EXPORTS = (
     "vorta_plan_create", "vorta_plan_set_routes", "vorta_plan_destroy", "vorta_plan_info",
@@ -30,7 +30,7 @@ EXPORTS = (
     "vorta_routed_attention", "vorta_routed_attention_host", "vorta_plan_set_profiling",
     "vorta_plan_stage_ms", "vorta_plan_stage_ms_at", "vorta_plan_last_launches", "vorta_device_status",
     "vorta_status_string", "vorta_routed_attention_static", "vorta_plan_device",
-    "vorta_router_gates", "vorta_soft_mixture", "vorta_shard_heads",
+    "vorta_router_gates", "vorta_soft_mixture", "vorta_shard_heads", "vorta_plan_kernel_in_use",
 )
 VORTA_STATIC_WORKSPACE_BYTES = 16 * 1024 * 1024
 
@@ -79,6 +79,8 @@ def lib() -> ctypes.CDLL:
     L.vorta_plan_info.argtypes = [vp, ctypes.POINTER(vorta_plan_info_t)]
     L.vorta_plan_block_mask.argtypes = [vp, vp]
     L.vorta_plan_set_kernel.argtypes = [vp, i32]
+    L.vorta_plan_kernel_in_use.argtypes = [vp]
+    L.vorta_plan_kernel_in_use.restype = i32
     L.vorta_coreset_select.argtypes = [vp, vp, i32, i32, vp, vp, vp]
     L.vorta_routed_attention.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp, ctypes.c_size_t, vp]
     L.vorta_routed_attention_host.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
@@ -155,6 +157,10 @@ def vorta_plan_block_mask(plan: int, n_tiles: int) -> np.ndarray:
 
 def vorta_plan_set_kernel(plan: int, kernel: int) -> None:
     _check(lib().vorta_plan_set_kernel(plan, kernel), "vorta_plan_set_kernel")
+
+
+def vorta_plan_kernel_in_use(plan: int) -> int:
+    return int(lib().vorta_plan_kernel_in_use(plan))
 
 
 def vorta_coreset_select(plan: int, X_ptr: int, Hx: int, dx: int, core_idx_ptr: int,
@@ -292,6 +298,10 @@ class Plan:
 
     def set_kernel(self, kernel: int):
         vorta_plan_set_kernel(self.handle, kernel)
+
+    def kernel_in_use(self) -> int:
+        """The VORTA_KERNEL_* the routed call runs with the current routes (AUTO resolved)."""
+        return vorta_plan_kernel_in_use(self.handle)
 
     def set_profiling(self, on: bool):
         vorta_plan_set_profiling(self.handle, on)

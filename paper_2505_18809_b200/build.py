@@ -9,7 +9,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libvorta.so")
-SOURCES = ("plan.cu", "select_scatter.cu", "attn_simt.cu", "attn_sm100.cu", "static_workspace.cu")
+SOURCES = ("plan.cu", "select_scatter.cu", "attn_simt.cu", "attn_sm100.cu", "attn_sm100_pair.cu",
+           "static_workspace.cu")
 NVCC_FLAGS = ("-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-fvisibility=hidden", "-I" + os.path.join(ROOT, "include"),
               "-I" + CSRC)

@@ -35,6 +35,8 @@ struct vorta_plan {
         WorkItem *d_items = nullptr;
         int32_t *d_cta_begin = nullptr, *d_cta_count = nullptr;
         int32_t n_items = 0;
+        int32_t n_linear = 0;  // items over consecutive rows (full and core-set heads); the others are sliding tiles
+        double linear_share = 0.0;  // their share of the attention work of the list
         int64_t items_cap = 0;
         double flops_issued = 0.0;
         bool built = false;
@@ -59,7 +61,7 @@ struct vorta_plan {
     int32_t *d_core_xslice = nullptr; // same for a shared X with one head
     int32_t *d_status = nullptr;
     double sliding_pairs = 0.0;  // sum over listed tile pairs of valid-token products
-    int32_t kernel = VORTA_KERNEL_TCGEN05;
+    int32_t kernel = VORTA_KERNEL_AUTO;
     // profiling: a ring of event sets, one per call, so that several calls can be
     // enqueued before their stage times are read
     static constexpr int kProfSlots = 64;
@@ -309,34 +311,55 @@ int build_list(vorta_plan *p, vorta_plan::WorkList &wl, const std::vector<uint8_
     }
     wl.flops_issued = issued;
 
-    // longest-processing-time assignment of items to the persistent CTAs
-    const int32_t grid = p->sm_count;
+    // Longest-processing-time assignment of items to the persistent CTAs.  Three lists share the
+    // device arrays: every item over the CTAs (the single-CTA kernel alone); and, for the hybrid
+    // mode, the items over consecutive rows over the CTA PAIRS (pair kernel) followed by the sliding
+    // items over the CTAs (single-CTA kernel beside it).  Items: [0, n) | [n, n + n_linear) |
+    // [n + n_linear, 2n); begin/count: [0, grid) | [grid, grid + grid/2) | [grid + grid/2, 2 grid + grid/2).
+    const int32_t grid = p->sm_count, n_pairs = grid / 2;
     std::vector<int32_t> order(items.size());
     for (size_t i = 0; i < order.size(); ++i) order[i] = (int32_t)i;
     std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return cost[a] > cost[b]; });
-    typedef std::pair<double, int32_t> Load;
-    std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
-    for (int32_t c = 0; c < grid; ++c) heap.push(Load(0.0, c));
-    std::vector<std::vector<int32_t>> per_cta(grid);
-    for (int32_t i : order) {
-        Load l = heap.top();
-        heap.pop();
-        per_cta[l.second].push_back(i);
-        heap.push(Load(l.first + cost[i], l.second));
-    }
     std::vector<WorkItem> sorted;
-    sorted.reserve(items.size());
-    std::vector<int32_t> begin(grid), count(grid);
-    for (int32_t c = 0; c < grid; ++c) {
-        begin[c] = (int32_t)sorted.size();
-        count[c] = (int32_t)per_cta[c].size();
-        for (int32_t i : per_cta[c]) sorted.push_back(items[i]);
+    sorted.reserve(2 * items.size());
+    const int32_t n_bins = 2 * grid + n_pairs;
+    std::vector<int32_t> begin(n_bins), count(n_bins);
+    // which: 0 every item, 1 the linear ones, 2 the sliding ones
+    auto assign = [&](int32_t bins, int32_t first_bin, int which) {
+        typedef std::pair<double, int32_t> Load;
+        std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
+        for (int32_t c = 0; c < bins; ++c) heap.push(Load(0.0, c));
+        std::vector<std::vector<int32_t>> per_bin(bins);
+        for (int32_t i : order) {
+            const bool tiles = items[i].mode == MODE_TILES;
+            if ((which == 1 && tiles) || (which == 2 && !tiles)) continue;
+            Load l = heap.top();
+            heap.pop();
+            per_bin[l.second].push_back(i);
+            heap.push(Load(l.first + cost[i], l.second));
+        }
+        const size_t base = sorted.size();
+        for (int32_t c = 0; c < bins; ++c) {
+            begin[first_bin + c] = (int32_t)(sorted.size() - base);
+            count[first_bin + c] = (int32_t)per_bin[c].size();
+            for (int32_t i : per_bin[c]) sorted.push_back(items[i]);
+        }
+        return (int32_t)(sorted.size() - base);
+    };
+    assign(grid, 0, 0);
+    wl.n_linear = assign(n_pairs, grid, 1);
+    assign(grid, grid + n_pairs, 2);
+    double cost_all = 0.0, cost_linear = 0.0;
+    for (size_t i = 0; i < items.size(); ++i) {
+        cost_all += cost[i];
+        if (items[i].mode != MODE_TILES) cost_linear += cost[i];
     }
-    wl.n_items = (int32_t)sorted.size();
+    wl.linear_share = cost_all > 0.0 ? cost_linear / cost_all : 0.0;
+    wl.n_items = (int32_t)items.size();
 
     if (!wl.d_cta_begin &&
-        (cudaMalloc(&wl.d_cta_begin, sizeof(int32_t) * grid) != cudaSuccess ||
-         cudaMalloc(&wl.d_cta_count, sizeof(int32_t) * grid) != cudaSuccess))
+        (cudaMalloc(&wl.d_cta_begin, sizeof(int32_t) * n_bins) != cudaSuccess ||
+         cudaMalloc(&wl.d_cta_count, sizeof(int32_t) * n_bins) != cudaSuccess))
         return VORTA_ERR_CUDA;
     if ((int64_t)sorted.size() > wl.items_cap) {
         cudaFree(wl.d_items);
@@ -349,8 +372,8 @@ int build_list(vorta_plan *p, vorta_plan::WorkList &wl, const std::vector<uint8_
     if (!sorted.empty() &&
         cudaMemcpy(wl.d_items, sorted.data(), sizeof(WorkItem) * sorted.size(), cudaMemcpyHostToDevice) != cudaSuccess)
         return VORTA_ERR_CUDA;
-    if (cudaMemcpy(wl.d_cta_begin, begin.data(), sizeof(int32_t) * grid, cudaMemcpyHostToDevice) != cudaSuccess ||
-        cudaMemcpy(wl.d_cta_count, count.data(), sizeof(int32_t) * grid, cudaMemcpyHostToDevice) != cudaSuccess)
+    if (cudaMemcpy(wl.d_cta_begin, begin.data(), sizeof(int32_t) * n_bins, cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(wl.d_cta_count, count.data(), sizeof(int32_t) * n_bins, cudaMemcpyHostToDevice) != cudaSuccess)
         return VORTA_ERR_CUDA;
     wl.built = true;
     return VORTA_OK;
@@ -475,6 +498,18 @@ struct DeviceGuard {
 bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 }  // namespace
+
+// the pair kernel is built for d = 128 and needs the SMs in pairs
+static bool pair_supported(const vorta_plan *p) { return p->g.d == 128 && (p->sm_count & 1) == 0 && p->sm_count >= 2; }
+
+// The kernel a call over `wl` runs: VORTA_KERNEL_AUTO takes the pair kernel (with the single-CTA
+// kernel for the sliding heads) where the full and core-set heads hold at least half of the work;
+// measured on a B200, that split is faster from there on and slower below.
+static int32_t resolve_kernel(const vorta_plan *p, const vorta_plan::WorkList &wl)
+{
+    if (p->kernel != VORTA_KERNEL_AUTO) return p->kernel;
+    return pair_supported(p) && wl.linear_share >= 0.5 ? VORTA_KERNEL_PAIR : VORTA_KERNEL_TCGEN05;
+}
 
 #ifdef VORTA_TRACE
 static long long *g_vorta_trace = nullptr;
@@ -665,6 +700,7 @@ int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
     p->kv_count.resize(2 * (size_t)g.n_tiles);
     ok = ok && cudaMemcpy(p->kv_count.data(), p->d_kv_count, sizeof(int32_t) * 2 * g.n_tiles, cudaMemcpyDeviceToHost) == cudaSuccess;
     ok = ok && attention_sm100_prepare() == cudaSuccess;
+    ok = ok && attention_sm100_pair_prepare() == cudaSuccess;
     if (!ok) { cudaGetLastError(); free_device(p); delete p; return VORTA_ERR_CUDA; }
     // self-check: the lists must hold exactly the blocks the window arithmetic predicts
     for (int32_t qt = 0; qt < g.n_tiles; ++qt)
@@ -779,9 +815,16 @@ int vorta_plan_block_mask(const vorta_plan *p, uint8_t *out_host)
 
 int vorta_plan_set_kernel(vorta_plan *p, int32_t kernel)
 {
-    if (!p || (kernel != VORTA_KERNEL_TCGEN05 && kernel != VORTA_KERNEL_SIMT)) return VORTA_ERR_INVALID_ARG;
+    if (!p || kernel < VORTA_KERNEL_TCGEN05 || kernel > VORTA_KERNEL_AUTO) return VORTA_ERR_INVALID_ARG;
+    if (kernel == VORTA_KERNEL_PAIR && !pair_supported(p)) return VORTA_ERR_UNSUPPORTED;
     p->kernel = kernel;
     return VORTA_OK;
+}
+
+int32_t vorta_plan_kernel_in_use(const vorta_plan *p)
+{
+    if (!p || p->host_only) return -1;
+    return resolve_kernel(p, p->routed);
 }
 
 int vorta_plan_set_profiling(vorta_plan *p, int32_t on)
@@ -869,7 +912,21 @@ static int run_layer(const vorta_plan *p, const vorta_plan::WorkList &wl, int32_
 
     AttnMaps maps;
     std::memset(&maps, 0, sizeof(maps));
-    if (p->kernel == VORTA_KERNEL_TCGEN05) {
+    // Hybrid mode: the items over consecutive rows (full and core-set heads) go to the pair kernel,
+    // the sliding items to the single-CTA kernel, each with its own lists behind the common ones.
+    const int32_t kernel = resolve_kernel(p, wl);
+    const bool pair = kernel == VORTA_KERNEL_PAIR;
+    AttnParams prm_pair = prm, prm_tiles = prm;
+    if (pair) {
+        const int32_t n_pairs = p->sm_count / 2;
+        prm_pair.items = wl.d_items + wl.n_items;
+        prm_pair.cta_begin = wl.d_cta_begin + p->sm_count;
+        prm_pair.cta_count = wl.d_cta_count + p->sm_count;
+        prm_tiles.items = wl.d_items + wl.n_items + wl.n_linear;
+        prm_tiles.cta_begin = wl.d_cta_begin + p->sm_count + n_pairs;
+        prm_tiles.cta_count = wl.d_cta_count + p->sm_count + n_pairs;
+    }
+    if (kernel == VORTA_KERNEL_TCGEN05 || pair) {
         const int64_t BH = (int64_t)g.B * g.heads;
         bool ok = true;
         const void *src[3] = {q, k, v};
@@ -893,6 +950,13 @@ static int run_layer(const vorta_plan *p, const vorta_plan::WorkList &wl, int32_
         for (int t = 0; t < 3 && ok; ++t) {
             if (n_prob) ok = ok && make_map(&dst[t][MODE_COMPACT], csrc[t], g.d, g.Lct, 1, 1, n_prob, kBlockM, 1, 1);
             else dst[t][MODE_COMPACT] = dst[t][MODE_LINEAR];
+        }
+        if (pair) {
+            // K in boxes of 64 rows: the first or second half of a block's keys for each CTA of a pair
+            ok = ok && make_map(&maps.k_half[MODE_LINEAR], k, g.d, g.Ltot, 1, 1, BH, kBlockM / 2, 1, 1);
+            maps.k_half[MODE_TILES] = maps.k_half[MODE_LINEAR];  // unused: sliding items run in the other kernel
+            if (n_prob) ok = ok && make_map(&maps.k_half[MODE_COMPACT], Kc, g.d, g.Lct, 1, 1, n_prob, kBlockM / 2, 1, 1);
+            else maps.k_half[MODE_COMPACT] = maps.k_half[MODE_LINEAR];
         }
         if (!ok) return VORTA_ERR_CUDA;
     }
@@ -929,10 +993,27 @@ static int run_layer(const vorta_plan *p, const vorta_plan::WorkList &wl, int32_
     }
     mark(2);
     if (wl.n_items > 0) {
-        e = p->kernel == VORTA_KERNEL_TCGEN05 ? launch_attention_sm100(prm, maps, p->sm_count, s)
-                                              : launch_attention_simt(prm, wl.n_items, s);
-        if (e != cudaSuccess) return VORTA_ERR_CUDA;
-        ++launches;
+        if (pair) {
+            // One after the other on the caller's stream.  (Run side by side on two queues, so that the
+            // second kernel's CTAs fill the SMs the first one's tail leaves, the single-CTA kernel's
+            // bounded waits expired at hunyuan-720p: CTAs of a cluster kernel and of a plain kernel
+            // are not mixed on the GPU here.)
+            if (wl.n_linear > 0) {
+                e = launch_attention_sm100_pair(prm_pair, maps, p->sm_count, s);
+                if (e != cudaSuccess) return VORTA_ERR_CUDA;
+                ++launches;
+            }
+            if (wl.n_items - wl.n_linear > 0) {
+                e = launch_attention_sm100(prm_tiles, maps, p->sm_count, s);
+                if (e != cudaSuccess) return VORTA_ERR_CUDA;
+                ++launches;
+            }
+        } else {
+            e = kernel == VORTA_KERNEL_TCGEN05 ? launch_attention_sm100(prm, maps, p->sm_count, s)
+                                                  : launch_attention_simt(prm, wl.n_items, s);
+            if (e != cudaSuccess) return VORTA_ERR_CUDA;
+            ++launches;
+        }
     }
     mark(3);
     if (n_prob) {

@@ -70,6 +70,7 @@ static_assert(sizeof(WorkItem) == 64, "WorkItem must stay 64 bytes");
 struct AttnMaps {
     CUtensorMap q[3], k[3], v[3];  // indexed by mode
     CUtensorMap kt, vt;            // text rows [L, L + Lt) of K and V in boxes of bn_tile rows (sliding items)
+    CUtensorMap k_half[3];         // pair kernel: K of the linear modes in boxes of 64 rows
 };
 
 struct AttnParams {
@@ -115,6 +116,9 @@ cudaError_t launch_attention_simt(const AttnParams &p, int32_t n_items, cudaStre
 cudaError_t launch_attention_sm100(const AttnParams &p, const AttnMaps &maps, int32_t grid,
                                    cudaStream_t s);
 cudaError_t attention_sm100_prepare();  // opt in to the kernel's dynamic shared memory
+cudaError_t launch_attention_sm100_pair(const AttnParams &p, const AttnMaps &maps, int32_t grid,
+                                        cudaStream_t s);  // p's work lists are indexed by CTA pair
+cudaError_t attention_sm100_pair_prepare();
 
 // Row r of an M-/KV-block -> token id; false if the row lies outside the grid/sequence.
 __host__ __device__ inline bool block_row_token(const Geometry &g, int32_t mode, const int32_t org[3],

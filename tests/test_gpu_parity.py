@@ -65,8 +65,23 @@ def small_workloads():
     ]
 
 
+KERNELS = [vb.VORTA_KERNEL_SIMT, vb.VORTA_KERNEL_TCGEN05, vb.VORTA_KERNEL_PAIR]
+KERNEL_IDS = ["simt", "tcgen05", "pair"]
+
+
+def set_kernel_or_skip(plan, kernel):
+    """The pair kernel takes d = 128 and boxes that halve along their slowest axis; other plans refuse it."""
+    try:
+        plan.set_kernel(kernel)
+    except vb.VortaError as e:
+        if kernel == vb.VORTA_KERNEL_PAIR and e.status == vb.VORTA_ERR_UNSUPPORTED:
+            plan.close()
+            pytest.skip("plan not eligible for the pair kernel")
+        raise
+
+
 def run_layer(plan, wl, Q, K, V, kernel):
-    plan.set_kernel(kernel)
+    set_kernel_or_skip(plan, kernel)
     O = torch.full_like(Q, float("nan"))
     plan.routed_attention(Q, K, V, O)
     assert plan.device_status() == 0
@@ -121,7 +136,7 @@ def test_coreset_select_other_feature_width_and_ties():
 
 
 # --------------------------------------------------------------------------- attention, small
-@pytest.mark.parametrize("kernel", [vb.VORTA_KERNEL_SIMT, vb.VORTA_KERNEL_TCGEN05], ids=["simt", "tcgen05"])
+@pytest.mark.parametrize("kernel", KERNELS, ids=KERNEL_IDS)
 @pytest.mark.parametrize("wl", small_workloads(), ids=lambda w: w.name)
 def test_routed_attention_small_all_rows(wl, kernel):
     Q, K, V = workloads.make_qkv(wl, DEV)
@@ -187,12 +202,13 @@ def test_longest_axis_the_library_takes(grid, tile, bucket):
         vb.Plan(1, 1, (1, 1, 32768), 64, tile, (3, 3, 3), 0.5, (0,), host_only=True)
 
 
-def test_pruned_rows_copy_their_centre_and_reruns_are_bitwise_equal():
+@pytest.mark.parametrize("kernel", [vb.VORTA_KERNEL_TCGEN05, vb.VORTA_KERNEL_PAIR], ids=["tcgen05", "pair"])
+def test_pruned_rows_copy_their_centre_and_reruns_are_bitwise_equal(kernel):
     wl = small_workloads()[2]
     Q, K, V = workloads.make_qkv(wl, DEV)
     p = vb.Plan.from_workload(wl)
-    O1 = run_layer(p, wl, Q, K, V, vb.VORTA_KERNEL_TCGEN05)
-    O2 = run_layer(p, wl, Q, K, V, vb.VORTA_KERNEL_TCGEN05)
+    O1 = run_layer(p, wl, Q, K, V, kernel)
+    O2 = run_layer(p, wl, Q, K, V, kernel)
     assert torch.equal(O1.view(torch.int16), O2.view(torch.int16))
     h = wl.routes.index(2)
     core, src = oracle.coreset_select(wl.grid, wl.bucket, float(np.float32(wl.ratio)), head_f64(K, 0, h))
@@ -224,18 +240,53 @@ def test_routes_can_change_between_steps_and_shared_selection_features():
     p.close()
 
 
-def test_growing_scores_exercise_the_lazy_rescale():
+def test_default_kernel_choice_follows_the_routes():
+    """VORTA_KERNEL_AUTO: the pair kernel where full and core-set heads hold at least half of the
+    work, the single-CTA kernel otherwise; the choice is remade when the routes change."""
+    wl = Workload("auto", (6, 16, 16), 3, 128, (2, 8, 8), (3, 3, 3), 0.5, (0, 1, 2), 64, False)
+    Q, K, V = workloads.make_qkv(wl, DEV)
+    p = vb.Plan.from_workload(wl)
+    for routes, want_kernel in [((0, 1, 0), vb.VORTA_KERNEL_PAIR), ((1, 1, 1), vb.VORTA_KERNEL_TCGEN05),
+                                ((2, 2, 0), vb.VORTA_KERNEL_PAIR), ((1, 1, 2), vb.VORTA_KERNEL_TCGEN05),
+                                ((0, 1, 2), None)]:   # near the boundary: either choice
+        p.set_routes(routes)
+        if want_kernel is None:
+            want_kernel = p.kernel_in_use()
+        assert p.kernel_in_use() == want_kernel, routes
+        O = torch.full_like(Q, float("nan"))
+        p.routed_attention(Q, K, V, O)
+        assert p.device_status() == 0
+        assert p.last_launches() == (2 if want_kernel == vb.VORTA_KERNEL_PAIR and 1 in routes else 1) + (3 if 2 in routes else 0)
+        for h in range(wl.heads):
+            want = oracle_head_rows(wl, Q, K, V, 0, h, None, route=routes[h])
+            assert_close(O[0, h], want, f"routes {routes} h{h}")
+    p.set_kernel(vb.VORTA_KERNEL_TCGEN05)
+    assert p.kernel_in_use() == vb.VORTA_KERNEL_TCGEN05
+    p.close()
+    # d = 64: the pair kernel is refused and never chosen
+    p64 = vb.Plan(1, 2, (4, 8, 8), 64, (2, 4, 4), (3, 3, 3), 0.5, (0, 0))
+    assert p64.kernel_in_use() == vb.VORTA_KERNEL_TCGEN05
+    with pytest.raises(vb.VortaError):
+        p64.set_kernel(vb.VORTA_KERNEL_PAIR)
+    p64.close()
+
+
+@pytest.mark.parametrize("kernel", [vb.VORTA_KERNEL_TCGEN05, vb.VORTA_KERNEL_PAIR], ids=["tcgen05", "pair"])
+def test_growing_scores_exercise_the_lazy_rescale(kernel):
     """Keys whose norm grows along the sequence: the running maximum keeps rising, by less than
-    the rescale threshold (P above 1 for a while) and by far more (O rescaled in place)."""
+    the rescale threshold (P above 1 for a while) and by far more (O rescaled in place).  In the
+    pair kernel the steps fall on blocks of all three softmax groups (shared reference maximum)."""
     wl = Workload("ramp", (4, 16, 32), 2, 128, (2, 8, 8), (3, 3, 3), 0.5, (0, 1), 41, False)
     Q, K, V = workloads.make_qkv(wl, DEV)
     ramp = torch.ones(wl.L, device=DEV)
     ramp[256:] = 2.0        # a few log2 units above the first blocks
     ramp[768:] = 4.0
     ramp[1280:] = 24.0      # tens of log2 units above everything before
+    ramp[1408:] = 96.0      # and again one and two blocks later: consecutive raises by different groups
+    ramp[1536:] = 400.0
     K = (K.float() * ramp[None, None, :, None]).to(torch.bfloat16).contiguous()
     p = vb.Plan.from_workload(wl)
-    O = run_layer(p, wl, Q, K, V, vb.VORTA_KERNEL_TCGEN05)
+    O = run_layer(p, wl, Q, K, V, kernel)
     for h in range(wl.heads):
         want = oracle_head_rows(wl, Q, K, V, 0, h, None)
         assert_close(O[0, h], want, f"ramp h{h}")
@@ -260,12 +311,12 @@ def test_router_gates_and_routes_match_the_oracle():
     assert set(r.tolist()) == {0, 1, 2}            # the random heads spread over all three branches
 
 
-@pytest.mark.parametrize("kernel", [vb.VORTA_KERNEL_SIMT, vb.VORTA_KERNEL_TCGEN05], ids=["simt", "tcgen05"])
+@pytest.mark.parametrize("kernel", KERNELS, ids=KERNEL_IDS)
 def test_soft_mixture_matches_the_oracle(kernel):
     wl = Workload("mix", (6, 10, 12), 3, 128, (2, 4, 4), (3, 3, 3), 0.5, (0, 1, 2), 61, False)
     Q, K, V = workloads.make_qkv(wl, DEV)
     p = vb.Plan.from_workload(wl)
-    p.set_kernel(kernel)
+    set_kernel_or_skip(p, kernel)
     gates = torch.tensor([[0.2, 0.5, 0.3], [1.0, 0.0, 0.0], [0.05, 0.15, 0.8]], dtype=torch.float32, device=DEV)
     O = torch.full_like(Q, float("nan"))
     p.soft_mixture(Q, K, V, gates, O)
@@ -283,7 +334,7 @@ def test_soft_mixture_matches_the_oracle(kernel):
     p.close()
 
 
-@pytest.mark.parametrize("kernel", [vb.VORTA_KERNEL_SIMT, vb.VORTA_KERNEL_TCGEN05], ids=["simt", "tcgen05"])
+@pytest.mark.parametrize("kernel", KERNELS, ids=KERNEL_IDS)
 @pytest.mark.parametrize("bucket,ratio", [((2, 3, 2), 0.5), ((2, 1, 1), 0.5), ((1, 2, 1), 0.5), ((1, 1, 2), 0.5),
                                           ((2, 3, 2), 0.25)])
 def test_merge_into_centre_and_average_pool_variants(bucket, ratio, kernel):
@@ -377,7 +428,7 @@ def joint_workloads():
     ]
 
 
-@pytest.mark.parametrize("kernel", [vb.VORTA_KERNEL_SIMT, vb.VORTA_KERNEL_TCGEN05], ids=["simt", "tcgen05"])
+@pytest.mark.parametrize("kernel", KERNELS, ids=KERNEL_IDS)
 @pytest.mark.parametrize("wl", joint_workloads(), ids=lambda w: w.name)
 def test_joint_sequence_all_rows(wl, kernel):
     """Video tokens followed by text tokens: text keys visible to every query, text queries see
@@ -425,9 +476,13 @@ def test_joint_sequence_host_entry_and_soft_mixture():
 
 
 # --------------------------------------------------------------------------- the named configurations
-def check_config(wl, rows_per_head, kernels=(vb.VORTA_KERNEL_TCGEN05,)):
+def check_config(wl, rows_per_head, kernels=(vb.VORTA_KERNEL_AUTO, vb.VORTA_KERNEL_TCGEN05), expect_in_use=None):
+    """A whole configuration: integer stages in full, outputs on all or on sampled rows, for the
+    default kernel choice (what bench.py times) and for the kernels named."""
     Q, K, V = workloads.make_qkv(wl, DEV)
     p = vb.Plan.from_workload(wl)
+    if expect_in_use is not None:
+        assert p.kernel_in_use() == expect_in_use
     # integer stages in full: block mask, indices and scatter map of every core-set head
     assert np.array_equal(p.block_mask(), oracle.sta_block_mask(wl.grid, wl.tile, wl.window))
     core_heads = [h for h in range(wl.heads) if wl.routes[h] == 2]
@@ -438,34 +493,42 @@ def check_config(wl, rows_per_head, kernels=(vb.VORTA_KERNEL_TCGEN05,)):
             assert np.array_equal(core[0, h].cpu().numpy(), c), h
             assert np.array_equal(src[0, h].cpu().numpy(), s), h
         del core, src
+    outs = []
     for kernel in kernels:
         O = run_layer(p, wl, Q, K, V, kernel)
         assert bool(torch.isfinite(O.float()).all())
-        worst = 0.0
-        for h in range(wl.heads):
-            rows = None if rows_per_head is None else sample_rows(wl, rows_per_head, 1000 + h)
-            want = oracle_head_rows(wl, Q, K, V, 0, h, rows)
+        outs.append(O)
+    worst = [0.0] * len(kernels)
+    for h in range(wl.heads):
+        rows = None if rows_per_head is None else sample_rows(wl, rows_per_head, 1000 + h)
+        want = oracle_head_rows(wl, Q, K, V, 0, h, rows)
+        for i, (kernel, O) in enumerate(zip(kernels, outs)):
             got = O[0, h] if rows is None else O[0, h][torch.from_numpy(rows).to(DEV)]
             mx, _ = assert_close(got, want, f"{wl.name} h{h} route {wl.routes[h]} kernel {kernel}")
-            worst = max(worst, mx)
-        print(f"{wl.name} kernel {kernel}: worst max-abs {worst:.3e}")
+            worst[i] = max(worst[i], mx)
+    for kernel, w in zip(kernels, worst):
+        print(f"{wl.name} kernel {kernel}: worst max-abs {w:.3e}")
     p.close()
 
 
 def test_config_tiny_all_rows():
-    check_config(workloads.config("tiny"), None, (vb.VORTA_KERNEL_SIMT, vb.VORTA_KERNEL_TCGEN05))
+    check_config(workloads.config("tiny"), None, (vb.VORTA_KERNEL_AUTO, vb.VORTA_KERNEL_SIMT, vb.VORTA_KERNEL_TCGEN05),
+                 expect_in_use=vb.VORTA_KERNEL_TCGEN05)  # d = 64: the pair kernel does not apply
 
 
 def test_config_wan13b_480p_sampled_rows():
-    check_config(workloads.config("wan1.3b-480p"), 96, (vb.VORTA_KERNEL_SIMT, vb.VORTA_KERNEL_TCGEN05))
+    check_config(workloads.config("wan1.3b-480p"), 96, (vb.VORTA_KERNEL_AUTO, vb.VORTA_KERNEL_SIMT, vb.VORTA_KERNEL_TCGEN05),
+                 expect_in_use=vb.VORTA_KERNEL_PAIR)
 
 
 def test_config_hunyuan_720p_sampled_rows():
-    check_config(workloads.config("hunyuan-720p"), 48)
+    check_config(workloads.config("hunyuan-720p"), 48, expect_in_use=vb.VORTA_KERNEL_PAIR)
 
 
 def test_config_wan14b_720p_sampled_rows():
-    check_config(workloads.config("wan14b-720p"), 32)
+    # sliding heads hold most of the work: the single-CTA kernel alone; the pair kernel is checked too
+    check_config(workloads.config("wan14b-720p"), 32, (vb.VORTA_KERNEL_AUTO, vb.VORTA_KERNEL_PAIR),
+                 expect_in_use=vb.VORTA_KERNEL_TCGEN05)
 
 
 def test_config_paper_window_18x27x24_sampled_rows():
