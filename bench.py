@@ -36,13 +36,13 @@ METRIC = "routed_attention_effective_tflops"
 UNIT = "TFLOP/s"
 DEFAULT_WORKLOAD = "hunyuan-720p"
 FALLBACK_PEAK_TFLOPS = 1590.0   # used only if MEASURED_PEAKS.json is absent
-# DRAM traffic of the attention kernels: ncu captures of the three-head profiling case
-# (profiles/attention_kernels__hunyuan-720p-3h.md), 304.1 MB of algorithmic bytes.  The single-CTA
-# kernel alone read 441.5 MB and wrote 62.6 MB; the pair kernel followed by the single-CTA kernel for
-# the sliding head read 553.2 MB and wrote 110.8 MB.  A launch of another workload is estimated by the
-# same ratio.
-# keys: VORTA_KERNEL_* ids (0 the single-CTA kernel, 2 the pair kernel + single-CTA kernel, 1 the debug kernel)
-ATTENTION_TRAFFIC_PER_ALGORITHMIC_BYTE = {0: 504.1 / 304.1, 2: 664.0 / 304.1}
+# DRAM traffic of the attention kernels per algorithmic byte, from ncu captures of the three-head
+# profiling case (profiles/): the single-CTA kernel over all three heads read 441.5 MB and wrote 62.6 MB
+# for 304.1 MB of algorithmic bytes; the pair kernel over the full and the core-set head read 461.4 MB
+# and wrote 99.2 MB for 182.5 MB.  A launch of another workload is estimated by the same ratio.
+ATTENTION_TRAFFIC_PER_ALGORITHMIC_BYTE = 504.1 / 304.1
+PAIR_KERNEL_TRAFFIC_PER_ALGORITHMIC_BYTE = 560.6 / 182.5
+# VORTA_KERNEL_* id -> what the attention stage launches
 ATTENTION_KERNEL_NAMES = {
     0: "attention_sm100_kernel",
     2: "attention_sm100_pair_kernel (full and core-set heads) then attention_sm100_kernel (sliding heads)",
@@ -350,24 +350,49 @@ def run_ours(args):
         stages = [plan.stage_ms(i) for i in range(n_hist)]
     st = [sum(s[i] for s in stages) / n_hist for i in range(4)]
     attn_ms = st[2]
+    # the attention stage by launch: [pair kernel or the only kernel, single-CTA kernel after the pair kernel]
+    by_launch = [attn_ms, 0.0]
+    if not args.mixture:
+        parts = [plan.attention_ms(i) for i in range(n_hist)]
+        by_launch = [sum(x[i] for x in parts) / n_hist for i in range(2)]
     n_core = info.n_coreset * wl.B
 
     out = None
     if rank == 0:
-        achieved = flops_step / (attn_ms * 1e-3) / 1e12
         kernel_used = plan.kernel_in_use()
-        traffic_ratio = ATTENTION_TRAFFIC_PER_ALGORITHMIC_BYTE.get(kernel_used)
-        roofline = {"bound": "tensor", "kernel": ATTENTION_KERNEL_NAMES.get(kernel_used, str(kernel_used)),
-                    "achieved": achieved,
+        stage_tflops = flops_step / (attn_ms * 1e-3) / 1e12
+        row = wl.d * 2
+        two = by_launch[1] > 0.0
+        if two:
+            # Two attention launches: the dominant kernel is the pair kernel (full and core-set heads);
+            # its own FLOPs and bytes over its own time.  The whole stage is reported beside it.
+            name = "attention_sm100_pair_kernel"
+            k_flops = wl.B * (info.n_full * info.flops_full_head + info.n_coreset * info.flops_coreset_head)
+            k_ms = by_launch[0]
+            k_bytes = wl.B * (info.n_full * 4.0 * info.L * row + info.n_coreset * 4.0 * info.Lc * row)
+            k_ratio = PAIR_KERNEL_TRAFFIC_PER_ALGORITHMIC_BYTE
+        else:
+            name = ATTENTION_KERNEL_NAMES.get(kernel_used, str(kernel_used))
+            if kernel_used == 2 and not args.mixture:   # one launch: only one kind of head is present
+                name = "attention_sm100_pair_kernel" if info.n_sliding == 0 else "attention_sm100_kernel"
+            k_flops, k_ms, k_bytes = flops_step, attn_ms, attention_algorithmic_bytes(info, wl)
+            k_ratio = (PAIR_KERNEL_TRAFFIC_PER_ALGORITHMIC_BYTE if name == "attention_sm100_pair_kernel"
+                       else ATTENTION_TRAFFIC_PER_ALGORITHMIC_BYTE)
+        achieved = k_flops / (k_ms * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "kernel": name, "achieved": achieved,
                     "peak": pk["bf16"], "unit": UNIT, "frac": achieved / pk["bf16"],
                     "peak_source": f"{pk['source']} burst bf16",
                     "frac_of_sustained": achieved / pk["bf16_sustained"] if pk["bf16_sustained"] else None,
                     "frac_of_nominal_2250": achieved / 2250.0,
-                    "issued_tflops": info.flops_issued_layer / (attn_ms * 1e-3) / 1e12,
-                    "kernel_ms": attn_ms,
-                    "algorithmic_bytes": attention_algorithmic_bytes(info, wl),
-                    "traffic": traffic_ratio * attention_algorithmic_bytes(info, wl) if traffic_ratio else None,
-                    "traffic_source": "ncu dram bytes of the 3-head capture scaled by algorithmic bytes"}
+                    "kernel_ms": k_ms, "kernel_algorithmic_tflop": k_flops / 1e12,
+                    "algorithmic_bytes": k_bytes,
+                    "traffic": k_ratio * k_bytes if not args.mixture else None,
+                    "traffic_source": "ncu dram bytes of this kernel in the 3-head capture, scaled by algorithmic bytes",
+                    "attention_stage": {"kernels": ATTENTION_KERNEL_NAMES.get(kernel_used, str(kernel_used)),
+                                        "ms_by_launch": by_launch, "ms": attn_ms, "tflops": stage_tflops,
+                                        "frac": stage_tflops / pk["bf16"],
+                                        "frac_of_sustained": stage_tflops / pk["bf16_sustained"] if pk["bf16_sustained"] else None,
+                                        "issued_tflops": info.flops_issued_layer / (attn_ms * 1e-3) / 1e12}}
         gbs = lambda b, ms: (b / (ms * 1e-3) / 1e9) if ms > 0 else None
         stage = {"select_ms": st[0], "gather_ms": st[1], "attention_ms": st[2], "scatter_ms": st[3],
                  "select_gbs": gbs(n_core * info.select_bytes_head, st[0]),

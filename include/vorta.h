@@ -75,7 +75,7 @@ enum {
                                  MMAs, K/V shared by an SM pair), sliding heads in the TCGEN05 kernel after it.
                                  d = 128 and an even number of SMs; VORTA_ERR_UNSUPPORTED otherwise */
     VORTA_KERNEL_AUTO = 3     /* default: PAIR where it is supported and the full and core-set heads hold
-                                 at least half of the attention work of the call, else TCGEN05 */
+                                 at least 60 % of the attention work of the call, else TCGEN05 */
 };
 
 typedef struct {
@@ -305,6 +305,10 @@ VORTA_API int vorta_plan_stage_ms(const vorta_plan *plan, float ms[4]);
 /* The same for an earlier call: calls_back = 0 is the last profiled call, 1 the one
  * before it, ... up to 63.  VORTA_ERR_INVALID_ARG if that call was never made. */
 VORTA_API int vorta_plan_stage_ms_at(const vorta_plan *plan, int32_t calls_back, float ms[4]);
+/* The attention stage of that call by launch: ms[0] the first attention kernel (the pair kernel
+ * under VORTA_KERNEL_PAIR, else the only one), ms[1] the single-CTA kernel that follows the pair
+ * kernel for the sliding heads (0 if there was one launch). */
+VORTA_API int vorta_plan_attention_ms_at(const vorta_plan *plan, int32_t calls_back, float ms[2]);
 
 /* Number of kernels the last vorta_routed_attention call launched. */
 VORTA_API int vorta_plan_last_launches(const vorta_plan *plan, int32_t *n);

@@ -31,6 +31,7 @@ EXPORTS = (
     "vorta_plan_stage_ms", "vorta_plan_stage_ms_at", "vorta_plan_last_launches", "vorta_device_status",
     "vorta_status_string", "vorta_routed_attention_static", "vorta_plan_device",
     "vorta_router_gates", "vorta_soft_mixture", "vorta_shard_heads", "vorta_plan_kernel_in_use",
+    "vorta_plan_attention_ms_at",
 )
 VORTA_STATIC_WORKSPACE_BYTES = 16 * 1024 * 1024
 
@@ -91,6 +92,7 @@ def lib() -> ctypes.CDLL:
     L.vorta_plan_set_profiling.argtypes = [vp, i32]
     L.vorta_plan_stage_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float * 4)]
     L.vorta_plan_stage_ms_at.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_float * 4)]
+    L.vorta_plan_attention_ms_at.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_float * 2)]
     L.vorta_plan_last_launches.argtypes = [vp, ctypes.POINTER(i32)]
     L.vorta_device_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
     L.vorta_status_string.argtypes = [ctypes.c_int]
@@ -225,6 +227,12 @@ def vorta_plan_stage_ms_at(plan: int, calls_back: int):
     return [float(x) for x in ms]
 
 
+def vorta_plan_attention_ms_at(plan: int, calls_back: int):
+    ms = (ctypes.c_float * 2)()
+    _check(lib().vorta_plan_attention_ms_at(plan, calls_back, ctypes.byref(ms)), "vorta_plan_attention_ms_at")
+    return [float(x) for x in ms]
+
+
 def vorta_plan_last_launches(plan: int) -> int:
     n = ctypes.c_int32()
     _check(lib().vorta_plan_last_launches(plan, ctypes.byref(n)), "vorta_plan_last_launches")
@@ -309,6 +317,10 @@ class Plan:
     def stage_ms(self, calls_back: int = 0):
         """[select, gather, attention, scatter] milliseconds of a profiled call."""
         return vorta_plan_stage_ms_at(self.handle, calls_back)
+
+    def attention_ms(self, calls_back: int = 0):
+        """[first attention kernel, single-CTA kernel after the pair kernel (0 if one launch)] milliseconds."""
+        return vorta_plan_attention_ms_at(self.handle, calls_back)
 
     def last_launches(self) -> int:
         return vorta_plan_last_launches(self.handle)

@@ -65,8 +65,8 @@ struct vorta_plan {
     // profiling: a ring of event sets, one per call, so that several calls can be
     // enqueued before their stage times are read
     static constexpr int kProfSlots = 64;
-    mutable cudaEvent_t ev[kProfSlots][5] = {};
-    mutable bool ev_valid[kProfSlots][5] = {};
+    mutable cudaEvent_t ev[kProfSlots][6] = {};  // 0..4 around the four stages; 5 between the two attention launches
+    mutable bool ev_valid[kProfSlots][6] = {};
     mutable int64_t prof_calls = 0;  // calls recorded so far
     bool profiling = false;
     mutable int32_t last_launches = 0;
@@ -503,12 +503,13 @@ bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) %
 static bool pair_supported(const vorta_plan *p) { return p->g.d == 128 && (p->sm_count & 1) == 0 && p->sm_count >= 2; }
 
 // The kernel a call over `wl` runs: VORTA_KERNEL_AUTO takes the pair kernel (with the single-CTA
-// kernel for the sliding heads) where the full and core-set heads hold at least half of the work;
-// measured on a B200, that split is faster from there on and slower below.
+// kernel for the sliding heads) where the full and core-set heads hold at least 60 % of the work:
+// measured on a B200, the split is 4 to 6 % faster at shares of 0.9 and above and 1 to 2 % slower at
+// 0.53 and below (two launches, two tails).
 static int32_t resolve_kernel(const vorta_plan *p, const vorta_plan::WorkList &wl)
 {
     if (p->kernel != VORTA_KERNEL_AUTO) return p->kernel;
-    return pair_supported(p) && wl.linear_share >= 0.5 ? VORTA_KERNEL_PAIR : VORTA_KERNEL_TCGEN05;
+    return pair_supported(p) && wl.linear_share >= 0.6 ? VORTA_KERNEL_PAIR : VORTA_KERNEL_TCGEN05;
 }
 
 #ifdef VORTA_TRACE
@@ -853,6 +854,28 @@ int vorta_plan_stage_ms_at(const vorta_plan *p, int32_t calls_back, float ms[4])
 
 int vorta_plan_stage_ms(const vorta_plan *p, float ms[4]) { return vorta_plan_stage_ms_at(p, 0, ms); }
 
+int vorta_plan_attention_ms_at(const vorta_plan *p, int32_t calls_back, float ms[2])
+{
+    if (!p || !ms || calls_back < 0 || calls_back >= vorta_plan::kProfSlots) return VORTA_ERR_INVALID_ARG;
+    if (p->host_only) return VORTA_ERR_UNSUPPORTED;
+    if (calls_back >= p->prof_calls) return VORTA_ERR_INVALID_ARG;
+    const int slot = (int)((p->prof_calls - 1 - calls_back) % vorta_plan::kProfSlots);
+    ms[0] = ms[1] = 0.f;
+    if (!p->ev_valid[slot][2] || !p->ev_valid[slot][3]) return VORTA_OK;
+    cudaError_t e;
+    if (p->ev_valid[slot][5]) {
+        e = cudaEventElapsedTime(&ms[0], p->ev[slot][2], p->ev[slot][5]);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms[1], p->ev[slot][5], p->ev[slot][3]);
+    } else {
+        e = cudaEventElapsedTime(&ms[0], p->ev[slot][2], p->ev[slot][3]);
+    }
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return VORTA_ERR_CUDA;
+    }
+    return VORTA_OK;
+}
+
 int vorta_plan_last_launches(const vorta_plan *p, int32_t *n)
 {
     if (!p || !n) return VORTA_ERR_INVALID_ARG;
@@ -1003,6 +1026,7 @@ static int run_layer(const vorta_plan *p, const vorta_plan::WorkList &wl, int32_
                 if (e != cudaSuccess) return VORTA_ERR_CUDA;
                 ++launches;
             }
+            if (wl.n_linear > 0 && wl.n_items - wl.n_linear > 0) mark(5);
             if (wl.n_items - wl.n_linear > 0) {
                 e = launch_attention_sm100(prm_tiles, maps, p->sm_count, s);
                 if (e != cudaSuccess) return VORTA_ERR_CUDA;

@@ -241,7 +241,7 @@ def test_routes_can_change_between_steps_and_shared_selection_features():
 
 
 def test_default_kernel_choice_follows_the_routes():
-    """VORTA_KERNEL_AUTO: the pair kernel where full and core-set heads hold at least half of the
+    """VORTA_KERNEL_AUTO: the pair kernel where full and core-set heads hold at least 60 % of the
     work, the single-CTA kernel otherwise; the choice is remade when the routes change."""
     wl = Workload("auto", (6, 16, 16), 3, 128, (2, 8, 8), (3, 3, 3), 0.5, (0, 1, 2), 64, False)
     Q, K, V = workloads.make_qkv(wl, DEV)
