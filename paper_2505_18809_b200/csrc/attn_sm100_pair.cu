@@ -37,8 +37,8 @@
 //
 // Barriers that collect arrivals from both CTAs (operand loads landed, P written, O read)
 // live in the even CTA; the odd CTA arrives on them through the cluster's shared-memory
-// window.  Commits of the pair's MMAs are multicast to the barrier at the same offset in
-// both CTAs.  No bulk load uses multicast.
+// window.  A commit of the pair's MMAs arrives on the barrier at the same offset in both
+// CTAs.  Every load is a plain copy into the issuing CTA's own shared memory.
 //
 // Every wait is bounded: a wait that sees no progress for about two seconds records a
 // code in the status word (1000 + the code, to tell it from the single-CTA kernel's),
@@ -218,7 +218,7 @@ __device__ __forceinline__ uint32_t elect_one()
 }
 
 // Tiled bulk load into this CTA's shared memory whose bytes are counted on a barrier of
-// the even CTA (`bar` is an address in the cluster window).  No multicast.
+// the even CTA (`bar` is an address in the cluster window); the data go to this CTA only.
 __device__ __forceinline__ void tma_load_5d_pair(uint32_t dst, const CUtensorMap *map, uint32_t bar, int32_t c0,
                                                  int32_t c1, int32_t c2, int32_t c3, int32_t c4)
 {
@@ -791,7 +791,7 @@ attention_sm100_pair_kernel(const __grid_constant__ AttnParams p, const __grid_c
     if (threadIdx.x == 0) {
         const uint32_t bars = smem_u32(ctl->bars);
         for (int i = 0; i < BAR_COUNT; ++i) {
-            uint32_t n = 1;  // one multicast commit
+            uint32_t n = 1;  // one commit of the pair's MMAs
             if (i == BAR_Q_FULL || (i >= BAR_KV_FULL && i < BAR_KV_FULL + kStages)) n = 2;  // one producer per CTA
             if (i >= BAR_P_LO && i < BAR_P_HI + kSBufs) n = 8;   // four warps of a group in each CTA
             if (i >= BAR_REF && i < BAR_EPI) n = 4;               // four warps of a group
