@@ -18,7 +18,8 @@
 // nor another group's block delays a softmax thread.
 //
 // Warp roles (448 threads per CTA, 128 registers each):
-//   warp 0        TMA producer of this CTA's Q tile and K/V halves (8-slot ring of 16 KB)
+//   warp 0        TMA producer of this CTA's Q tile and K/V halves (4-slot ring of 32 KB: the K
+//                 half of block i and the V half of block i-3, which the MMA warp needs together)
 //   warp 1        tensor-memory allocation; in the even CTA the MMA issuer of the pair
 //   warps 2-13    softmax: three groups of four warps, one thread per query row; group k
 //                 owns score buffer k, i.e. the KV blocks whose running number is k modulo
@@ -58,12 +59,13 @@ namespace {
 namespace ptx = cuda::ptx;
 
 constexpr int D = 128;                   // head dimension this kernel is built for
-constexpr int kStages = 8;               // ring slots: one K half or one V half each
+constexpr int kStages = 4;               // ring slots: the K half of one block and the V half of another
 constexpr int kSBufs = 3;                // score buffers in tensor memory
 constexpr uint32_t kSlabBytes = 16384;   // 128 rows x 64 bf16: one swizzled slab of Q or of a V half
 constexpr uint32_t kKSlabBytes = 8192;   // 64 rows x 64 bf16: one slab of a K half
 constexpr uint32_t kQBytes = 2 * kSlabBytes;
-constexpr uint32_t kSlotBytes = 16384;
+constexpr uint32_t kHalfBytes = 16384;   // a K half (two 8 KB slabs) or a V half (one slab)
+constexpr uint32_t kSlotBytes = 2 * kHalfBytes;  // K half at +0, V half at +kHalfBytes
 constexpr uint32_t kSmemQ = 0;
 constexpr uint32_t kSmemKV = kQBytes;
 constexpr uint32_t kSmemCtl = kSmemKV + kStages * kSlotBytes;
@@ -81,9 +83,8 @@ enum {
     BAR_KV_EMPTY = BAR_KV_FULL + kStages,    // +slot: the MMAs reading the slot are done
     BAR_S_FULL = BAR_KV_EMPTY + kStages,     // +buffer: S of a block written
     BAR_PV_DONE = BAR_S_FULL + kSBufs,       // +buffer: O += P V of a block done
-    BAR_P_LO = BAR_PV_DONE + kSBufs,         // +buffer, even: P of keys [0, 64) written over S
-    BAR_P_HI = BAR_P_LO + kSBufs,            // +buffer, even: P of the other keys written
-    BAR_REF = BAR_P_HI + kSBufs,             // +group: reference maxima of a block published
+    BAR_P_READY = BAR_PV_DONE + kSBufs,      // +buffer, even: P of a block written over S by both CTAs
+    BAR_REF = BAR_P_READY + kSBufs,          // +group: reference maxima of a block published
     BAR_STAGGER = BAR_REF + kGroups,         // +0 / +1: the group of the item's first / second block is halfway into it
     BAR_EPI = BAR_STAGGER + 2,               // partial row sums of an item published
     BAR_O_FREE = BAR_EPI + 1,                // even: both epilogues have read O out of tensor memory
@@ -332,12 +333,11 @@ __device__ __forceinline__ void exp_half(uint32_t (&s)[64], float scale, float n
     }
 }
 
-// write the 32 packed P words of 64 keys held in s[0 .. 32) to t_p
+// write the 32 packed P words of 64 keys held in s[0 .. 32) to t_p (the caller waits for the stores)
 __device__ __forceinline__ void store_p(uint32_t t_p, uint32_t (&s)[64])
 {
     uint32_t(&all)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[0]);
     ptx::tcgen05_st_32x32b(t_p, all);
-    tc_wait_st();
 }
 
 // this thread's row of O times a
@@ -369,19 +369,13 @@ __device__ __forceinline__ float row_max64(const uint32_t (&s)[64])
     return fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
 }
 
-// One step of the item's K/V load sequence, the order in which the MMA warp consumes the
-// blocks: K_0, K_1, K_2, then V_j followed by K_{j+3} for j = 0, 1, ...  Step t of an item
-// with n KV blocks is (is_v, block).
-__device__ __forceinline__ void kv_step(int32_t t, int32_t n, bool &is_v, int32_t &block)
-{
-    const int32_t lead = min(n, kSBufs);
-    if (t < lead) { is_v = false; block = t; return; }
-    const int32_t u = t - lead;           // position in the V_j, K_{j+3} part
-    const int32_t paired = n - lead;      // V blocks that are followed by a K block
-    if (u < 2 * paired) { is_v = (u & 1) == 0; block = is_v ? (u >> 1) : (u >> 1) + kSBufs; return; }
-    is_v = true;
-    block = paired + (u - 2 * paired);
-}
+// The K/V load sequence of an item with n KV blocks, in the order the MMA warp consumes it: step i
+// carries K_i (if i < n) and V_{i-3} (if 3 <= i < n + 3), so that what block j needs after its own K,
+// namely V_j, and what follows it in the tensor pipe, K_{j+3}, arrive together in one ring slot behind
+// one barrier.  Steps that carry nothing (i in [n, 3) of an item shorter than three blocks) are skipped
+// by both sides.
+__device__ __forceinline__ bool step_has_k(int32_t i, int32_t n) { return i < n; }
+__device__ __forceinline__ bool step_has_v(int32_t i, int32_t n) { return i >= kSBufs && i < n + kSBufs; }
 
 // ------------------------------------------------------------------ roles
 // Loads of CTA `rank`: its Q tile, and of every KV block its half of K (keys) and of V (channels).
@@ -404,24 +398,26 @@ __device__ __forceinline__ void producer_role(const AttnParams &p, const AttnMap
                 mbar_arrive_cluster(even_bars + 8 * BAR_Q_FULL);  // no second tile: nothing to load
             }
         }
-        for (int32_t t = 0; t < 2 * w.kv_count; ++t) {
-            bool is_v;
-            int32_t j;
-            kv_step(t, w.kv_count, is_v, j);
+        for (int32_t i = 0; i < w.kv_count + kSBufs; ++i) {
+            const bool has_k = step_has_k(i, w.kv_count), has_v = step_has_v(i, w.kv_count);
+            if (!has_k && !has_v) continue;
             const uint32_t slot = kv_it % kStages;
             if (!mbar_wait(bars + 8 * (BAR_KV_EMPTY + slot), ((kv_it / kStages) & 1) ^ 1, ctl, p.status, 102)) return;
             if (lane == 0) {
                 const uint32_t full = even_bars + 8 * (BAR_KV_FULL + slot);
                 const uint32_t dst = smem_base + kSmemKV + slot * kSlotBytes;
-                mbar_expect_tx_cluster(full, kSlotBytes);  // rows past the end of the sequence arrive as zeros
-                if (is_v) {
-                    // the 128 keys of the block, channels [64 rank, 64 rank + 64)
-                    tma_load_5d_pair(dst, &maps.v[w.mode], full, (int32_t)rank * 64, j * kBlockM, 0, 0, w.slice);
-                } else {
-                    // keys [64 rank, 64 rank + 64) of the block, all channels
+                // rows past the end of the sequence arrive as zeros and count like the others
+                mbar_expect_tx_cluster(full, (has_k ? kHalfBytes : 0u) + (has_v ? kHalfBytes : 0u));
+                if (has_k) {
+                    // keys [64 rank, 64 rank + 64) of block i, all channels
                     for (int h = 0; h < 2; ++h)
                         tma_load_5d_pair(dst + h * kKSlabBytes, &maps.k_half[w.mode], full, h * 64,
-                                         j * kBlockM + (int32_t)rank * (kBlockM / 2), 0, 0, w.slice);
+                                         i * kBlockM + (int32_t)rank * (kBlockM / 2), 0, 0, w.slice);
+                }
+                if (has_v) {
+                    // the 128 keys of block i - 3, channels [64 rank, 64 rank + 64)
+                    tma_load_5d_pair(dst + kHalfBytes, &maps.v[w.mode], full, (int32_t)rank * 64, (i - kSBufs) * kBlockM,
+                                     0, 0, w.slice);
                 }
             }
             ++kv_it;
@@ -446,12 +442,12 @@ __device__ __forceinline__ void mma_role(const AttnParams &p, Ctl *ctl, uint32_t
     // (16-byte granular) address field, so one 64-bit add moves between them.
     const uint64_t q_desc = smem_desc(smem_base + kSmemQ, 16, 1024);
     const uint64_t k_desc0 = smem_desc(smem_base + kSmemKV, 16, 1024);          // K-major, 64-row slabs
-    const uint64_t v_desc0 = smem_desc(smem_base + kSmemKV, kSlabBytes, 1024);  // MN-major, one 64-channel slab
+    const uint64_t v_desc0 = smem_desc(smem_base + kSmemKV + kHalfBytes, kSlabBytes, 1024);  // MN-major, one 64-channel slab
     constexpr uint64_t kSlotStep = kSlotBytes >> 4;
     const uint32_t idesc_pv = instr_desc_pair((uint32_t)D, 1), idesc_qk = instr_desc_pair((uint32_t)kBlockM, 0);
     const uint32_t t_o = tmem + kSBufs * 128;
 
-    // next step of the load sequence: wait for both halves of its block, return the ring slot
+    // next step of the load sequence: wait for both CTAs' halves of it, return the ring slot
     auto next_kv = [&](uint32_t &slot, int32_t code) {
         slot = kv_it % kStages;
         const bool ok = mbar_wait_uniform(bars + 8 * (BAR_KV_FULL + slot), (kv_it / kStages) & 1, ctl, p.status, code);
@@ -459,42 +455,38 @@ __device__ __forceinline__ void mma_role(const AttnParams &p, Ctl *ctl, uint32_t
         return ok;
     };
     auto free_kv = [&](uint32_t slot) { tc_commit_pair(bars + 8 * (BAR_KV_EMPTY + slot), leader); };
-    // S[buf] = Q K^T over the K block in `slot` (16 channels per MMA)
-    auto issue_qk = [&](uint32_t buf, uint32_t slot, uint32_t idesc) {
+    // S[buf] = Q K^T over the K half-blocks in `slot` (16 channels per MMA)
+    auto issue_qk = [&](uint32_t buf, uint32_t slot) {
         const uint64_t kb = k_desc0 + (uint64_t)slot * kSlotStep;
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
             const uint64_t qoff = (uint64_t)(((kk / 4) * kSlabBytes + (kk % 4) * 32) >> 4);
             const uint64_t koff = (uint64_t)(((kk / 4) * kKSlabBytes + (kk % 4) * 32) >> 4);
-            mma_pair_ss(tmem + buf * 128, q_desc + qoff, kb + koff, idesc, kk > 0 ? 1u : 0u, leader);
+            mma_pair_ss(tmem + buf * 128, q_desc + qoff, kb + koff, idesc_qk, kk > 0 ? 1u : 0u, leader);
         }
     };
-    // O (+)= P[buf] V over the V block in `slot`; P is packed bf16 in the first columns of S[buf]
-    // (16 keys per MMA: steps [k0, k0 + 4) of the block, cut at `ksteps`)
-    auto issue_pv = [&](uint32_t buf, uint32_t slot, int k0, int ksteps, bool first) {
+    // O (+)= P[buf] V over the V half-blocks in `slot`; P is packed bf16 in the first 64 columns of
+    // S[buf] (16 keys per MMA)
+    auto issue_pv = [&](uint32_t buf, uint32_t slot, bool first) {
         const uint64_t vb = v_desc0 + (uint64_t)slot * kSlotStep;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int kk = k0 + i;
-            if (kk < ksteps)
-                mma_pair_ts(t_o, tmem + buf * 128 + kk * 8, vb + (uint64_t)(kk * (2048 >> 4)), idesc_pv,
-                            (!first || kk > 0) ? 1u : 0u, leader);
-        }
+        for (int kk = 0; kk < kBlockM / 16; ++kk)
+            mma_pair_ts(t_o, tmem + buf * 128 + kk * 8, vb + (uint64_t)(kk * (2048 >> 4)), idesc_pv,
+                        (!first || kk > 0) ? 1u : 0u, leader);
     };
 
     for (int32_t it = 0; it < count; ++it) {
         const WorkItem *w = p.items + begin + it;
         const int32_t n = (int32_t)uniform_u32((uint32_t)w->kv_count);
-        constexpr int ksteps = kBlockM / 16;
 
         if (!mbar_wait_uniform(bars + 8 * BAR_Q_FULL, it & 1, ctl, p.status, 201)) return;
-        // scores of the first blocks, one per buffer
+        // scores of the first blocks, one per buffer (steps 0 .. 2 carry K only)
         for (int32_t j = 0; j < min(n, kSBufs); ++j) {
             uint32_t slot;
             if (!next_kv(slot, 202)) return;
             tc_fence_after();
             const uint32_t buf = (g0 + j) % kSBufs;
-            issue_qk(buf, slot, idesc_qk);
+            issue_qk(buf, slot);
             tc_commit_pair(bars + 8 * (BAR_S_FULL + buf), leader);
             free_kv(slot);
         }
@@ -502,37 +494,28 @@ __device__ __forceinline__ void mma_role(const AttnParams &p, Ctl *ctl, uint32_t
 
         for (int32_t j = 0; j < n; ++j) {
             const uint32_t g = g0 + (uint32_t)j, buf = g % kSBufs, par = (g / kSBufs) & 1;
-            uint32_t slot_v;
-            if (!next_kv(slot_v, 203)) return;
+            // step j + 3: V_j and, if the item has it, K_{j+3}
+            uint32_t slot;
+            if (!next_kv(slot, 203)) return;
             if (leader) TRACE(0, g, 0);
-            // first half of P: the PV MMAs over keys [0, 64) start while the other half is still written
-            if (!mbar_wait_uniform(bars + 8 * (BAR_P_LO + buf), par, ctl, p.status, 204)) return;
+            if (!mbar_wait_uniform(bars + 8 * (BAR_P_READY + buf), par, ctl, p.status, 204)) return;
             if (j == 0) {
                 // the previous item's epilogues must have read O out of tensor memory
                 if (!mbar_wait_uniform(bars + 8 * BAR_O_FREE, (it & 1) ^ 1, ctl, p.status, 205)) return;
             }
             tc_fence_after();
             if (leader) TRACE(0, g, 1);
-            issue_pv(buf, slot_v, 0, ksteps, j == 0);
-            if (!mbar_wait_uniform(bars + 8 * (BAR_P_HI + buf), par, ctl, p.status, 208)) return;
-            tc_fence_after();
-            if (leader) TRACE(0, g, 2);
-            issue_pv(buf, slot_v, 4, ksteps, false);
+            issue_pv(buf, slot, j == 0);
             tc_commit_pair(bars + 8 * (BAR_PV_DONE + buf), leader);
-            free_kv(slot_v);
             if (leader) TRACE(0, g, 3);
             if (j + kSBufs < n) {
                 // the buffer P(j) leaves takes the scores of block j+3
-                uint32_t slot_k;
-                if (!next_kv(slot_k, 206)) return;
-                tc_fence_after();
-                if (leader) TRACE(0, g, 4);
-                issue_qk(buf, slot_k, idesc_qk);
+                issue_qk(buf, slot);
                 tc_commit_pair(bars + 8 * (BAR_S_FULL + buf), leader);
-                free_kv(slot_k);
-                if (leader) TRACE(0, g, 5);
                 if (j + kSBufs == n - 1) tc_commit_pair(bars + 8 * BAR_Q_EMPTY, leader);
             }
+            free_kv(slot);
+            if (leader) TRACE(0, g, 5);
         }
         g0 += (uint32_t)n;
     }
@@ -634,25 +617,23 @@ __device__ __forceinline__ bool softmax_block(const AttnParams &p, Ctl *ctl, con
         my_sum *= ex2(st.known - cur);  // known = -inf only while the sum is 0
         st.known = cur;
     }
-    // P = exp2(S * scale - reference) as packed bf16 over the first half of the buffer, handed
-    // over in two halves of 64 keys
+    // P = exp2(S * scale - reference) as packed bf16 over the first half of the buffer
     float2 sum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
     exp_half(s, scale, -cur, sum);
     store_p(t_s, s);
-    tc_fence_before();
-    __syncwarp();
-    if (lane == 0) {
-        arrive_even(bars, even_bars, rank, BAR_P_LO + buf);
-        if (jb < 2) mbar_arrive(bars + 8 * (BAR_STAGGER + jb));  // the next block's group may start
+    if (jb < 2) {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars + 8 * (BAR_STAGGER + jb));  // halfway: the next block's group may start
     }
     if (tr) TRACE(trole, g, 4);
     // P of keys [0, 64) went to columns [0, 32): the scores of the other keys are still in place
     load_half(1);
     exp_half(s, scale, -cur, sum);
     store_p(t_s + 32, s);
+    tc_wait_st();  // both halves of P are in tensor memory
     tc_fence_before();
     __syncwarp();
-    if (lane == 0) arrive_even(bars, even_bars, rank, BAR_P_HI + buf);
+    if (lane == 0) arrive_even(bars, even_bars, rank, BAR_P_READY + buf);
     if (tr) TRACE(trole, g, 5);
     st.sum = my_sum + ((sum[0].x + sum[0].y) + (sum[1].x + sum[1].y));
     return true;
@@ -670,7 +651,7 @@ __device__ __noinline__ bool softmax_block_full(const AttnParams &p, Ctl *ctl, c
     return softmax_block<true>(p, ctl, wp, t_row, g, jb, grp, row, rank, st);
 }
 
-// The thread of query row `row` in group `grp` (blocks whose running number is grp modulo 2).
+// The thread of query row `row` in group `grp` (blocks whose running number is grp modulo 3).
 // A CTA without a tile in an item only keeps the barrier phases of the pair moving.
 __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint32_t tmem, int32_t begin, int32_t count,
                                              int grp, int quad, int lane, uint32_t rank)
@@ -709,8 +690,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
                 __syncwarp();
                 if (lane == 0) {
                     mbar_arrive(bars + 8 * (BAR_REF + g % kGroups));  // keeps the phase of this barrier in step with g
-                    arrive_even(bars, even_bars, rank, BAR_P_LO + buf);
-                    arrive_even(bars, even_bars, rank, BAR_P_HI + buf);
+                    arrive_even(bars, even_bars, rank, BAR_P_READY + buf);
                 }
             }
             if (!mbar_wait(bars + 8 * (BAR_PV_DONE + gl % kSBufs), (gl / kSBufs) & 1, ctl, p.status, 393 + grp)) return;
@@ -793,7 +773,7 @@ attention_sm100_pair_kernel(const __grid_constant__ AttnParams p, const __grid_c
         for (int i = 0; i < BAR_COUNT; ++i) {
             uint32_t n = 1;  // one commit of the pair's MMAs
             if (i == BAR_Q_FULL || (i >= BAR_KV_FULL && i < BAR_KV_FULL + kStages)) n = 2;  // one producer per CTA
-            if (i >= BAR_P_LO && i < BAR_P_HI + kSBufs) n = 8;   // four warps of a group in each CTA
+            if (i >= BAR_P_READY && i < BAR_P_READY + kSBufs) n = 8;  // four warps of a group in each CTA
             if (i >= BAR_REF && i < BAR_EPI) n = 4;               // four warps of a group
             if (i == BAR_EPI) n = kSoftmaxWarps;
             if (i == BAR_O_FREE) n = 2 * kSoftmaxWarps;
