@@ -32,17 +32,15 @@
 // records a code in the status word, raises the CTA's abort flag and every role
 // leaves its loop; the CTA then gives outstanding copies time to land, frees its
 // TMEM and returns.
-#include <cuda/ptx>
-
 #include <type_traits>
 
-#include "vorta_internal.h"
+#include "sm100_common.cuh"
 
 namespace vorta {
 
 namespace {
 
-namespace ptx = cuda::ptx;
+using namespace sm100;
 
 constexpr int kStages = 4;                // KV ring slots (K and V blocks alternate)
 constexpr uint32_t kHalfBytes = 16384;    // 128 rows x 64 bf16: one swizzled half tile
@@ -53,8 +51,6 @@ constexpr uint32_t kSmemBars = kSmemKV + kStages * kTileBytes;
 constexpr uint32_t kCtlBytes = 2048;  // control block: barriers, flags, the column-mask classes
 constexpr uint32_t kSmemTotal = kSmemBars + kCtlBytes;
 constexpr uint32_t kSmemAlloc = kSmemTotal + 1024;  // slack to align the base to 1024 B
-constexpr float kRescaleThreshold = 8.0f;           // log2 units the row maximum may grow before O is rescaled
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 // barrier indices
 enum {
@@ -70,6 +66,7 @@ enum {
 };
 
 struct Ctl {
+    static constexpr int32_t kStatusBase = 0;  // added to the code of an expired wait in the status word
     uint64_t bars[BAR_COUNT];
     uint32_t tmem_base;
     volatile int32_t abort;
@@ -93,93 +90,6 @@ static_assert(kMaxMasks * 4 <= kAttnThreads, "one thread copies one word of the 
 #endif
 
 // ------------------------------------------------------------------ PTX helpers
-__device__ __forceinline__ uint32_t smem_u32(const void *p)
-{
-    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.shared::cta.b64 st, [%0];\n\t}" ::"r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n\t}" ::"r"(bar),
-                 "r"(bytes)
-                 : "memory");
-}
-
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-
-__device__ __forceinline__ unsigned long long global_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-
-// Bounded wait on a phase of an mbarrier.  Returns false if the CTA is aborting.
-__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, Ctl *ctl, int32_t *status, int32_t code)
-{
-    const unsigned long long t0 = global_ns();
-    for (uint32_t spin = 1;; ++spin) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((spin & 63u) == 0) {
-            if (ctl->abort) return false;
-            if (global_ns() - t0 > kWaitLimitNs) {
-                ctl->abort = code;
-                atomicCAS(status, 0, code);
-                return false;
-            }
-        }
-    }
-}
-
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, Ctl *ctl, int32_t *status, int32_t code)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, ctl, status, code);
-}
-
-// The same wait with a warp-uniform verdict, and a warp-uniform copy of a value all
-// lanes hold: both come out of warp-wide reductions, which the compiler can keep in
-// uniform registers.  The MMA warp needs this: the operands of tcgen05.mma are uniform
-// registers, and only provably uniform values and control flow reach them without a
-// per-instruction detour through vector registers.
-__device__ __forceinline__ bool mbar_wait_uniform(uint32_t bar, uint32_t parity, Ctl *ctl, int32_t *status,
-                                                  int32_t code)
-{
-    return __all_sync(0xffffffffu, mbar_wait(bar, parity, ctl, status, code)) != 0;
-}
-
-__device__ __forceinline__ uint32_t uniform_u32(uint32_t v) { return __reduce_max_sync(0xffffffffu, v); }
-
-__device__ __forceinline__ uint32_t elect_one()
-{
-    uint32_t leader;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(leader));
-    return leader;
-}
-
 __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int32_t c0,
                                             int32_t c1, int32_t c2, int32_t c3, int32_t c4)
 {
@@ -189,11 +99,6 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar)
         : "memory");
 }
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // The MMA warp stays converged: every lane runs the (warp-uniform) descriptor
 // arithmetic, and `leader` (1 in lane 0, 0 elsewhere) guards the instruction itself.
@@ -228,47 +133,11 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
         : "memory");
 }
 
-// Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1.
-// lbo/sbo in bytes: for a K-major operand sbo is the pitch of 8-row groups; for an
-// MN-major operand lbo is the pitch of 64-element column blocks and sbo the pitch
-// of 8-row (K) groups.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((addr & 0x3ffffu) >> 4);
-    d |= (uint64_t)((lbo >> 4) & 0x3fffu) << 16;
-    d |= (uint64_t)((sbo >> 4) & 0x3fffu) << 32;
-    d |= (uint64_t)1 << 46;  // version
-    d |= (uint64_t)2 << 61;  // SWIZZLE_128B
-    return d;
-}
-
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128.  (A and B must have the same
 // 16-bit format: an fp16 P against a bf16 V is rejected by the hardware.)
 __device__ __forceinline__ uint32_t instr_desc(uint32_t n, uint32_t b_mn_major)
 {
     return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
-}
-
-__device__ __forceinline__ float ex2(float x)
-{
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
-{
-    uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
-
-__device__ __forceinline__ float max3(float a, float b, float c)
-{
-    float r;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
-    return r;
 }
 
 // Coordinates of block `j` of the item's KV sequence and its column-mask class.  text: the
@@ -288,28 +157,6 @@ __device__ __forceinline__ void kv_block_coords(const AttnParams &p, const WorkI
     }
 }
 
-// exp2(s * scale - ref) for the 64 scores of a sub-block, packed two bf16 per word IN
-// PLACE into s[0 .. 32): a packed word never lands on a score still to be read.
-// The row sums take the ROUNDED values the PV MMA will use, so that O / sum stays a true
-// weighted mean of V rows (with the unrounded ones a row that attends to a single key is
-// off by up to 2^-9 of |v|, beyond the output tolerance).  Scale-and-shift and the sums
-// use the packed two-wide fp32 instructions.
-__device__ __forceinline__ void exp_block(uint32_t (&s)[64], float scale, float neg_ref, float2 (&sum)[2])
-{
-    const float2 sc = make_float2(scale, scale), nr = make_float2(neg_ref, neg_ref);
-#pragma unroll
-    for (int c = 0; c < 64; c += 4) {
-        float2 x0 = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), sc, nr);
-        float2 x1 = __ffma2_rn(make_float2(__uint_as_float(s[c + 2]), __uint_as_float(s[c + 3])), sc, nr);
-        const uint32_t k0 = pack_bf16(ex2(x0.x), ex2(x0.y));
-        const uint32_t k1 = pack_bf16(ex2(x1.x), ex2(x1.y));
-        s[c >> 1] = k0;
-        s[(c >> 1) + 1] = k1;
-        sum[0] = __fadd2_rn(sum[0], make_float2(__uint_as_float(k0 << 16), __uint_as_float(k0 & 0xffff0000u)));
-        sum[1] = __fadd2_rn(sum[1], make_float2(__uint_as_float(k1 << 16), __uint_as_float(k1 & 0xffff0000u)));
-    }
-}
-
 // write the packed P words of a sub-block of `width` keys to the first width/2 columns at t_p
 __device__ __forceinline__ void store_p(uint32_t t_p, int32_t width, uint32_t (&s)[64])
 {
@@ -324,35 +171,6 @@ __device__ __forceinline__ void store_p(uint32_t t_p, int32_t width, uint32_t (&
         }
     }
     tc_wait_st();
-}
-
-// this thread's row of O times a
-template <int D>
-__device__ __forceinline__ void rescale_o(uint32_t t_o, float a)
-{
-#pragma unroll
-    for (int c = 0; c < D / 32; ++c) {
-        uint32_t o[32];
-        ptx::tcgen05_ld_32x32b(o, t_o + c * 32);
-        tc_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * a);
-        ptx::tcgen05_st_32x32b(t_o + c * 32, o);
-    }
-}
-
-// maximum of the 64 scores of a sub-block (four independent chains of three-input max)
-__device__ __forceinline__ float row_max64(const uint32_t (&s)[64])
-{
-    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-    for (int c = 0; c < 64; c += 8) {
-        mx0 = max3(mx0, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
-        mx1 = max3(mx1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
-        mx2 = max3(mx2, __uint_as_float(s[c + 4]), __uint_as_float(s[c + 5]));
-        mx3 = max3(mx3, __uint_as_float(s[c + 6]), __uint_as_float(s[c + 7]));
-    }
-    return fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
 }
 
 // ------------------------------------------------------------------ roles

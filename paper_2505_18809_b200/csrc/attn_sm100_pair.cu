@@ -46,17 +46,15 @@
 // raises the CTA's abort flag and every role of the CTA leaves its loop (the peer's waits
 // then run out the same way); the CTAs meet at a cluster barrier, free their tensor
 // memory, meet again and return.
-#include <cuda/ptx>
-
 #include <type_traits>
 
-#include "vorta_internal.h"
+#include "sm100_common.cuh"
 
 namespace vorta {
 
 namespace {
 
-namespace ptx = cuda::ptx;
+using namespace sm100;
 
 constexpr int D = 128;                   // head dimension this kernel is built for
 constexpr int kStages = 4;               // ring slots: the K half of one block and the V half of another
@@ -69,8 +67,6 @@ constexpr uint32_t kSlotBytes = 2 * kHalfBytes;  // K half at +0, V half at +kHa
 constexpr uint32_t kSmemQ = 0;
 constexpr uint32_t kSmemKV = kQBytes;
 constexpr uint32_t kSmemCtl = kSmemKV + kStages * kSlotBytes;
-constexpr float kRescaleThreshold = 8.0f;  // log2 units a row maximum may exceed the reference by
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 constexpr int kGroups = 3;                // softmax groups: group k owns score buffer k
 constexpr int kSoftmaxWarps = 4 * kGroups;
 constexpr int kPairThreads = 64 + 32 * kSoftmaxWarps;
@@ -93,6 +89,7 @@ enum {
 };
 
 struct Ctl {
+    static constexpr int32_t kStatusBase = 1000;  // this kernel's wait codes in the status word: 1xxx
     uint64_t bars[BAR_COUNT];
     uint32_t tmem_base;
     volatile int32_t abort;
@@ -119,21 +116,6 @@ static_assert(kSBufs == kGroups, "a softmax group owns one score buffer");
 #endif
 
 // ------------------------------------------------------------------ PTX helpers
-__device__ __forceinline__ uint32_t smem_u32(const void *p)
-{
-    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.shared::cta.b64 st, [%0];\n\t}" ::"r"(bar) : "memory");
-}
-
 // address, in the cluster's shared-memory window, of this CTA's `addr` in CTA `rank`
 __device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank)
 {
@@ -154,69 +136,8 @@ __device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t cluster_addr, ui
                  : "memory");
 }
 
-// (Barriers that also take arrivals from the peer CTA are waited on in the same way: the data behind
+// (Barriers that also take arrivals from the peer CTA are waited on like the others: the data behind
 // those arrivals is in tensor memory or was written by TMA.)
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-
-__device__ __forceinline__ unsigned long long global_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-
-// Bounded wait on a phase of an mbarrier.  Returns false if the CTA is aborting.
-__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, Ctl *ctl, int32_t *status, int32_t code)
-{
-    const unsigned long long t0 = global_ns();
-    for (uint32_t spin = 1;; ++spin) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((spin & 63u) == 0) {
-            if (ctl->abort) return false;
-            if (global_ns() - t0 > kWaitLimitNs) {
-                ctl->abort = code;
-                atomicCAS(status, 0, 1000 + code);  // 1xxx: this kernel (the single-CTA kernel reports xxx)
-                return false;
-            }
-        }
-    }
-}
-
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, Ctl *ctl, int32_t *status, int32_t code)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, ctl, status, code);
-}
-
-// The same wait with a warp-uniform verdict, and a warp-uniform copy of a value all lanes
-// hold (the MMA warp's descriptors and loop counts must reach uniform registers).
-__device__ __forceinline__ bool mbar_wait_uniform(uint32_t bar, uint32_t parity, Ctl *ctl, int32_t *status,
-                                                  int32_t code)
-{
-    return __all_sync(0xffffffffu, mbar_wait(bar, parity, ctl, status, code)) != 0;
-}
-
-__device__ __forceinline__ uint32_t uniform_u32(uint32_t v) { return __reduce_max_sync(0xffffffffu, v); }
-
-__device__ __forceinline__ uint32_t elect_one()
-{
-    uint32_t leader;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(leader));
-    return leader;
-}
 
 // Tiled bulk load into this CTA's shared memory whose bytes are counted on a barrier of
 // the even CTA (`bar` is an address in the cluster window); the data go to this CTA only.
@@ -229,11 +150,6 @@ __device__ __forceinline__ void tma_load_5d_pair(uint32_t dst, const CUtensorMap
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar)
         : "memory");
 }
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ void cluster_sync_all()
 {
@@ -274,63 +190,10 @@ __device__ __forceinline__ void mma_pair_ts(uint32_t d_tmem, uint32_t a_tmem, ui
         : "memory");
 }
 
-// Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1 (lbo/sbo in bytes:
-// sbo is the pitch of 8-row groups; lbo the pitch of 64-element column blocks of an MN-major operand).
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((addr & 0x3ffffu) >> 4);
-    d |= (uint64_t)((lbo >> 4) & 0x3fffu) << 16;
-    d |= (uint64_t)((sbo >> 4) & 0x3fffu) << 32;
-    d |= (uint64_t)1 << 46;  // version
-    d |= (uint64_t)2 << 61;  // SWIZZLE_128B
-    return d;
-}
-
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 256 (128 rows in each CTA), N = n over the pair.
 __device__ __forceinline__ uint32_t instr_desc_pair(uint32_t n, uint32_t b_mn_major)
 {
     return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major << 16) | ((n >> 3) << 17) | ((256u >> 4) << 24);
-}
-
-__device__ __forceinline__ float ex2(float x)
-{
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
-{
-    uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
-
-__device__ __forceinline__ float max3(float a, float b, float c)
-{
-    float r;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
-    return r;
-}
-
-// exp2(s * scale - ref) for 64 scores of a row, packed two bf16 per word IN PLACE into
-// s[0 .. 32): a packed word never lands on a score still to be read.  The row sums take the
-// ROUNDED values the PV MMA will use, so that O / sum stays a true weighted mean of V rows.
-__device__ __forceinline__ void exp_half(uint32_t (&s)[64], float scale, float neg_ref, float2 (&sum)[2])
-{
-    const float2 sc = make_float2(scale, scale), nr = make_float2(neg_ref, neg_ref);
-#pragma unroll
-    for (int c = 0; c < 64; c += 4) {
-        float2 x0 = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), sc, nr);
-        float2 x1 = __ffma2_rn(make_float2(__uint_as_float(s[c + 2]), __uint_as_float(s[c + 3])), sc, nr);
-        const uint32_t k0 = pack_bf16(ex2(x0.x), ex2(x0.y));
-        const uint32_t k1 = pack_bf16(ex2(x1.x), ex2(x1.y));
-        s[c >> 1] = k0;
-        s[(c >> 1) + 1] = k1;
-        sum[0] = __fadd2_rn(sum[0], make_float2(__uint_as_float(k0 << 16), __uint_as_float(k0 & 0xffff0000u)));
-        sum[1] = __fadd2_rn(sum[1], make_float2(__uint_as_float(k1 << 16), __uint_as_float(k1 & 0xffff0000u)));
-    }
 }
 
 // write the 32 packed P words of 64 keys held in s[0 .. 32) to t_p (the caller waits for the stores)
@@ -338,35 +201,6 @@ __device__ __forceinline__ void store_p(uint32_t t_p, uint32_t (&s)[64])
 {
     uint32_t(&all)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[0]);
     ptx::tcgen05_st_32x32b(t_p, all);
-}
-
-// this thread's row of O times a
-__device__ __forceinline__ void rescale_o(uint32_t t_o, float a)
-{
-#pragma unroll
-    for (int c = 0; c < D / 32; ++c) {
-        uint32_t o[32];
-        ptx::tcgen05_ld_32x32b(o, t_o + c * 32);
-        tc_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * a);
-        ptx::tcgen05_st_32x32b(t_o + c * 32, o);
-    }
-    tc_wait_st();
-}
-
-// maximum of 64 scores (four independent chains of three-input max)
-__device__ __forceinline__ float row_max64(const uint32_t (&s)[64])
-{
-    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-    for (int c = 0; c < 64; c += 8) {
-        mx0 = max3(mx0, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
-        mx1 = max3(mx1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
-        mx2 = max3(mx2, __uint_as_float(s[c + 4]), __uint_as_float(s[c + 5]));
-        mx3 = max3(mx3, __uint_as_float(s[c + 6]), __uint_as_float(s[c + 7]));
-    }
-    return fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
 }
 
 // The K/V load sequence of an item with n KV blocks, in the order the MMA warp consumes it: step i
@@ -610,7 +444,8 @@ __device__ __forceinline__ bool softmax_block(const AttnParams &p, Ctl *ctl, con
         const uint32_t gb = g - 1;
         if (!mbar_wait(bars + 8 * (BAR_PV_DONE + gb % kSBufs), (gb / kSBufs) & 1, ctl, p.status, 321 + grp)) return false;
         tc_fence_after();
-        rescale_o(t_o, raise ? ex2(prev - cur) : 1.f);
+        rescale_o<D>(t_o, raise ? ex2(prev - cur) : 1.f);
+        tc_wait_st();
     }
     float my_sum = st.sum;
     if (st.known != cur) {
@@ -619,7 +454,7 @@ __device__ __forceinline__ bool softmax_block(const AttnParams &p, Ctl *ctl, con
     }
     // P = exp2(S * scale - reference) as packed bf16 over the first half of the buffer
     float2 sum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-    exp_half(s, scale, -cur, sum);
+    exp_block(s, scale, -cur, sum);
     store_p(t_s, s);
     if (jb < 2) {
         __syncwarp();
@@ -628,7 +463,7 @@ __device__ __forceinline__ bool softmax_block(const AttnParams &p, Ctl *ctl, con
     if (tr) TRACE(trole, g, 4);
     // P of keys [0, 64) went to columns [0, 32): the scores of the other keys are still in place
     load_half(1);
-    exp_half(s, scale, -cur, sum);
+    exp_block(s, scale, -cur, sum);
     store_p(t_s + 32, s);
     tc_wait_st();  // both halves of P are in tensor memory
     tc_fence_before();
