@@ -86,6 +86,18 @@ def test_null_arguments_are_errors_not_crashes():
     assert L.vorta_routed_attention(p.handle, 16, 16, 16, 16, None, 0, None, 0, None) == vb.VORTA_ERR_UNSUPPORTED
     assert L.vorta_plan_block_mask(p.handle, 16) == vb.VORTA_ERR_UNSUPPORTED
     assert L.vorta_coreset_select(p.handle, 16, 1, 64, 16, 16, None) == vb.VORTA_ERR_UNSUPPORTED
+    # kernel selection: ids outside the enum are refused; a plan without SMs in pairs has no pair kernel;
+    # a host-only plan runs no kernel
+    assert L.vorta_plan_set_kernel(None, 0) == vb.VORTA_ERR_INVALID_ARG
+    for bad in (-1, 4, 99):
+        assert L.vorta_plan_set_kernel(p.handle, bad) == vb.VORTA_ERR_INVALID_ARG
+    for ok in (vb.VORTA_KERNEL_TCGEN05, vb.VORTA_KERNEL_SIMT, vb.VORTA_KERNEL_AUTO):
+        assert L.vorta_plan_set_kernel(p.handle, ok) == vb.VORTA_OK
+    assert L.vorta_plan_set_kernel(p.handle, vb.VORTA_KERNEL_PAIR) == vb.VORTA_ERR_UNSUPPORTED
+    assert L.vorta_plan_kernel_in_use(p.handle) < 0 and L.vorta_plan_kernel_in_use(None) < 0
+    ms = (ctypes.c_float * 2)()
+    assert L.vorta_plan_attention_ms_at(p.handle, 0, ctypes.byref(ms)) == vb.VORTA_ERR_UNSUPPORTED
+    assert L.vorta_plan_attention_ms_at(None, 0, ctypes.byref(ms)) == vb.VORTA_ERR_INVALID_ARG
     p.close()
 
 

@@ -271,6 +271,25 @@ def test_default_kernel_choice_follows_the_routes():
     p64.close()
 
 
+def test_stage_times_by_launch():
+    """Profiling events: the four stage times of a call, and the attention stage split by launch."""
+    wl = Workload("prof", (6, 16, 16), 3, 128, (2, 8, 8), (3, 3, 3), 0.5, (0, 1, 0), 65, False)
+    Q, K, V = workloads.make_qkv(wl, DEV)
+    p = vb.Plan.from_workload(wl)
+    p.set_profiling(True)
+    O = torch.empty_like(Q)
+    for kernel, launches in [(vb.VORTA_KERNEL_PAIR, 2), (vb.VORTA_KERNEL_TCGEN05, 1)]:
+        p.set_kernel(kernel)
+        p.routed_attention(Q, K, V, O)
+        torch.cuda.synchronize()
+        assert p.device_status() == 0 and p.last_launches() == launches
+        st, at = p.stage_ms(0), p.attention_ms(0)
+        assert max(st[0], st[1], st[3]) < 0.01 < st[2]   # no core-set head: only gaps between events around the attention
+        assert at[0] > 0.0 and (at[1] > 0.0) == (launches == 2)
+        assert abs(at[0] + at[1] - st[2]) < 0.02 * st[2] + 1e-3
+    p.close()
+
+
 @pytest.mark.parametrize("kernel", [vb.VORTA_KERNEL_TCGEN05, vb.VORTA_KERNEL_PAIR], ids=["tcgen05", "pair"])
 def test_growing_scores_exercise_the_lazy_rescale(kernel):
     """Keys whose norm grows along the sequence: the running maximum keeps rising, by less than
