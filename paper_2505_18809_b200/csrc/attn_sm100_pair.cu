@@ -99,7 +99,10 @@ struct Ctl {
 constexpr uint32_t kSmemTotal = kSmemCtl + ((sizeof(Ctl) + 127) / 128) * 128;
 constexpr uint32_t kSmemAlloc = kSmemTotal + 1024;  // slack to align the base to 1024 B
 static_assert(kSmemAlloc <= 232448, "shared memory budget of an sm_100 CTA");
-static_assert(kSBufs == kGroups, "a softmax group owns one score buffer");
+// A group's consecutive blocks use the same score buffer, so it asks for a buffer's scores one phase
+// after the other.  (A group hopping between buffers could ask for a buffer's next scores before its
+// previous ones were produced, and a parity wait two phases ahead passes at once.)
+static_assert(kSBufs == kGroups, "the parity waits on BAR_S_FULL rely on one score buffer per softmax group");
 
 // Optional cycle trace of CTA pair 0 (compiled in only with -DVORTA_TRACE; a debugging aid):
 // role 0 the MMA warp, 1 / 2 the first warp of softmax group 0 / 1 in the even CTA, 3 group 0 in the odd CTA.

@@ -149,14 +149,17 @@ def test_routed_attention_small_all_rows(wl, kernel):
     p.close()
 
 
-def test_many_slices_small_heads():
+@pytest.mark.parametrize("d,kernel", [(64, vb.VORTA_KERNEL_TCGEN05), (128, vb.VORTA_KERNEL_TCGEN05), (128, vb.VORTA_KERNEL_PAIR)],
+                         ids=["d64-tcgen05", "d128-tcgen05", "d128-pair"])
+def test_many_slices_small_heads(d, kernel):
     """Batch 3 x 70 heads of 48 tokens: slice indexing of every stage (the 5th TMA coordinate,
-    compact problem numbering, per-batch core-set tables) with far more heads than SMs' items."""
+    compact problem numbering, per-batch core-set tables) with far more heads than SMs' items; in
+    the pair kernel every item has one tile (the odd CTA of a pair only loads its K/V halves)."""
     routes = tuple((h * 7 + 3) % 3 for h in range(70))
-    wl = Workload("many-slices", (2, 4, 6), 70, 64, (1, 2, 2), (3, 3, 3), 0.5, routes, 61, False, 3)
+    wl = Workload("many-slices", (2, 4, 6), 70, d, (1, 2, 2), (3, 3, 3), 0.5, routes, 61, False, 3)
     Q, K, V = workloads.make_qkv(wl, DEV)
     p = vb.Plan.from_workload(wl)
-    O = run_layer(p, wl, Q, K, V, vb.VORTA_KERNEL_TCGEN05)
+    O = run_layer(p, wl, Q, K, V, kernel)
     for b in range(wl.B):
         for h in range(0, wl.heads, 3):
             for hh in (h, min(h + 1 + b, wl.heads - 1)):
