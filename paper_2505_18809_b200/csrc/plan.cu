@@ -1158,8 +1158,23 @@ int vorta_routed_attention_host(const vorta_plan *p, const void *Qh, const void 
         return VORTA_ERR_CUDA;
     int64_t ws_off = 0;
     int32_t ci = 0;
+    // Which attention kernels the previous group launched.  The pair kernel (clusters) and the single-CTA
+    // kernel are never left to share the GPU (run side by side they made the latter's bounded waits expire):
+    // where consecutive groups would mix them, the later group's queue waits for the earlier group's kernels.
+    bool prev_pair = false, prev_single = false;
+    const vorta_plan::HostChunk *prev = nullptr;
     for (const vorta_plan::HostChunk &c : p->chunks) {
         cudaStream_t sk = (ci++ & 1) ? p->s_alt : s;
+        const int32_t kernel = resolve_kernel(p, c.wl);
+        const bool use_pair = kernel == VORTA_KERNEL_PAIR && c.wl.n_linear > 0;
+        const bool use_single = kernel == VORTA_KERNEL_TCGEN05 ? c.wl.n_items > 0
+                                                               : (kernel == VORTA_KERNEL_PAIR && c.wl.n_items > c.wl.n_linear);
+        if (prev && ((prev_pair && use_single) || (prev_single && use_pair)) &&
+            cudaStreamWaitEvent(sk, prev->ev_done, 0) != cudaSuccess)
+            return VORTA_ERR_CUDA;
+        prev_pair = use_pair;
+        prev_single = use_single;
+        prev = &c;
         for (int32_t b = 0; b < g.B; ++b)
             for (int32_t h : c.heads) {
                 const int64_t off = ((int64_t)b * g.heads + h) * hb;
