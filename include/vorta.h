@@ -118,8 +118,9 @@ typedef struct {
     double flops_coreset_head;   /* 4 d (Lc + Lt)^2 */
     double flops_layer;          /* B * sum over heads, current routes */
     double flops_issued_layer;   /* what the tensor cores are really given (padding to 128-row blocks
-                                    and partial tiles included); 0 for a host-only plan */
-    int64_t n_work_items;        /* (head, query block) items in one launch; 0 for a host-only plan */
+                                    and partial tiles included; not the idle half of the pair kernel's
+                                    MMAs on a one-tile item); 0 for a host-only plan */
+    int64_t n_work_items;        /* (head, query block) items of a call's attention stage; 0 for a host-only plan */
     /* Algorithmic bytes of the memory-bound stages, per core-set (batch, head). */
     int64_t select_bytes_head;   /* L*dx*2 read + (Lc + L)*4 written, with dx = d */
     int64_t gather_bytes_head;   /* 3 * (Lc + Lt)*d*2 read and written */
@@ -255,8 +256,8 @@ VORTA_API int vorta_router_gates(const float *T_dev, const float *WR_dev, int32_
 /*
  * Soft mixture of the three branches (Section 3.3, Eq. 5: the forward pass used to
  * train the router): O[b, h] = g[h][0] full(.) + g[h][1] sliding(.) + g[h][2] coreset(.).
- * Every head runs all three branches in ONE attention launch (the plan's routes are
- * ignored), then the branch outputs are combined in fp32.
+ * Every head runs all three branches in one attention stage (one launch, or the two of
+ * VORTA_KERNEL_PAIR; the plan's routes are ignored), then the branch outputs are combined in fp32.
  *   gates_dev  f32 [heads, 3], device
  *   workspace  device, >= vorta_plan_info().mixture_workspace_bytes, 256-byte aligned
  * Core-set selection is on K of each head.  The first call builds the work list
