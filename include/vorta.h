@@ -220,7 +220,7 @@ VORTA_API int vorta_routed_attention(const vorta_plan *plan, const void *Q, cons
 /*
  * The same layer with HOST buffers (bf16 [B, heads, L, d]; pinned memory, or the
  * copies neither overlap nor return early).  The heads are worked through in up to
- * eight groups, most expensive first: the plan's own copy-in stream brings a group's
+ * twelve groups, most expensive first: the plan's own copy-in stream brings a group's
  * Q, K, V into dev_scratch, the layer's kernels for that group run on `stream` or on
  * a second kernel stream of the plan (groups alternate, so that one group's kernels
  * start in the SMs the previous group's last blocks leave), and the plan's copy-out

@@ -385,7 +385,7 @@ int build_list(vorta_plan *p, vorta_plan::WorkList &wl, const std::vector<uint8_
 // The first group's copy in and the last group's copy out are the only transfers nothing
 // overlaps, so the first groups are small (1, then 2 heads) and so is the last (1 head); the
 // heads between are split evenly.
-constexpr int kHostChunks = 8;
+constexpr int kHostChunks = 12;  // measured: 8 and 16 groups are 2 % slower end to end at hunyuan-720p
 
 std::vector<int32_t> host_chunk_sizes(int32_t heads)
 {
