@@ -84,7 +84,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, Ctl *ct
     return mbar_wait_slow(bar, parity, ctl, status, code);
 }
 
-// The same wait with a warp-uniform verdict, and a warp-uniform copy of a value all
+// The same wait with a warp-uniform result, and a warp-uniform copy of a value all
 // lanes hold: both come out of warp-wide reductions, which the compiler can keep in
 // uniform registers.  The MMA warp needs this: the operands of tcgen05.mma are uniform
 // registers, and only provably uniform values and control flow reach them without a
