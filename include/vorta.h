@@ -228,7 +228,9 @@ VORTA_API int vorta_routed_attention(const vorta_plan *plan, const void *Q, cons
  * `stream` ends up waiting for the last copy out: to the caller it is one operation
  * on `stream`.  Returns after enqueueing (synchronise `stream` before reading
  * O_host or reusing dev_scratch from another stream).  The result is the one
- * vorta_routed_attention gives.  dev_scratch: device memory of at least
+ * vorta_routed_attention gives (bit for bit under a fixed kernel choice; under
+ * VORTA_KERNEL_AUTO every group of heads makes its own choice, and a head served by
+ * another kernel than in the one-call path may differ in the last bf16 bit).  dev_scratch: device memory of at least
  * vorta_plan_info().host_call_scratch_bytes, 256-byte aligned.  Two calls on the
  * same plan must not be in flight on different streams at once (they share the
  * plan's copy streams and events).  The first call after plan creation or a route
