@@ -168,15 +168,16 @@ def test_many_slices_small_heads(d, kernel):
     p.close()
 
 
-def test_the_most_slices_the_library_takes():
+@pytest.mark.parametrize("d,kernel", [(64, vb.VORTA_KERNEL_TCGEN05), (128, vb.VORTA_KERNEL_PAIR)], ids=["d64-tcgen05", "d128-pair"])
+def test_the_most_slices_the_library_takes(d, kernel):
     """B * heads = 65 535 (the limit) heads of 12 tokens: the last slices of every stage."""
     heads = 65535
     routes = tuple(h % 3 for h in range(heads))
-    wl = Workload("max-slices", (1, 3, 4), heads, 64, (1, 2, 2), (1, 1, 1), 0.5, routes, 62, False)
+    wl = Workload("max-slices", (1, 3, 4), heads, d, (1, 2, 2), (1, 1, 1), 0.5, routes, 62, False)
     g = torch.Generator(device=DEV).manual_seed(62)
     Q, K, V = (torch.randn((1, heads, wl.L, wl.d), generator=g, device=DEV).to(torch.bfloat16) for _ in range(3))
     p = vb.Plan.from_workload(wl)
-    O = run_layer(p, wl, Q, K, V, vb.VORTA_KERNEL_TCGEN05)
+    O = run_layer(p, wl, Q, K, V, kernel)
     assert bool(torch.isfinite(O.float()).all())
     for h in (0, 1, 2, 32767, 32768, 65532, 65533, 65534):
         want = oracle_head_rows(wl, Q, K, V, 0, h, None)
