@@ -61,8 +61,8 @@ enum { VORTA_ROUTE_FULL = 0, VORTA_ROUTE_SLIDING = 1, VORTA_ROUTE_CORESET = 2 };
 enum {
     VORTA_PLAN_HOST_ONLY = 1, /* geometry and accounting only: needs no GPU, cannot launch */
     VORTA_PLAN_POOL_MERGE = 2 /* core-set heads: the centre's rows of Q, K, V become the mean over the
-                                 centre and the tokens pruned from its bucket before attending (Section 3.2,
-                                 "merged into the center"; the paper does not give the operator).  With a
+                                 centre and the tokens pruned from its bucket before attending (Section 3.2
+                                 mentions such a merge and does not give the operator).  With a
                                  bucket that keeps one token this is average pooling: bucket (2,1,1),
                                  (1,2,1) or (1,1,2) at ratio 0.5 are the AP variants of Section 4.2. */
 };
@@ -194,7 +194,11 @@ VORTA_API int32_t vorta_plan_kernel_in_use(const vorta_plan *plan);
  *                each bucket the centre first, then the other kept tokens ascending
  *   src_slot_dev int32 [B, Hx, L]  out: position in core_idx of the token whose
  *                attention output each token receives (its own, or its centre's)
- * Scores are evaluated in fp64 on the device.
+ * Precision of the scores: features of a width other than 128 are scored in fp64 (the
+ * products of bf16 values are exact there).  For dx == 128 the scores are first taken in
+ * fp32; a bucket in which two scores on either side of the keep/prune boundary lie within
+ * 2^-13 of each other, or whose norms leave the range fp32 handles safely, is scored again
+ * in fp64, so the decisions are the fp64 ones in both cases.
  */
 VORTA_API int vorta_coreset_select(const vorta_plan *plan, const void *X_dev, int32_t Hx, int32_t dx,
                                    int32_t *core_idx_dev, int32_t *src_slot_dev, void *stream);
@@ -211,7 +215,13 @@ VORTA_API int vorta_coreset_select(const vorta_plan *plan, const void *X_dev, in
  *   workspace    device, >= vorta_plan_info().workspace_bytes, 256-byte aligned
  *                (may be NULL when no head is routed to core-set); contents are
  *                scratch and undefined afterwards
+ * Hx is the head count of X (ignored when X is NULL).
  * Launch order on `stream`: select, gather, attention, scatter.
+ * Calls into this library on one device must be ordered with respect to each other (one
+ * stream, or streams chained by events): the attention stage is made of persistent kernels
+ * that each expect the whole GPU, and two of them from different calls running side by side
+ * have been seen to starve each other until a bounded wait gave up (the call then reports
+ * VORTA_ERR_TIMEOUT through vorta_device_status and O is incomplete).
  */
 VORTA_API int vorta_routed_attention(const vorta_plan *plan, const void *Q, const void *K,
                                      const void *V, void *O, const void *X_or_null, int32_t Hx,
@@ -282,7 +292,10 @@ VORTA_API int vorta_soft_mixture(vorta_plan *plan, const void *Q, const void *K,
  *   - The call itself allocates nothing (no cudaMalloc/cudaFree, no allocating
  *     library routine).  The first call on each device looks up the array's device
  *     address (cudaGetSymbolAddress with that device current); make that first call
- *     before starting any stream capture.
+ *     before starting any stream capture.  With CUDA's lazy module loading that look-up
+ *     is also the moment the driver sets the array's bytes aside on that device: on a
+ *     device with no room left it fails, the call returns VORTA_ERR_CUDA and launches
+ *     nothing.
  *   - All calls on a device share the one array.  It keeps whatever the last call
  *     left in it; nothing in it needs clearing, because every region is written
  *     before it is read within a call.  Two calls whose kernels overlap on the GPU

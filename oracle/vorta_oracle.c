@@ -4,15 +4,15 @@
  * A plain, slow, fp64 CPU statement of what VORTA's routed attention computes:
  * full 3D attention (Eq. 2), 3D sliding tile attention (Algorithm 1 of
  * Appendix A.1), and core-set attention = unpool . attn . pool with bucketed
- * core-set selection (Section 3.2 and Appendix A.1, "Bucketed coreset
- * selection").  It exists so that the CUDA library can be checked against
+ * core-set selection (Section 3.2 and the paragraph on it in Appendix
+ * A.1).  It exists so that the CUDA library can be checked against
  * something written straight from the paper.  It shares no code with the CUDA
  * path and is only used by the tests, by the smoke check and by the benchmark's
  * CPU-baseline leg.
  *
  * Conventions (the paper leaves them open; both sides use the same reading):
- *   - tokens are 0-based and frame-major: i = (t*H + h)*W + w  (Section 2,
- *     "flattened into a sequence of length L = F x H x W");
+ *   - tokens are 0-based and frame-major: i = (t*H + h)*W + w  (Section 2:
+ *     the frames x height x width latent is flattened into one sequence);
  *   - scores are scaled by `scale` (the caller passes 1/sqrt(d));
  *   - a video axis with fewer tiles than the window spans is unrestricted;
  *   - the similarity of bucketed core-set selection is the cosine;
@@ -60,8 +60,8 @@ static void token_coord(int64_t i, const int32_t v[3], int32_t c[3])
     c[0] = (int32_t)(i / ((int64_t)v[2] * v[1]));
 }
 
-/* Algorithm 1, "get tile id from token id": per-axis floor division. */
-static void get_tile_id_3d(int64_t i, const int32_t v[3], const int32_t t[3], int32_t q[3])
+/* Algorithm 1, first step: the 3D tile a token lies in (per-axis floor division). */
+static void tile_of_token(int64_t i, const int32_t v[3], const int32_t t[3], int32_t q[3])
 {
     int32_t c[3];
     token_coord(i, v, c);
@@ -74,13 +74,13 @@ static int32_t tiles_on_axis(const int32_t v[3], const int32_t t[3], int a)
 }
 
 /*
- * Algorithm 1, "all queries within the same window share the same tile id as
- * the window center tile id": the query's tile id is moved inward so that a
+ * Algorithm 1, second step: every query of a window takes the window's centre
+ * tile as its own, i.e. the query's tile id is moved inward so that a
  * window of w tiles centred on it stays inside the tile grid.  restricted[a]
  * is 0 when the grid has no more tiles on that axis than the window spans; the
  * window test is then skipped for the axis.
  */
-static void get_window_center_id(const int32_t q[3], const int32_t v[3], const int32_t t[3],
+static void window_centre_tile(const int32_t q[3], const int32_t v[3], const int32_t t[3],
                                  const int32_t w[3], int32_t c[3], int restricted[3])
 {
     for (int a = 0; a < 3; ++a) {
@@ -97,7 +97,7 @@ static void get_window_center_id(const int32_t q[3], const int32_t v[3], const i
     }
 }
 
-/* Algorithm 1, the three "abs(q - k) <= w/2" tests on tile ids. */
+/* Algorithm 1, third step: per axis, the centre tile and the key tile are at most half a window apart. */
 static int window_test(const int32_t c[3], const int32_t k[3], const int32_t w[3],
                        const int restricted[3])
 {
@@ -115,9 +115,9 @@ static int sta_mask_pair(int64_t i, int64_t j, const int32_t v[3], const int32_t
 {
     int32_t q[3], k[3], c[3];
     int restricted[3];
-    get_tile_id_3d(i, v, t, q);
-    get_tile_id_3d(j, v, t, k);
-    get_window_center_id(q, v, t, w, c, restricted);
+    tile_of_token(i, v, t, q);
+    tile_of_token(j, v, t, k);
+    window_centre_tile(q, v, t, w, c, restricted);
     return window_test(c, k, w, restricted);
 }
 
@@ -147,7 +147,7 @@ VO_API int vo_sta_block_mask(const int32_t v[3], const int32_t t[3], const int32
                         (int32_t)(qt % nt[2])};
         int32_t c[3];
         int restricted[3];
-        get_window_center_id(q, v, t, w, c, restricted);
+        window_centre_tile(q, v, t, w, c, restricted);
         for (int64_t kt = 0; kt < n; ++kt) {
             int32_t k[3] = {(int32_t)(kt / ((int64_t)nt[1] * nt[2])),
                             (int32_t)((kt / nt[2]) % nt[1]), (int32_t)(kt % nt[2])};
@@ -422,8 +422,8 @@ VO_API int64_t vo_coreset_select(const int32_t v[3], const int32_t b[3], double 
  * O is [nq, d].  Returns Lc, or -1 on allocation failure.
  */
 /*
- * merge != 0: the pruned tokens' information is merged into the centre (Section 3.2: "their
- * representational information is merged into the center"; the operator is not given -- the
+ * merge != 0: the pruned tokens' information is merged into the centre (Section 3.2 says so in
+ * one clause and does not give the operator -- the
  * reading here is the plain mean): the centre's rows of Q, K and V in the compact sequences
  * become the mean over the centre and the tokens pruned from its bucket.  With a bucket
  * that keeps one token this is average pooling (the AP variants of Section 4.2).
