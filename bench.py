@@ -2,6 +2,7 @@
 """Benchmark of one routed-attention layer (select + gather + attention + scatter).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+  python bench.py --sweep [--steps K]     the route-mix sweep with the speed-up over all-full attention
 
 A step is one call of vorta_routed_attention on one layer's Q/K/V (seeded
 synthetic, resident in HBM).  The line printed by rank 0 carries:
@@ -205,6 +206,26 @@ def whole_job_tflops(flops_per_rank_step: float, world: int, ms_per_step: float)
     return world * flops_per_rank_step / (ms_per_step * 1e-3) / 1e12
 
 
+def config_dict(wl, info, n_bytes_per_tensor: float, shard_heads: bool = False, mixture: bool = False):
+    """The `config` object of the JSON line: the same for the library's arm and the oracle's."""
+    return {"workload": wl.name + ("+soft-mixture" if mixture else ""), "grid": list(wl.grid),
+            "tokens": wl.L, "text_tokens": getattr(wl, "text", 0), "heads": wl.heads,
+            "d": wl.d, "tile": list(wl.tile), "window_tiles": list(wl.window),
+            "coreset_ratio": wl.ratio, "routes": list(wl.routes),
+            "heads_full_sliding_coreset": [info.n_full, info.n_sliding, info.n_coreset],
+            "algorithmic_tflop_per_layer": info.flops_layer / 1e12,
+            "l2": "inputs (3 x %.0f MB) larger than L2" % (n_bytes_per_tensor / 1e6),
+            "per_rank": ("heads of one layer split over the GPUs (vorta_shard_heads), no collective on the "
+                         "data path; roofline and stages are rank 0's share") if shard_heads
+            else "one layer per GPU, no collective on the data path"}
+
+
+def sharded_job_tflops(full_layer_flops: float, ms_per_step: float) -> float:
+    """--shard-heads (strong scaling): ONE layer whose heads are split over the ranks; the job's
+    throughput is the whole layer's work over the slowest rank's time."""
+    return full_layer_flops / (ms_per_step * 1e-3) / 1e12
+
+
 # ----------------------------------------------------------------------------- arms
 def run_reference(args):
     """The oracle as the timed arm: each step is a bounded sample of rows of the workload."""
@@ -230,11 +251,16 @@ def run_reference(args):
         secs += t
     value = flops / secs / 1e12
     sample = f"{rows} random query rows of each of {heads} heads per step, all their keys"
+    from paper_2505_18809_b200 import binding as vb
+    from paper_2505_18809_b200 import build as vbuild
+    vbuild.build()
+    host_plan = vb.Plan.from_workload(wl, host_only=True)   # geometry and FLOP accounting only: launches nothing
+    cfg = config_dict(wl, host_plan.info, Q.numel() * 2)
+    host_plan.close()
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic", "config": {"workload": wl.name, "grid": list(wl.grid), "heads": wl.heads,
-                                            "d": wl.d, "routes": list(wl.routes)},
+            "data": "synthetic", "config": cfg,
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -311,7 +337,8 @@ def run_ours(args):
         else:
             plan.routed_attention(Q, K, V, O, workspace=ws)
 
-    for _ in range(max(args.warmup, 3)):
+    warmup_run = max(args.warmup, 3)   # the timing rules ask for at least three
+    for _ in range(warmup_run):
         step()
     assert plan.device_status() == 0
 
@@ -321,24 +348,28 @@ def run_ours(args):
         sampler.start()
         time.sleep(0.3)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]   # between the steps: median and min
     barrier()
     t_wall0 = time.time()
     e0.record(stream)
     launches = 0
-    for _ in range(args.steps):
+    marks[0].record(stream)
+    for i in range(args.steps):
         step()
+        marks[i + 1].record(stream)
         launches += plan.last_launches()
     e1.record(stream)
     barrier()
     t_wall1 = time.time()
     ms_total = e0.elapsed_time(e1)
+    per_step = [marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps)]
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
     assert plan.device_status() == 0
     ms_total = reduce_max_ms(ms_total, world, dev)
     ms_step = ms_total / args.steps
     value = whole_job_tflops(flops_step, world, ms_step)
     if full_layer_flops is not None:
-        value = full_layer_flops / (ms_step * 1e-3) / 1e12   # the whole layer over the slowest rank's time
+        value = sharded_job_tflops(full_layer_flops, ms_step)
 
     # stage times of the timed steps (CUDA events recorded by the library on the same stream)
     n_hist = min(args.steps, 64)
@@ -400,23 +431,18 @@ def run_ours(args):
                  "scatter_gbs": gbs(n_core * info.scatter_bytes_head, st[3]),
                  "hbm_peak_gbs": pk["hbm"]}
         out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-               "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "ms_per_layer": ms_step,
+               "warmup": warmup_run, "ms_per_step": ms_step, "ms_per_layer": ms_step,
+               "ms_per_step_median": statistics.median(per_step), "ms_per_step_min": min(per_step),
                "higher_is_better": True, "scaling": "strong" if args.shard_heads else "weak", "vs_baseline": None,
                "dtype": "bf16",
                "data": "synthetic",
-               "config": {"workload": wl.name + ("+soft-mixture" if args.mixture else ""), "grid": list(wl.grid),
-                          "tokens": wl.L, "text_tokens": getattr(wl, "text", 0), "heads": wl.heads,
-                          "d": wl.d, "tile": list(wl.tile), "window_tiles": list(wl.window),
-                          "coreset_ratio": wl.ratio, "routes": list(wl.routes),
-                          "heads_full_sliding_coreset": [info.n_full, info.n_sliding, info.n_coreset],
-                          "algorithmic_tflop_per_layer": info.flops_layer / 1e12,
-                          "issued_tflop_per_layer": info.flops_issued_layer / 1e12,
-                          "l2": "inputs (3 x %.0f MB) larger than L2" % (Q.numel() * 2 / 1e6),
-                          "per_rank": ("heads of one layer split over the GPUs (vorta_shard_heads), no collective on the "
-                                       "data path; roofline and stages are rank 0's share") if args.shard_heads
-                          else "one layer per GPU, no collective on the data path"},
+               "config": config_dict(wl, info, Q.numel() * 2, args.shard_heads, args.mixture),
+               "issued_tflop_per_layer": info.flops_issued_layer / 1e12,
                "frac_of_bf16_peak": value / world / pk["bf16"],
                "roofline": roofline, "stages": stage, "gpu_launches": launches, "clocks": clocks}
+        if clocks and clocks.get("sm_mhz"):
+            # the run may sit on the power cap: time x clock tells a cycle win from a clock change
+            out["mcycles_per_step_at_sampled_clock"] = ms_step * clocks["sm_mhz"] * 1e-3   # ms x MHz = 1e3 cycles
 
     # ---- end to end through the host-buffer entry point (rank-local, max over ranks)
     e2e = None
@@ -427,7 +453,7 @@ def run_ours(args):
         for _ in range(2):
             plan.routed_attention_host(Qh, Kh, Vh, Oh, scratch)
         barrier()
-        n_e2e = max(2, min(args.steps, 5))
+        n_e2e = max(2, args.steps)
         e0.record(stream)
         for _ in range(n_e2e):
             plan.routed_attention_host(Qh, Kh, Vh, Oh, scratch)
@@ -435,7 +461,7 @@ def run_ours(args):
         barrier()
         ms_e2e = reduce_max_ms(e0.elapsed_time(e1) / n_e2e, world, dev)
         tb = Q.numel() * 2
-        e2e_value = (full_layer_flops / (ms_e2e * 1e-3) / 1e12 if full_layer_flops is not None
+        e2e_value = (sharded_job_tflops(full_layer_flops, ms_e2e) if full_layer_flops is not None
                      else whole_job_tflops(info.flops_layer, world, ms_e2e))
         e2e = {"value": e2e_value, "unit": UNIT,
                "ms_per_step": ms_e2e, "steps": n_e2e, "h2d_bytes_per_step": 3 * tb, "d2h_bytes_per_step": tb,
@@ -464,6 +490,80 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """The route-mix sweep on the HunyuanVideo-720p shape (full-head fraction 0 / .25 / .5 / 1, the rest
+    split evenly between sliding and core-set, core-set ratio .25 / .5; seeds 4-11): per point ms/layer,
+    effective TFLOP/s, fraction of the measured peak and the speed-up over the SAME kernels running all
+    24 heads as full attention.  One GPU; prints a table and one JSON line ({"sweep": [...]})."""
+    import dataclasses
+    import torch
+    from paper_2505_18809_b200 import binding as vb
+    from paper_2505_18809_b200 import build as vbuild
+    from paper_2505_18809_b200 import workloads
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA library has no CPU fallback")
+    torch.cuda.set_device(0)
+    dev = "cuda:0"
+    vbuild.build()
+    vb.lib()
+    pk = peaks()
+    stream = torch.cuda.current_stream()
+    points = workloads.route_mix_sweep()
+    ref = dataclasses.replace(points[0], name="hunyuan-720p-all-full", routes=(0,) * points[0].heads)
+    rows = []
+    sampler = ClockSampler(0)
+    sampler.start()
+    stamps = []
+    for wl in [ref] + points:
+        Q, K, V = workloads.make_qkv(wl, dev)
+        O = torch.empty_like(Q)
+        plan = vb.Plan.from_workload(wl)
+        if args.kernel >= 0:
+            plan.set_kernel(args.kernel)
+        info = plan.info
+        ws = plan.workspace(dev)
+        for _ in range(max(args.warmup, 3)):
+            plan.routed_attention(Q, K, V, O, workspace=ws)
+        assert plan.device_status() == 0
+        marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+        torch.cuda.synchronize()
+        t0 = time.time()
+        marks[0].record(stream)
+        for i in range(args.steps):
+            plan.routed_attention(Q, K, V, O, workspace=ws)
+            marks[i + 1].record(stream)
+        torch.cuda.synchronize()
+        t1 = time.time()
+        assert plan.device_status() == 0
+        per_step = [marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps)]
+        ms = marks[0].elapsed_time(marks[-1]) / args.steps
+        stamps.append((t0, t1))
+        rows.append({"workload": wl.name, "heads_full_sliding_coreset": [info.n_full, info.n_sliding, info.n_coreset],
+                     "coreset_ratio": wl.ratio, "seed": wl.seed, "algorithmic_tflop": info.flops_layer / 1e12,
+                     "ms_per_layer": ms, "ms_median": statistics.median(per_step), "ms_min": min(per_step),
+                     "tflops": info.flops_layer / (ms * 1e-3) / 1e12,
+                     "frac_of_bf16_peak": info.flops_layer / (ms * 1e-3) / 1e12 / pk["bf16"],
+                     "kernel_in_use": plan.kernel_in_use()})
+        plan.close()
+        del Q, K, V, O, ws
+        torch.cuda.empty_cache()
+    all_full_ms = rows[0]["ms_per_layer"]
+    for r, (t0, t1) in zip(rows, stamps):
+        r["speedup_vs_all_full"] = all_full_ms / r["ms_per_layer"]
+    clocks = sampler.stop(stamps[0][0], stamps[-1][1])
+    print("| workload | full/sliding/core-set | r | TFLOP | ms/layer (median, min) | TFLOP/s | of peak | speed-up vs all-full |",
+          file=sys.stderr)
+    print("|---|---|---|---|---|---|---|---|", file=sys.stderr)
+    for r in rows:
+        f, s_, c = r["heads_full_sliding_coreset"]
+        print(f"| {r['workload']} | {f}/{s_}/{c} | {r['coreset_ratio']:g} | {r['algorithmic_tflop']:.2f} | "
+              f"{r['ms_per_layer']:.2f} ({r['ms_median']:.2f}, {r['ms_min']:.2f}) | {r['tflops']:.0f} | "
+              f"{100 * r['frac_of_bf16_peak']:.1f} % | {r['speedup_vs_all_full']:.2f}x |", file=sys.stderr)
+    print(json.dumps({"metric": METRIC, "unit": UNIT, "sweep": rows, "steps": args.steps, "warmup": max(args.warmup, 3),
+                      "peak": pk["bf16"], "peak_source": f"{pk['source']} burst bf16", "clocks": clocks,
+                      "dtype": "bf16", "data": "synthetic"}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -479,11 +579,15 @@ def main():
                     help="core-set heads merge the pruned tokens into their centre (mean) before attention")
     ap.add_argument("--shard-heads", action="store_true",
                     help="strong scaling: one layer, heads split over the ranks (default: one layer per rank)")
+    ap.add_argument("--sweep", action="store_true",
+                    help="the route-mix sweep on the HunyuanVideo-720p shape, with the speed-up over all-full attention")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.sweep:
+        run_sweep(args)
     else:
         run_ours(args)
 

@@ -64,11 +64,96 @@ def sample_rows(wl, n: int, seed: int) -> np.ndarray:
     return np.asarray(rows, dtype=np.int64)
 
 
-def assert_close(got_rows: torch.Tensor, want: np.ndarray, what: str):
+def _spread(g, members: np.ndarray, k: int) -> list:
+    """k members of a sorted index array, one from each of k equal stretches of it
+    (all of them if there are no more than k)."""
+    n = len(members)
+    if n <= k:
+        return [int(e) for e in members]
+    edges = np.linspace(0, n, k + 1).astype(np.int64)
+    return [int(members[int(g.integers(edges[i], max(edges[i] + 1, edges[i + 1])))]) for i in range(k)]
+
+
+def stratified_rows(wl, route: int, n: int, seed: int, core_idx=None, src_slot=None) -> np.ndarray:
+    """At least ~n query rows of one head, chosen so that every unit of work of the head
+    and every kind of row the route knows is hit, not merely likely to be:
+
+    full head      every block of 128 consecutive rows (so every 256-row work item, both of
+                   its query tiles, the first and the last item of the head and its short
+                   tail block) gets the same number of rows;
+    sliding head   every tile gets the same number of rows, spread over the tile in raster
+                   order (so both boxes of a 256-token tile, every partial-tile class -- cut
+                   on T, on H, on W and the corners -- and every tile whose window is shifted
+                   inward at a border of any axis), plus the grid's corner tokens;
+    core-set head  (core_idx, src_slot are the oracle's) every block of 128 compact rows gets
+                   the same number of kept tokens, bucket centres and other kept tokens alike;
+                   then as many pruned tokens, spread over the sequence, and for a share of
+                   them the centre they copy, so that pruned row and centre row are both read;
+    text tokens    the first, the last and a few random ones, for every route.
+    """
+    T, H, W = wl.grid
+    L, text = wl.L, getattr(wl, "text", 0)
+    g = np.random.default_rng(seed)
+    rows = {0, L - 1, W - 1, (H - 1) * W, (T - 1) * H * W, L // 2}
+    if route == 0:
+        nblk = -(-L // 128)
+        k = max(2, -(-n // nblk))
+        for b in range(nblk):
+            rows |= set(_spread(g, np.arange(b * 128, min(L, b * 128 + 128)), k))
+    elif route == 1:
+        t_, h_, w_ = wl.tile
+        nt = [-(-T // t_), -(-H // h_), -(-W // w_)]
+        k = max(3, -(-n // (nt[0] * nt[1] * nt[2])))
+        for qt in range(nt[0]):
+            for qh in range(nt[1]):
+                for qw in range(nt[2]):
+                    tt = np.arange(qt * t_, min(T, qt * t_ + t_))
+                    hh = np.arange(qh * h_, min(H, qh * h_ + h_))
+                    ww = np.arange(qw * w_, min(W, qw * w_ + w_))
+                    tok = ((tt[:, None, None] * H + hh[None, :, None]) * W + ww[None, None, :]).reshape(-1)
+                    rows |= set(_spread(g, tok, k))
+    else:
+        assert core_idx is not None and src_slot is not None
+        Lc = len(core_idx)
+        own = np.asarray(core_idx)[np.asarray(src_slot)] == np.arange(L)   # token kept (it is its own slot)
+        nblk = -(-Lc // 128)
+        k = max(2, -(-(n // 2) // nblk))
+        for b in range(nblk):
+            rows |= {int(core_idx[s]) for s in _spread(g, np.arange(b * 128, min(Lc, b * 128 + 128)), k)}
+        pruned = np.flatnonzero(~own)
+        if len(pruned):
+            take = _spread(g, pruned, max(4, n // 2))
+            rows |= set(take)
+            rows |= {int(core_idx[src_slot[i]]) for i in take[::4]}        # the centres some of them copy
+        centres = np.unique(np.asarray(src_slot)[~own]) if len(pruned) else np.zeros(0, np.int64)
+        is_centre = np.zeros(Lc, bool)
+        is_centre[centres] = True
+        got = np.asarray(sorted(rows))
+        slots = np.asarray(src_slot)[got]
+        kinds = {"centre": bool((own[got] & is_centre[slots]).any()) or not len(pruned),
+                 "kept non-centre": bool((own[got] & ~is_centre[slots]).any()) or bool(is_centre.all()),
+                 "pruned": bool((~own[got]).any()) or not len(pruned)}
+        assert all(kinds.values()), kinds
+    if text:
+        rows |= {L, L + text - 1} | {L + int(e) for e in g.integers(0, text, size=6)}
+    return np.asarray(sorted(rows), dtype=np.int64)
+
+
+def assert_close(got_rows: torch.Tensor, want: np.ndarray, what: str, stats: dict = None):
+    """The parity bars of the task, per call (one head).  stats, if given, collects the worst
+    absolute and RELATIVE figures seen (max-abs / max |O| and mean-abs / mean |O| of the head's
+    rows): the bars are absolute, the relative figures say how much of the signal they are."""
     got = got_rows.detach().to("cpu", torch.float64).numpy()
     assert got.shape == want.shape, (got.shape, want.shape)
     assert np.isfinite(got).all(), f"{what}: non-finite output"
     err = np.abs(got - want)
     assert err.max() <= MAX_ABS_TOL, f"{what}: max-abs {err.max():.3e} > {MAX_ABS_TOL}"
     assert err.mean() <= MEAN_ABS_TOL, f"{what}: mean-abs {err.mean():.3e} > {MEAN_ABS_TOL}"
+    if stats is not None:
+        mag = np.abs(want)
+        stats["max_abs"] = max(stats.get("max_abs", 0.0), float(err.max()))
+        stats["mean_abs"] = max(stats.get("mean_abs", 0.0), float(err.mean()))
+        stats["rel_max"] = max(stats.get("rel_max", 0.0), float(err.max() / max(mag.max(), 1e-30)))
+        stats["rel_mean"] = max(stats.get("rel_mean", 0.0), float(err.mean() / max(mag.mean(), 1e-30)))
+        stats["rows"] = stats.get("rows", 0) + got.shape[0]
     return float(err.max()), float(err.mean())

@@ -49,6 +49,48 @@ def test_two_ranks_report_the_slowest_time_and_the_aggregate():
     assert abs(value - 2 * 53.45e12 / 52.5e-3 / 1e12) < 1e-9
 
 
+def _shard_worker(rank, world, port, out):
+    """bench.py --shard-heads on CPU: the partition the library gives, every rank's own share of the
+    layer's work, a time proportional to that share, the slowest rank's time, the whole layer over it."""
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_2505_18809_b200 import binding as vb, sharding, workloads
+    wl = workloads.config("hunyuan-720p")
+    host_plan = vb.Plan.from_workload(wl, host_only=True)
+    full = host_plan.info.flops_layer
+    host_plan.close()
+    rank_of_head, rank_flops = sharding.shard_heads(wl, world)
+    local = sharding.local_workload(wl, sharding.heads_of_rank(rank_of_head, rank))
+    local_plan = vb.Plan.from_workload(local, host_only=True)
+    mine = local_plan.info.flops_layer
+    local_plan.close()
+    local_ms = mine / 1.0e15 * 1e3                       # every rank at 1000 TFLOP/s
+    ms = bench.reduce_max_ms(local_ms, world, "cpu")
+    value = bench.sharded_job_tflops(full, ms)
+    dist.barrier()
+    out[rank] = (mine, float(rank_flops[rank]), full, ms, value)
+    dist.destroy_process_group()
+
+
+def test_two_ranks_sharding_one_layer_report_the_whole_layer_over_the_slowest_rank():
+    world, port = 2, _free_port()
+    with mp.Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(_shard_worker, args=(world, port, out), nprocs=world, join=True)
+        res = dict(out)
+    mine = [res[r][0] for r in range(world)]
+    full, ms, value = res[0][2], res[0][3], res[0][4]
+    for r in range(world):
+        assert res[r][0] == pytest.approx(res[r][1], rel=1e-12)     # the rank's plan counts what the partition promised
+        assert res[r][2:] == res[0][2:]                             # both ranks report the same job figures
+    assert sum(mine) == pytest.approx(full, rel=1e-12)              # the shares add up to the layer
+    assert ms == pytest.approx(max(mine) / 1.0e15 * 1e3, rel=1e-12)
+    # strong scaling: the whole layer over the slowest rank; below world x the per-rank rate by the imbalance
+    assert value == pytest.approx(full / max(mine) * 1000.0, rel=1e-12)
+    assert 1000.0 < value <= 1000.0 * world
+
+
 def test_single_rank_needs_no_process_group():
     assert bench.reduce_max_ms(7.0, 1, "cpu") == 7.0
     assert abs(bench.whole_job_tflops(1e12, 1, 1.0) - 1000.0) < 1e-9
