@@ -28,7 +28,11 @@ attention_simt_kernel(AttnParams p)
     const float scale = p.scale_log2 * 0.6931471805599453f;
 
     int32_t qtok = 0;
-    const bool q_valid = mblk < w.n_mblk && block_row_token(g, w.mode, w.q_org[mblk], w.kv_len, r, &qtok);
+    // packed item: rows 0-63 of the one query block are the first tile's, rows 64-127 the second's
+    const bool packed = (w.flags & kItemPacked) != 0;
+    const uint32_t my_vis = packed ? 1u + (uint32_t)(r >> 6) : 0u;
+    const bool q_valid = mblk < w.n_mblk &&
+                         block_row_token(g, w.mode, w.q_org[packed ? (r >> 6) : mblk], w.kv_len, packed ? (r & 63) : r, &qtok);
     __nv_bfloat162 q[D / 2];  // packed: the row and its accumulator must both fit in registers
     float acc[D];
 #pragma unroll
@@ -47,15 +51,18 @@ attention_simt_kernel(AttnParams p)
         // the last kv_text blocks of a sliding item are runs of bn_tile text tokens (rows L + ...)
         const bool text = w.mode == MODE_TILES && j >= w.kv_count - w.kv_text;
         int32_t kv_mode = w.mode, kv_len = w.kv_len;
+        uint32_t vis = 0;  // packed items: which of the two tiles sees the block (0: both)
         if (text) {
             kv_mode = MODE_LINEAR;
             kv_len = g.Ltot;
             org[0] = g.L + (j - (w.kv_count - w.kv_text)) * g.bn_tile; org[1] = 0; org[2] = 0;
         } else if (w.mode == MODE_TILES) {
-            KvEntry e = p.kv_list[w.kv_begin + j];
+            KvEntry e = (packed ? p.kv_pairs : p.kv_list)[w.kv_begin + j];
             org[0] = e.w0; org[1] = e.h0; org[2] = e.t0;
-            if (e.mask_id)
-                for (int i = 0; i < 4; ++i) mask[i] = p.colmasks[e.mask_id * 4 + i];
+            vis = e.mask_id >> kVisShift;
+            const uint32_t id = e.mask_id & kMaskIdBits;
+            if (id)
+                for (int i = 0; i < 4; ++i) mask[i] = p.colmasks[id * 4 + i];
         } else {
             org[0] = j * kBlockM; org[1] = 0; org[2] = 0;
         }
@@ -81,7 +88,7 @@ attention_simt_kernel(AttnParams p)
                 *reinterpret_cast<uint4 *>(&sV[n][c * 8]) = vv;
             }
             __syncthreads();
-            if (!q_valid) continue;
+            if (!q_valid || (vis && vis != my_vis)) continue;
             for (int n = 0; n < kKvChunk; ++n) {
                 if (sTok[n] < 0) continue;
                 float s = 0.f;

@@ -150,11 +150,22 @@ __device__ __forceinline__ void kv_block_coords(const AttnParams &p, const WorkI
     if (text) {
         c1 = (j - (w.kv_count - w.kv_text)) * p.g.bn_tile; c2 = 0; c3 = 0; mask_id = 0;
     } else if (w.mode == MODE_TILES) {
-        const KvEntry e = p.kv_list[w.kv_begin + j];
-        c1 = e.w0; c2 = e.h0; c3 = e.t0; mask_id = e.mask_id;
+        const KvEntry e = ((w.flags & kItemPacked) ? p.kv_pairs : p.kv_list)[w.kv_begin + j];
+        c1 = e.w0; c2 = e.h0; c3 = e.t0; mask_id = e.mask_id & kMaskIdBits;
     } else {
         c1 = j * kBlockM; c2 = 0; c3 = 0; mask_id = 0;
     }
+}
+
+// A KV block of n keys (a multiple of 16, at most 128) of an item worked through as `spb` sub-blocks
+// per block: the widths of the two sub-blocks.  With two sub-blocks per block both get at least 16
+// columns (a block of 16 keys gets a second sub-block of 16 columns that are no keys).
+__host__ __device__ __forceinline__ void split_block(int32_t n, int32_t spb, int32_t &w0, int32_t &w1)
+{
+    if (spb == 1) { w0 = n; w1 = 0; }
+    else if (n > 64) { w0 = 64; w1 = n - 64; }
+    else if (n >= 32) { w0 = ((n >> 1) + 15) & ~15; w1 = n - w0; }
+    else { w0 = 16; w1 = 16; }
 }
 
 // write the packed P words of a sub-block of `width` keys to the first width/2 columns at t_p
@@ -187,18 +198,30 @@ __device__ __forceinline__ void producer_role(const AttnParams &p, const AttnMap
         const uint32_t half_bytes = rows * 128u;
         if (!mbar_wait(bars + 8 * BAR_Q_EMPTY, (it & 1) ^ 1, ctl, p.status, 101)) return;
         if (lane == 0) {
-            mbar_expect_tx(bars + 8 * BAR_Q_FULL, half_bytes * kHalves * w.n_mblk);
-            for (int m = 0; m < w.n_mblk; ++m)
-                for (int h = 0; h < kHalves; ++h)
-                    tma_load_5d(smem_base + kSmemQ + m * kTileBytes + h * kHalfBytes, &maps.q[w.mode],
-                                bars + 8 * BAR_Q_FULL, h * 64, w.q_org[m][0], w.q_org[m][1], w.q_org[m][2], w.slice);
+            if (w.flags & kItemPacked) {
+                // two tiles of at most 64 tokens in one query block: the second one 64 rows further down
+                mbar_expect_tx(bars + 8 * BAR_Q_FULL, half_bytes * kHalves * 2);
+                for (int t = 0; t < 2; ++t)
+                    for (int h = 0; h < kHalves; ++h)
+                        tma_load_5d(smem_base + kSmemQ + h * kHalfBytes + t * (kHalfBytes / 2), &maps.q[w.mode],
+                                    bars + 8 * BAR_Q_FULL, h * 64, w.q_org[t][0], w.q_org[t][1], w.q_org[t][2], w.slice);
+            } else {
+                mbar_expect_tx(bars + 8 * BAR_Q_FULL, half_bytes * kHalves * w.n_mblk);
+                for (int m = 0; m < w.n_mblk; ++m)
+                    for (int h = 0; h < kHalves; ++h)
+                        tma_load_5d(smem_base + kSmemQ + m * kTileBytes + h * kHalfBytes, &maps.q[w.mode],
+                                    bars + 8 * BAR_Q_FULL, h * 64, w.q_org[m][0], w.q_org[m][1], w.q_org[m][2], w.slice);
+            }
         }
         for (int32_t j = 0; j < w.kv_count; ++j) {
             int32_t c1, c2, c3;
             uint32_t mask_id;
             bool text;
             kv_block_coords(p, w, j, c1, c2, c3, mask_id, text);
-            const uint32_t kv_bytes = (text ? (uint32_t)p.g.bn_tile * 128u : half_bytes) * kHalves;
+            // a box the grid cuts is fetched as its part inside the grid: a short run of real keys
+            const uint32_t shape = (!text && w.mode == MODE_TILES) ? p.cls_shape[mask_id] : 0u;
+            const uint32_t kv_bytes = (text ? (uint32_t)p.g.bn_tile * 128u
+                                            : (shape ? (uint32_t)p.shape_rows[shape] * 128u : half_bytes)) * kHalves;
 #pragma unroll
             for (int kv = 0; kv < 2; ++kv) {
                 const uint32_t slot = kv_it % kStages;
@@ -207,7 +230,8 @@ __device__ __forceinline__ void producer_role(const AttnParams &p, const AttnMap
                     const uint32_t full = bars + 8 * (BAR_KV_FULL + slot);
                     mbar_expect_tx(full, kv_bytes);
                     const CUtensorMap *map = text ? (kv == 0 ? &maps.kt : &maps.vt)
-                                                  : (kv == 0 ? &maps.k[w.mode] : &maps.v[w.mode]);
+                                             : shape ? (kv == 0 ? &maps.k_cut[shape] : &maps.v_cut[shape])
+                                                     : (kv == 0 ? &maps.k[w.mode] : &maps.v[w.mode]);
                     for (int h = 0; h < kHalves; ++h)
                         tma_load_5d(smem_base + kSmemKV + slot * kTileBytes + h * kHalfBytes, map, full, h * 64, c1,
                                     c2, c3, w.slice);
@@ -237,7 +261,6 @@ __device__ __forceinline__ void mma_role(const AttnParams &p, Ctl *ctl, uint32_t
     const uint64_t k_desc0 = smem_desc(smem_base + kSmemKV, 16, 1024);          // K-major
     const uint64_t v_desc0 = smem_desc(smem_base + kSmemKV, kHalfBytes, 1024);  // MN-major
     constexpr uint64_t kTileStep = kTileBytes >> 4;
-    constexpr uint64_t kSubStep = (64 * 128) >> 4;  // 64 keys further down a K or V tile
     const uint32_t idesc_pv = instr_desc((uint32_t)D, 1);
 
     auto wait_kv = [&](uint32_t pos, int32_t code) {
@@ -245,9 +268,10 @@ __device__ __forceinline__ void mma_role(const AttnParams &p, Ctl *ctl, uint32_t
     };
     auto free_kv = [&](uint32_t pos) { tc_commit(bars + 8 * (BAR_KV_EMPTY + pos % kStages), leader); };
     // S_m[buffer b] = Q_m K^T over sub-block h of the K block at ring position pos (16 channels per MMA)
-    auto issue_qk = [&](int m, uint32_t pos, int b, int h, uint32_t idesc) {
+    // (koff: where the sub-block starts in its K or V block, in 16-byte units: 8 per key)
+    auto issue_qk = [&](int m, uint32_t pos, int b, uint32_t koff, uint32_t idesc) {
         const uint64_t qa = q_desc0 + (uint64_t)m * kTileStep;
-        const uint64_t kb = k_desc0 + (uint64_t)(pos % kStages) * kTileStep + (uint64_t)h * kSubStep;
+        const uint64_t kb = k_desc0 + (uint64_t)(pos % kStages) * kTileStep + (uint64_t)koff;
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
             const uint64_t off = (uint64_t)(((kk / 4) * kHalfBytes + (kk % 4) * 32) >> 4);
@@ -255,8 +279,8 @@ __device__ __forceinline__ void mma_role(const AttnParams &p, Ctl *ctl, uint32_t
         }
     };
     // O_m (+)= P_m[buffer b] V over sub-block h of the V block at pos (16 keys per MMA)
-    auto issue_pv = [&](int m, uint32_t pos, int b, int h, int ksteps, bool first) {
-        const uint64_t vb = v_desc0 + (uint64_t)(pos % kStages) * kTileStep + (uint64_t)h * kSubStep;
+    auto issue_pv = [&](int m, uint32_t pos, int b, uint32_t koff, int ksteps, bool first) {
+        const uint64_t vb = v_desc0 + (uint64_t)(pos % kStages) * kTileStep + (uint64_t)koff;
 #pragma unroll
         for (int i = 0; i < 4; ++i)
             if (i < ksteps)
@@ -271,17 +295,50 @@ __device__ __forceinline__ void mma_role(const AttnParams &p, Ctl *ctl, uint32_t
         const int32_t nm = (int32_t)uniform_u32((uint32_t)w->n_mblk);
         const int32_t spb = bn > 64 ? 2 : 1;  // sub-blocks per KV block
         const int32_t n_sub = n * spb;
-        const int32_t width0 = min(bn, 64), width1 = max(bn - 64, 16);
-        const uint32_t idesc_qk0 = instr_desc((uint32_t)width0, 0), idesc_qk1 = instr_desc((uint32_t)width1, 0);
+        int32_t width0, width1;
+        split_block(bn, spb, width0, width1);
+        // Sub-block widths of block j.  The boxes a sliding item lists after its kv_fast whole ones may be
+        // short (the part of a cut box inside the grid): their key count comes from the box's class.
+        const bool tiles = uniform_u32((uint32_t)w->mode) == MODE_TILES;
+        const int32_t first_cut = tiles ? (int32_t)uniform_u32((uint32_t)w->kv_fast) : n;
+        const int32_t n_boxes = n - (tiles ? (int32_t)uniform_u32((uint32_t)w->kv_text) : 0);
+        const KvEntry *entries = (uniform_u32((uint32_t)w->flags) & kItemPacked ? p.kv_pairs : p.kv_list) +
+                                 (tiles ? (int32_t)uniform_u32((uint32_t)w->kv_begin) : 0);
+        // The classes of 32 consecutive blocks are fetched with one load (lane l holds block tab_first + l)
+        // and handed round by shuffle: a load per block would put a trip to global memory on this warp's
+        // path every time a cut box comes up.
+        int32_t tab_first = -1;
+        uint32_t tab_shape = 0;
+        auto block_widths = [&](int32_t j, int32_t &w0, int32_t &w1) {
+            w0 = width0;
+            w1 = width1;
+            if (j >= first_cut && j < n_boxes) {
+                if (tab_first < 0 || j < tab_first || j >= tab_first + 32) {
+                    tab_first = j;
+                    const int32_t mine = j + (int32_t)(threadIdx.x & 31);
+                    tab_shape = mine < n_boxes ? (uint32_t)p.cls_shape[entries[mine].mask_id & kMaskIdBits] : 0u;
+                }
+                const uint32_t shape = uniform_u32(__shfl_sync(0xffffffffu, tab_shape, j - tab_first));
+                if (shape) {
+                    split_block((int32_t)uniform_u32((uint32_t)((p.shape_rows[shape] + 15) & ~15)), spb, w0, w1);
+                    w0 = (int32_t)uniform_u32((uint32_t)w0);
+                    w1 = (int32_t)uniform_u32((uint32_t)w1);
+                }
+            }
+        };
+        const uint32_t idesc_qk0 = instr_desc((uint32_t)width0, 0), idesc_qk1 = instr_desc((uint32_t)max(width1, 16), 0);
+        int32_t kj = -1, kw0 = 0, kw1 = 0, vj = -1, vw0 = 0, vw1 = 0;  // widths of the K / V block in hand
 
         if (!mbar_wait_uniform(bars + 8 * BAR_Q_FULL, it & 1, ctl, p.status, 201)) return;
         // the first two score sub-blocks of both tiles
         for (int32_t u = 0; u < min(n_sub, 2); ++u) {
             const int32_t j = u / spb, h = u - j * spb;
+            if (j != kj) { block_widths(j, kw0, kw1); kj = j; }
             if (h == 0 && !wait_kv(kv_base + 2 * j, 202)) return;
             tc_fence_after();
+            const uint32_t idesc = instr_desc((uint32_t)(h ? kw1 : kw0), 0);
             for (int m = 0; m < nm; ++m) {
-                issue_qk(m, kv_base + 2 * j, u & 1, h, h ? idesc_qk1 : idesc_qk0);
+                issue_qk(m, kv_base + 2 * j, u & 1, h ? (uint32_t)kw0 * 8u : 0u, idesc);
                 tc_commit(bars + 8 * (BAR_S_FULL + 2 * m + (u & 1)), leader);
             }
             if (h == spb - 1) free_kv(kv_base + 2 * j);
@@ -293,6 +350,18 @@ __device__ __forceinline__ void mma_role(const AttnParams &p, Ctl *ctl, uint32_t
             const int32_t u2 = u + 2, jk = u2 / spb, h2 = u2 - jk * spb;
             const bool has2 = u2 < n_sub;
             const uint32_t pos_v = kv_base + 2 * jv + 1, pos_k = kv_base + 2 * jk;
+            // blocks before the item's first cut box (all of them, for most items) keep the item's constants
+            uint32_t idesc_k = h2 ? idesc_qk1 : idesc_qk0, koff_k = h2 ? (uint32_t)width0 * 8u : 0u;
+            uint32_t koff_v = h ? (uint32_t)width0 * 8u : 0u;
+            int32_t ksteps_v = (h ? width1 : width0) >> 4;
+            if (max(jv, has2 ? jk : 0) >= first_cut) {
+                if (jv != vj) { block_widths(jv, vw0, vw1); vj = jv; }
+                if (has2 && jk != kj) { block_widths(jk, kw0, kw1); kj = jk; }
+                idesc_k = instr_desc((uint32_t)(h2 ? kw1 : kw0), 0);
+                koff_k = h2 ? (uint32_t)kw0 * 8u : 0u;
+                koff_v = h ? (uint32_t)vw0 * 8u : 0u;
+                ksteps_v = (h ? vw1 : vw0) >> 4;
+            }
             if (h == 0 && !wait_kv(pos_v, 203)) return;
             if (has2 && h2 == 0 && !wait_kv(pos_k, 206)) return;
             for (int m = 0; m < nm; ++m) {
@@ -305,8 +374,8 @@ __device__ __forceinline__ void mma_role(const AttnParams &p, Ctl *ctl, uint32_t
                 }
                 tc_fence_after();
                 if (leader) TRACE(m, u, 0);
-                issue_pv(m, pos_v, b, h, (h ? width1 : width0) >> 4, u == 0);
-                if (has2) issue_qk(m, pos_k, b, h2, h2 ? idesc_qk1 : idesc_qk0);
+                issue_pv(m, pos_v, b, koff_v, ksteps_v, u == 0);
+                if (has2) issue_qk(m, pos_k, b, koff_k, idesc_k);
                 // S(u+2) is ready; and, for the lazy rescale and the epilogue: PV(u) is done
                 tc_commit(bars + 8 * (BAR_S_FULL + 2 * m + b), leader);
                 if (leader) TRACE(m, u, 1);
@@ -338,32 +407,30 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
         const WorkItem *wp = p.items + begin + it;
         if (m >= wp->n_mblk) continue;
         const int32_t w_mode = wp->mode, w_kv_len = wp->kv_len, w_kv_count = wp->kv_count;
-        const KvEntry *kv_entries = p.kv_list + wp->kv_begin;
+        const bool packed = (wp->flags & kItemPacked) != 0;
+        const KvEntry *kv_entries = (packed ? p.kv_pairs : p.kv_list) + wp->kv_begin;
+        // packed item: this row belongs to the first (rows 0-63) or the second tile; a block that only the
+        // other tile has in its window holds no key for it (visibility code in the entry's top bits)
+        const uint32_t my_vis = packed ? 1u + (uint32_t)(row >> 6) : 0u;
         const bool has_text = w_mode == MODE_TILES && wp->kv_text > 0;
         const int32_t n_boxes = has_text ? w_kv_count - wp->kv_text : w_kv_count;  // the rest: text-token blocks
         const int32_t bn = w_mode == MODE_TILES ? p.g.bn_tile : kBlockM;
         const int32_t sh = bn > 64 ? 1 : 0;  // log2 of the sub-blocks per KV block
         const int32_t n_sub = w_kv_count << sh;
-        const int32_t width0 = min(bn, 64), width1 = bn - 64;
+        int32_t width0, width1;
+        split_block(bn, 1 << sh, width0, width1);
         // columns of a short block: every block of a sliding head whose tile has fewer than 128
         // tokens, else the last block of the sequence
         const int32_t tail_valid = w_mode == MODE_TILES ? bn : w_kv_len - (w_kv_count - 1) * kBlockM;
         const bool tail_partial = tail_valid < kBlockM;
-        uint32_t tail_mask[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int32_t v = min(max(tail_valid - 32 * i, 0), 32);
-            tail_mask[i] = v == 32 ? 0xffffffffu : ((1u << v) - 1u);
-        }
         float row_max = -INFINITY, row_sum = 0.f;
 
         // wait for S(u) and read this thread's row of it (all 64 columns, or `width` of them)
-        auto load_sub = [&](auto full, int32_t u, uint32_t(&s)[64]) -> bool {
+        auto load_sub = [&](auto full, int32_t u, int32_t width, uint32_t(&s)[64]) -> bool {
             const int32_t b = u & 1;
             if (!mbar_wait(bars + 8 * (BAR_S_FULL + 2 * m + b), (s_par >> b) & 1, ctl, p.status, 301 + m)) return false;
             s_par ^= 1u << b;
             tc_fence_after();
-            const int32_t width = decltype(full)::value ? 64 : ((u & sh) ? width1 : width0);
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 uint32_t(&chunk)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[32 * c]);
@@ -372,36 +439,60 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
             tc_wait_ld();
             return true;
         };
-        // strike the columns of sub-block u that are not keys (mask class `id` of its block,
-        // fetched ahead by the caller; blocks of text tokens have none: their last one is cut at Lt)
-        auto apply_mask = [&](auto with_text, int32_t u, uint32_t id, uint32_t(&s)[64]) {
-            const int32_t h = u & sh;
-            uint32_t m0 = 0, m1 = 0;
-            bool partial = false;
-            if (decltype(with_text)::value && (u >> sh) >= n_boxes) {
-                // text keys of this sub-block: what is left of Lt, at most the block's bn columns
-                const int32_t valid = min(p.g.Lt - ((u >> sh) - n_boxes) * bn, bn) - 64 * h;
-                if (valid < 64) {
-                    const int32_t v0 = min(max(valid, 0), 32), v1 = min(max(valid - 32, 0), 32);
-                    m0 = v0 == 32 ? 0xffffffffu : ((1u << v0) - 1u);
-                    m1 = v1 == 32 ? 0xffffffffu : ((1u << v1) - 1u);
-                    partial = true;
-                }
+        // Sub-block u of the generic path: its width in columns, how many of its leading columns are
+        // keys (64 and more: all that the registers hold), and the class whose column mask applies
+        // instead (0: none).  id: mask class of the sub-block's KV block (0 for whole boxes and for the
+        // linear modes), fetched ahead by the caller.
+        //   text-token block      the last one is cut at Lt;
+        //   box the grid cuts     fetched as its part inside the grid, a short run of real keys
+        //                         (classes without such a map keep the whole box and a column mask);
+        //   tile under 128 tokens / last block of a sequence: a prefix of the block.
+        auto sub_dims = [&](auto with_text, int32_t u, uint32_t raw_id, int32_t &width, int32_t &valid, uint32_t &mask_id) {
+            const int32_t j = u >> sh, h = u & sh;
+            const uint32_t id = raw_id & kMaskIdBits, vis = raw_id >> kVisShift;
+            width = h ? width1 : width0;
+            valid = 64;
+            mask_id = 0;
+            if (decltype(with_text)::value && j >= n_boxes) {
+                valid = min(p.g.Lt - (j - n_boxes) * bn, bn) - 64 * h;
             } else if (id) {
-                m0 = ctl->colmasks[id * 4 + 2 * h];
-                m1 = ctl->colmasks[id * 4 + 2 * h + 1];
-                partial = true;
-            } else if (tail_partial && (w_mode == MODE_TILES || (u >> sh) == w_kv_count - 1)) {
-                m0 = h ? tail_mask[2] : tail_mask[0];
-                m1 = h ? tail_mask[3] : tail_mask[1];
-                partial = true;
+                const uint32_t shape = p.cls_shape[id];
+                if (shape) {
+                    const int32_t rows = p.shape_rows[shape];
+                    int32_t w0, w1;
+                    split_block((rows + 15) & ~15, 1 << sh, w0, w1);
+                    width = h ? w1 : w0;
+                    valid = rows - (h ? w0 : 0);
+                } else {
+                    mask_id = id;
+                }
+            } else if (tail_partial && (w_mode == MODE_TILES || j == w_kv_count - 1)) {
+                valid = tail_valid - 64 * h;
             }
-            if (partial) {
-#pragma unroll
-                for (int c = 0; c < 64; ++c)
-                    if (!(((c < 32 ? m0 : m1) >> (c & 31)) & 1u)) s[c] = 0xff800000u;  // -inf: not a key
+            if (!mask_id) valid = min(valid, width);  // columns past the width were never loaded
+            if (vis && vis != my_vis) {                // the other tile's block
+                valid = 0;
+                mask_id = 0;
             }
         };
+        // strike the columns that are not keys
+        auto apply_mask = [&](int32_t u, int32_t valid, uint32_t mask_id, uint32_t(&s)[64]) {
+            uint32_t m0, m1;
+            if (mask_id) {
+                m0 = ctl->colmasks[mask_id * 4 + 2 * (u & sh)];
+                m1 = ctl->colmasks[mask_id * 4 + 2 * (u & sh) + 1];
+            } else if (valid < 64) {
+                const int32_t v0 = min(max(valid, 0), 32), v1 = min(max(valid - 32, 0), 32);
+                m0 = v0 == 32 ? 0xffffffffu : ((1u << v0) - 1u);
+                m1 = v1 == 32 ? 0xffffffffu : ((1u << v1) - 1u);
+            } else {
+                return;
+            }
+#pragma unroll
+            for (int c = 0; c < 64; ++c)
+                if (!(((c < 32 ? m0 : m1) >> (c & 31)) & 1u)) s[c] = 0xff800000u;  // -inf: not a key
+        };
+        int32_t cur_width = 64;  // width of the sub-block whose scores s holds (generic path)
         // One sub-block: s holds the scores of u and row_max covers them.  Writes P(u), then
         // reads S(u+1) and moves row_max over it.  full: u and u+1 are both whole 64-key
         // sub-blocks of unmasked blocks, so nothing about widths or masks is looked at.
@@ -418,18 +509,25 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
             if (row == 0) TRACE(2 + m, u, 0);
             // P = exp2(S * scale - max) as packed bf16 over the first half of the buffer
             float2 sum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-            exp_block(s, scale, -row_max, sum);
+            if (kFull) exp_block(s, scale, -row_max, sum);
+            else exp_block<false>(s, scale, -row_max, sum, cur_width);
             if (row == 0) TRACE(2 + m, u, 1);
-            store_p(t_s + b * 64, kFull ? 64 : ((u & sh) ? width1 : width0), s);
+            store_p(t_s + b * 64, kFull ? 64 : cur_width, s);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bars + 8 * (BAR_P_READY + 2 * m + b));
             if (row == 0) TRACE(2 + m, u, 2);
             row_sum += (sum[0].x + sum[0].y) + (sum[1].x + sum[1].y);
             if (has_next) {
-                if (!load_sub(full, u + 1, s)) return false;
+                int32_t width = 64, valid = 64;
+                uint32_t mask_id = 0;
+                if (!kFull) sub_dims(with_text, u + 1, next_id, width, valid, mask_id);
+                if (!load_sub(full, u + 1, width, s)) return false;
                 if (row == 0) TRACE(2 + m, u, 3);
-                if (!kFull) apply_mask(with_text, u + 1, next_id, s);
+                if (!kFull) {
+                    apply_mask(u + 1, valid, mask_id, s);
+                    cur_width = width;
+                }
                 const float m_new = fmaxf(row_max, row_max64(s) * scale);
                 if (__any_sync(0xffffffffu, m_new - row_max > kRescaleThreshold)) {
                     // Lazy rescale: O and the row sum move to the new maximum only when it grew by
@@ -449,8 +547,14 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
         };
 
         uint32_t s[64];
-        if (!load_sub(std::false_type{}, 0, s)) return;
-        apply_mask(std::true_type{}, 0, (w_mode == MODE_TILES && n_boxes > 0) ? kv_entries[0].mask_id : 0u, s);
+        {
+            int32_t valid;
+            uint32_t mask_id;
+            sub_dims(std::true_type{}, 0, (w_mode == MODE_TILES && n_boxes > 0) ? kv_entries[0].mask_id : 0u, cur_width, valid,
+                     mask_id);
+            if (!load_sub(std::false_type{}, 0, cur_width, s)) return;
+            apply_mask(0, valid, mask_id, s);
+        }
         row_max = row_max64(s) * scale;
         // the leading unmasked blocks, then whatever is cut, short or last
         const int32_t n_full = min(2 * wp->kv_fast, n_sub) - 1;  // steps whose u and u+1 are both whole
@@ -473,8 +577,9 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
         tc_fence_after();
         // epilogue: O / row_sum -> bf16 -> global memory
         int32_t token = 0;
-        const int32_t q_org[3] = {wp->q_org[m][0], wp->q_org[m][1], wp->q_org[m][2]};
-        const bool valid = block_row_token(p.g, w_mode, q_org, w_kv_len, row, &token);
+        const int qi = packed ? (row >> 6) : m;
+        const int32_t q_org[3] = {wp->q_org[qi][0], wp->q_org[qi][1], wp->q_org[qi][2]};
+        const bool valid = block_row_token(p.g, w_mode, q_org, w_kv_len, packed ? (row & 63) : row, &token);
         const int64_t rows = w_mode == MODE_COMPACT ? p.g.Lct : p.g.Ltot;
         __nv_bfloat16 *out = (w_mode == MODE_COMPACT ? p.Oc + (int64_t)wp->slice * rows * D : p.O + (int64_t)wp->out_slice * rows * D) +
                              (int64_t)token * D;

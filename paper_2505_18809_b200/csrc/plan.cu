@@ -4,6 +4,7 @@
 #include <cmath>
 #include <cstring>
 #include <functional>
+#include <mutex>
 #include <new>
 #include <queue>
 
@@ -27,6 +28,18 @@ struct vorta_plan {
     KvEntry *d_kv_list = nullptr;
     int32_t *d_kv_count = nullptr;
     uint32_t *d_colmasks = nullptr;
+    // Packed query blocks (tiles of at most 64 tokens in one box): tiles 2k and 2k+1 of a row of tiles along
+    // W share one 128-row query block; their KV list is the union of the two windows.  Per pair
+    // ((tile_T * nt_H + tile_H) * (nt_W / 2) + k): first entry, entries, and key columns issued.
+    KvEntry *d_kv_pairs = nullptr;
+    std::vector<int32_t> pair_begin, pair_count;
+    std::vector<int64_t> pair_keys;
+    bool pack_tiles = false;
+    // KV boxes the grid cuts (sliding branch): column-mask class -> box shape, and per shape the extents
+    // (T, H, W) and the number of keys of the part of the box that lies inside the grid
+    uint8_t cls_shape[kMaxMasks + 7] = {};
+    int16_t shape_rows[kBoxShapes] = {};
+    int32_t shape_ext[kBoxShapes][3] = {};
     int32_t *d_seg_start = nullptr;
     int32_t *d_bucket_tab = nullptr;  // [8 shape classes][kBucketTabStride]
     // the ordered work of one attention launch: `routed` follows the current routes,
@@ -41,7 +54,26 @@ struct vorta_plan {
         double flops_issued = 0.0;
         bool built = false;
     };
-    WorkList routed, mixture;
+    WorkList routed, mixture;  // `routed` is a copy of the active cache entry's list (the entry owns the buffers)
+    // Work lists by route vector.  The router picks routes per timestep (Section 3.3) and a sampler
+    // revisits few distinct vectors, so the lists of the last few are kept, each with device buffers of
+    // its own: switching back to a known vector touches nothing on the device, and building a new one
+    // never writes to buffers a kernel in flight may be reading (an entry is reused only after the last
+    // call that used it has finished).
+    struct RouteEntry {
+        std::vector<uint8_t> routes;
+        WorkList wl;
+        std::vector<int32_t> core_heads;
+        int32_t *d_core_slice = nullptr, *d_core_xslice = nullptr;
+        cudaEvent_t used = nullptr;  // recorded after the last call that ran this entry's lists
+        bool used_valid = false;
+        uint64_t stamp = 0;          // activation order, for least-recently-used replacement
+    };
+    static constexpr int kRouteCache = 4;
+    mutable std::vector<RouteEntry> cache;
+    int cur = -1;
+    uint64_t activations = 0;
+    bool host_call_made = false;  // ev_out has been recorded: the groups' lists may be in use until it completes
     // The host-buffer entry point works through the heads in groups, so that the copies
     // of one group run under the kernels of another: each group has its own work list
     // and core-set problem tables, built with the routes.
@@ -70,6 +102,9 @@ struct vorta_plan {
     mutable int64_t prof_calls = 0;  // calls recorded so far
     bool profiling = false;
     mutable int32_t last_launches = 0;
+    // set when a route change failed half-way (an allocation or a copy): counts, routes and device
+    // lists may then disagree, so nothing is launched until a later vorta_plan_set_routes succeeds
+    bool broken = false;
 };
 
 namespace {
@@ -177,11 +212,15 @@ int64_t mixture_workspace_bytes(const Geometry &g)
 void free_device(vorta_plan *p)
 {
     cudaFree(p->d_bm); cudaFree(p->d_kv_list); cudaFree(p->d_kv_count); cudaFree(p->d_colmasks);
+    cudaFree(p->d_kv_pairs);
     cudaFree(p->d_seg_start); cudaFree(p->d_bucket_tab);
-    for (vorta_plan::WorkList *wl : {&p->routed, &p->mixture}) {
-        cudaFree(wl->d_items); cudaFree(wl->d_cta_begin); cudaFree(wl->d_cta_count);
+    cudaFree(p->mixture.d_items); cudaFree(p->mixture.d_cta_begin); cudaFree(p->mixture.d_cta_count);
+    for (auto &e : p->cache) {
+        cudaFree(e.wl.d_items); cudaFree(e.wl.d_cta_begin); cudaFree(e.wl.d_cta_count);
+        cudaFree(e.d_core_slice); cudaFree(e.d_core_xslice);
+        if (e.used) cudaEventDestroy(e.used);
     }
-    cudaFree(p->d_core_slice); cudaFree(p->d_core_xslice);
+    p->cache.clear();
     for (auto &c : p->chunks) {
         cudaFree(c.wl.d_items); cudaFree(c.wl.d_cta_begin); cudaFree(c.wl.d_cta_count);
         cudaFree(c.d_core_slice); cudaFree(c.d_core_xslice);
@@ -229,6 +268,121 @@ double sliding_valid_pairs(const Geometry &g)
     return total;
 }
 
+// Key columns the tensor-core kernel issues for the window of query tile qt: whole boxes count
+// bn_tile columns, a box the grid cuts counts the keys of its part inside the grid, rounded up to the
+// MMA granularity of 16 (classes without a short map keep the whole box).
+int64_t tile_issued_keys(const vorta_plan *p, int32_t qt)
+{
+    const Geometry &g = p->g;
+    const int32_t dim[3] = {g.T, g.H, g.W};
+    const int32_t q[3] = {qt / (g.nt[2] * g.nt[1]), (qt / g.nt[2]) % g.nt[1], qt % g.nt[2]};
+    int32_t lo[3], hi[3];
+    for (int a = 0; a < 3; ++a) {
+        lo[a] = 0;
+        hi[a] = g.nt[a] - 1;
+        if (g.restricted[a]) {
+            const int32_t c = std::min(std::max(q[a], g.half[a]), g.nt[a] - 1 - g.half[a]);
+            lo[a] = c - g.half[a];
+            hi[a] = c + g.half[a];
+        }
+    }
+    int64_t keys = 0;
+    for (int32_t kt = lo[0]; kt <= hi[0]; ++kt)
+        for (int32_t kh = lo[1]; kh <= hi[1]; ++kh)
+            for (int32_t kw = lo[2]; kw <= hi[2]; ++kw) {
+                const int32_t k[3] = {kt, kh, kw};
+                int32_t code = 0;
+                for (int a = 0; a < 3; ++a)
+                    if (dim[a] - k[a] * g.tile[a] < g.tile[a]) code |= 4 >> a;
+                for (int32_t bx = 0; bx < g.boxes_per_tile; ++bx) {
+                    const int32_t b[3] = {bx / (g.nbox[1] * g.nbox[2]), (bx / g.nbox[2]) % g.nbox[1], bx % g.nbox[2]};
+                    bool inside = true;
+                    for (int a = 0; a < 3; ++a) inside = inside && k[a] * g.tile[a] + b[a] * g.box[a] < dim[a];
+                    if (!inside) continue;
+                    const int32_t shape = code ? p->cls_shape[1 + code * g.boxes_per_tile + bx] : 0;
+                    if (!shape) { keys += g.bn_tile; continue; }
+                    const int32_t n = (p->shape_rows[shape] + 15) / 16 * 16;
+                    keys += (g.bn_tile > 64 && n < 32) ? 32 : n;  // two sub-blocks per block: at least 16 columns each
+                }
+            }
+    return keys;
+}
+
+// host -> device on the plan's copy stream (the caller waits for that stream before the data are used)
+cudaError_t upload(vorta_plan *p, void *dst, const void *src, size_t bytes)
+{
+    return cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, p->s_in);
+}
+
+// window of query tile index q on axis a: key tiles [lo, hi]
+inline void tile_window(const Geometry &g, int a, int32_t q, int32_t &lo, int32_t &hi)
+{
+    lo = 0;
+    hi = g.nt[a] - 1;
+    if (g.restricted[a]) {
+        const int32_t c = std::min(std::max(q, g.half[a]), g.nt[a] - 1 - g.half[a]);
+        lo = c - g.half[a];
+        hi = c + g.half[a];
+    }
+}
+
+// KV lists of the packed query blocks (see vorta_plan::d_kv_pairs): the blocks both tiles have in their
+// windows first (a row's first block must hold a key for it), then those only one of them has, marked.
+int build_pair_lists(vorta_plan *p)
+{
+    const Geometry &g = p->g;
+    p->pack_tiles = g.boxes_per_tile == 1 && g.box_rows <= 64 && g.nt[2] >= 2;
+    if (!p->pack_tiles) return VORTA_OK;
+    const int32_t dim[3] = {g.T, g.H, g.W};
+    const int32_t per_row = g.nt[2] / 2;
+    std::vector<KvEntry> all;
+    for (int32_t qt = 0; qt < g.nt[0]; ++qt)
+        for (int32_t qh = 0; qh < g.nt[1]; ++qh)
+            for (int32_t k = 0; k < per_row; ++k) {
+                int32_t lo[3], hi[3], loB, hiB;
+                tile_window(g, 0, qt, lo[0], hi[0]);
+                tile_window(g, 1, qh, lo[1], hi[1]);
+                tile_window(g, 2, 2 * k, lo[2], hi[2]);
+                tile_window(g, 2, 2 * k + 1, loB, hiB);
+                p->pair_begin.push_back((int32_t)all.size());
+                int64_t keys = 0;
+                for (int pass = 0; pass < 2; ++pass)
+                    for (int32_t kt = lo[0]; kt <= hi[0]; ++kt)
+                        for (int32_t kh = lo[1]; kh <= hi[1]; ++kh)
+                            for (int32_t kw = std::min(lo[2], loB); kw <= std::max(hi[2], hiB); ++kw) {
+                                const bool inA = kw >= lo[2] && kw <= hi[2], inB = kw >= loB && kw <= hiB;
+                                const uint32_t vis = inA && inB ? 0u : (inA ? 1u : 2u);
+                                if ((vis == 0) != (pass == 0)) continue;
+                                const int32_t kk[3] = {kt, kh, kw};
+                                int32_t code = 0;
+                                for (int a = 0; a < 3; ++a)
+                                    if (dim[a] - kk[a] * g.tile[a] < g.tile[a]) code |= 4 >> a;
+                                const bool whole = code == 0 && g.box_rows == g.bn_tile;
+                                const uint32_t id = whole ? 0u : (uint32_t)(1 + code);  // one box per tile
+                                KvEntry e;
+                                e.w0 = (int16_t)(kw * g.tile[2]);
+                                e.h0 = (int16_t)(kh * g.tile[1]);
+                                e.t0 = (int16_t)(kt * g.tile[0]);
+                                e.mask_id = (uint16_t)(id | (vis << kVisShift));
+                                all.push_back(e);
+                                const int32_t shape = p->cls_shape[id];
+                                keys += shape ? (p->shape_rows[shape] + 15) / 16 * 16 : g.bn_tile;
+                            }
+                // The first block of a list must hold a key for every row of the query block.  Two windows with
+                // no tile in common (a window of one tile along W) give no such block: the pair is not packed.
+                bool shared = false;
+                for (size_t i = (size_t)p->pair_begin.back(); i < all.size(); ++i) shared = shared || (all[i].mask_id >> kVisShift) == 0;
+                if (!shared) all.resize((size_t)p->pair_begin.back());
+                p->pair_count.push_back((int32_t)all.size() - p->pair_begin.back());
+                p->pair_keys.push_back(keys);
+            }
+    if (all.empty()) { p->pack_tiles = false; return VORTA_OK; }  // no pair can be packed
+    if (cudaMalloc(&p->d_kv_pairs, sizeof(KvEntry) * all.size()) != cudaSuccess ||
+        cudaMemcpy(p->d_kv_pairs, all.data(), sizeof(KvEntry) * all.size(), cudaMemcpyHostToDevice) != cudaSuccess)
+        return VORTA_ERR_CUDA;
+    return VORTA_OK;
+}
+
 // Build the ordered work list of one attention launch and upload it.  `branches[h]` is a
 // bit set of the branches head h runs (bit r = route r); a head with several branches
 // writes branch r to output slice r * B * heads + (b * heads + h).  Core-set problems are
@@ -243,6 +397,14 @@ int build_list(vorta_plan *p, vorta_plan::WorkList &wl, const std::vector<uint8_
     const int32_t BH = g.B * g.heads;
     std::vector<WorkItem> items;
     std::vector<double> cost;
+    std::vector<int64_t> item_keys;    // key columns issued per query block of the item
+    std::vector<int64_t> issued_keys;  // per query tile (sliding branch)
+    bool any_sliding = false;
+    for (int32_t h = 0; h < g.heads; ++h) any_sliding = any_sliding || (branches[h] & (1u << VORTA_ROUTE_SLIDING));
+    if (any_sliding) {
+        issued_keys.resize(g.n_tiles);
+        for (int32_t qt = 0; qt < g.n_tiles; ++qt) issued_keys[qt] = tile_issued_keys(p, qt);
+    }
     // query rows [q0, q1) of a sequence of `len` keys, two 128-row blocks per item
     auto linear_items = [&](int32_t mode, int32_t slice, int32_t out_slice, int32_t len, int32_t q0, int32_t q1) {
         int32_t nblk = (q1 - q0 + kBlockM - 1) / kBlockM;
@@ -254,6 +416,7 @@ int build_list(vorta_plan *p, vorta_plan::WorkList &wl, const std::vector<uint8_
             w.n_mblk = std::min(2, nblk - b0);
             for (int m = 0; m < w.n_mblk; ++m) w.q_org[m][0] = q0 + (b0 + m) * kBlockM;
             items.push_back(w);
+            item_keys.push_back((int64_t)kv * kBlockM);
             cost.push_back((double)w.n_mblk * kv + 2.0);
         }
     };
@@ -265,6 +428,29 @@ int build_list(vorta_plan *p, vorta_plan::WorkList &wl, const std::vector<uint8_
             if (branches[h] & (1u << VORTA_ROUTE_SLIDING)) {
                 for (int32_t qt = 0; qt < g.n_tiles; ++qt) {
                     int32_t q[3] = {qt / (g.nt[2] * g.nt[1]), (qt / g.nt[2]) % g.nt[1], qt % g.nt[2]};
+                    const int32_t pi = (q[0] * g.nt[1] + q[1]) * (g.nt[2] / 2) + q[2] / 2;
+                    if (p->pack_tiles && q[2] < (g.nt[2] & ~1) && p->pair_count[pi] > 0) {
+                        // tiles of at most 64 tokens: this tile and its right-hand neighbour in one query block
+                        if (q[2] & 1) continue;  // taken with the tile before it
+                        WorkItem w{};
+                        w.mode = MODE_TILES; w.slice = slice;
+                        w.out_slice = by_branch ? VORTA_ROUTE_SLIDING * BH + slice : slice;
+                        w.flags = kItemPacked;
+                        w.kv_text = g.text_blocks;
+                        w.kv_count = p->pair_count[pi] + w.kv_text;
+                        w.kv_fast = 0;
+                        w.kv_begin = p->pair_begin[pi];
+                        w.n_mblk = 1;
+                        for (int t = 0; t < 2; ++t) {
+                            w.q_org[t][0] = (q[2] + t) * g.tile[2];
+                            w.q_org[t][1] = q[1] * g.tile[1];
+                            w.q_org[t][2] = q[0] * g.tile[0];
+                        }
+                        items.push_back(w);
+                        item_keys.push_back(p->pair_keys[pi] + (int64_t)w.kv_text * g.bn_tile);
+                        cost.push_back((double)item_keys.back() / 128.0 + 2.0);
+                        continue;
+                    }
                     // the boxes of the tile that start inside the grid, two per item
                     int32_t org[kMaxBoxes][3], nb = 0;
                     for (int32_t bx = 0; bx < g.boxes_per_tile; ++bx) {
@@ -289,7 +475,8 @@ int build_list(vorta_plan *p, vorta_plan::WorkList &wl, const std::vector<uint8_
                         for (int m = 0; m < w.n_mblk; ++m)
                             for (int a = 0; a < 3; ++a) w.q_org[m][a] = org[b0 + m][a];
                         items.push_back(w);
-                        cost.push_back((double)w.n_mblk * w.kv_count * g.bn_tile / 128.0 + 2.0);
+                        item_keys.push_back(issued_keys[qt] + (int64_t)w.kv_text * g.bn_tile);
+                        cost.push_back((double)w.n_mblk * (double)item_keys.back() / 128.0 + 2.0);
                     }
                 }
                 // the text queries of a sliding head see every key: linear items over rows [L, L + Lt)
@@ -303,13 +490,9 @@ int build_list(vorta_plan *p, vorta_plan::WorkList &wl, const std::vector<uint8_
             }
         }
     }
-    // issued tensor-core work: every block is a 128 x bn QK^T and a 128 x d PV
+    // issued tensor-core work: per query block of 128 rows a QK^T and a PV over the item's key columns
     double issued = 0.0;
-    for (auto &w : items) {
-        double bn = w.mode == MODE_TILES ? g.bn_tile : 128;
-        issued += (double)w.n_mblk * w.kv_count * 4.0 * kBlockM * bn * g.d;
-    }
-    wl.flops_issued = issued;
+    for (size_t i = 0; i < items.size(); ++i) issued += (double)items[i].n_mblk * 4.0 * kBlockM * (double)item_keys[i] * g.d;
 
     // Longest-processing-time assignment of items to the persistent CTAs.  Three lists share the
     // device arrays: every item over the CTAs (the single-CTA kernel alone); and, for the hybrid
@@ -347,15 +530,15 @@ int build_list(vorta_plan *p, vorta_plan::WorkList &wl, const std::vector<uint8_
         return (int32_t)(sorted.size() - base);
     };
     assign(grid, 0, 0);
-    wl.n_linear = assign(n_pairs, grid, 1);
+    const int32_t n_linear = assign(n_pairs, grid, 1);
     assign(grid, grid + n_pairs, 2);
     double cost_all = 0.0, cost_linear = 0.0;
     for (size_t i = 0; i < items.size(); ++i) {
         cost_all += cost[i];
         if (items[i].mode != MODE_TILES) cost_linear += cost[i];
     }
-    wl.linear_share = cost_all > 0.0 ? cost_linear / cost_all : 0.0;
-    wl.n_items = (int32_t)items.size();
+    const double linear_share = cost_all > 0.0 ? cost_linear / cost_all : 0.0;
+    wl.built = false;  // until the new lists are on the device
 
     if (!wl.d_cta_begin &&
         (cudaMalloc(&wl.d_cta_begin, sizeof(int32_t) * n_bins) != cudaSuccess ||
@@ -368,13 +551,20 @@ int build_list(vorta_plan *p, vorta_plan::WorkList &wl, const std::vector<uint8_
         if (cudaMalloc(&wl.d_items, sizeof(WorkItem) * std::max<size_t>(sorted.size(), 1)) != cudaSuccess)
             return VORTA_ERR_CUDA;
     }
-    // synchronous copies: the caller may change routes between steps
-    if (!sorted.empty() &&
-        cudaMemcpy(wl.d_items, sorted.data(), sizeof(WorkItem) * sorted.size(), cudaMemcpyHostToDevice) != cudaSuccess)
+    // Copies on the plan's own (non-blocking) copy stream, and a wait for just these copies: a plain
+    // cudaMemcpy would queue behind everything in the legacy default stream, i.e. behind the attention
+    // kernels of the step still running.  The destinations are not in use (see RouteEntry).
+    if (!sorted.empty() && upload(p, wl.d_items, sorted.data(), sizeof(WorkItem) * sorted.size()) != cudaSuccess)
         return VORTA_ERR_CUDA;
-    if (cudaMemcpy(wl.d_cta_begin, begin.data(), sizeof(int32_t) * n_bins, cudaMemcpyHostToDevice) != cudaSuccess ||
-        cudaMemcpy(wl.d_cta_count, count.data(), sizeof(int32_t) * n_bins, cudaMemcpyHostToDevice) != cudaSuccess)
+    if (upload(p, wl.d_cta_begin, begin.data(), sizeof(int32_t) * n_bins) != cudaSuccess ||
+        upload(p, wl.d_cta_count, count.data(), sizeof(int32_t) * n_bins) != cudaSuccess ||
+        cudaStreamSynchronize(p->s_in) != cudaSuccess)
         return VORTA_ERR_CUDA;
+    // the counts follow the device lists: set only now that every allocation and copy has succeeded
+    wl.n_items = (int32_t)items.size();
+    wl.n_linear = n_linear;
+    wl.linear_share = linear_share;
+    wl.flops_issued = issued;
     wl.built = true;
     return VORTA_OK;
 }
@@ -405,6 +595,8 @@ std::vector<int32_t> host_chunk_sizes(int32_t heads)
 int build_host_chunks(vorta_plan *p)
 {
     const Geometry &g = p->g;
+    // the groups' lists and tables are rewritten in place: the last host-buffer call must be through with them
+    if (p->host_call_made && cudaEventSynchronize(p->ev_out) != cudaSuccess) return VORTA_ERR_CUDA;
     std::vector<double> cost(g.heads);
     for (int32_t h = 0; h < g.heads; ++h) {
         const uint8_t r = p->routes[h];
@@ -448,38 +640,115 @@ int build_host_chunks(vorta_plan *p)
                 cx[(size_t)b * c.n_core + k] = b;
             }
         if (c.n_core &&
-            (cudaMemcpy(c.d_core_slice, cs.data(), sizeof(int32_t) * g.B * c.n_core, cudaMemcpyHostToDevice) != cudaSuccess ||
-             cudaMemcpy(c.d_core_xslice, cx.data(), sizeof(int32_t) * g.B * c.n_core, cudaMemcpyHostToDevice) != cudaSuccess))
+            (upload(p, c.d_core_slice, cs.data(), sizeof(int32_t) * g.B * c.n_core) != cudaSuccess ||
+             upload(p, c.d_core_xslice, cx.data(), sizeof(int32_t) * g.B * c.n_core) != cudaSuccess ||
+             cudaStreamSynchronize(p->s_in) != cudaSuccess))
             return VORTA_ERR_CUDA;
     }
     return VORTA_OK;
 }
 
-// (Re)build the work list for the current routes.
+// Make the work list of the current routes the active one: a list kept from an earlier use of the same
+// route vector, or a new one built into the least recently used entry.
 int build_work(vorta_plan *p)
 {
     const Geometry &g = p->g;
-    p->core_heads.clear();
+    std::vector<int32_t> core_heads;
     for (int32_t h = 0; h < g.heads; ++h)
-        if (p->routes[h] == VORTA_ROUTE_CORESET) p->core_heads.push_back(h);
-    if (p->host_only) return VORTA_OK;
-    std::vector<uint8_t> branches(g.heads);
-    for (int32_t h = 0; h < g.heads; ++h) branches[h] = (uint8_t)(1u << p->routes[h]);
-    int rc = build_list(p, p->routed, branches, false);
-    if (rc != VORTA_OK) return rc;
-    const int32_t n_core = (int32_t)p->core_heads.size();
-    std::vector<int32_t> core_slice((size_t)g.B * std::max(n_core, 1)), core_x(core_slice.size());
-    for (int32_t b = 0; b < g.B; ++b)
-        for (int32_t k = 0; k < n_core; ++k) {
-            core_slice[(size_t)b * n_core + k] = b * g.heads + p->core_heads[k];
-            core_x[(size_t)b * n_core + k] = b;
+        if (p->routes[h] == VORTA_ROUTE_CORESET) core_heads.push_back(h);
+    if (p->host_only) {
+        p->core_heads = core_heads;
+        return VORTA_OK;
+    }
+    int hit = -1;
+    for (size_t i = 0; i < p->cache.size(); ++i)
+        if (p->cache[i].routes == p->routes) hit = (int)i;
+    if (hit < 0) {
+        if ((int)p->cache.size() < vorta_plan::kRouteCache) {
+            p->cache.emplace_back();
+            hit = (int)p->cache.size() - 1;
+            vorta_plan::RouteEntry &e = p->cache[hit];
+            if (cudaEventCreateWithFlags(&e.used, cudaEventDisableTiming) != cudaSuccess ||
+                cudaMalloc(&e.d_core_slice, sizeof(int32_t) * (size_t)g.B * g.heads) != cudaSuccess ||
+                cudaMalloc(&e.d_core_xslice, sizeof(int32_t) * (size_t)g.B * g.heads) != cudaSuccess)
+                return VORTA_ERR_CUDA;
+        } else {
+            hit = 0;
+            for (size_t i = 1; i < p->cache.size(); ++i)
+                if (p->cache[i].stamp < p->cache[hit].stamp) hit = (int)i;
+            // its buffers are about to be overwritten: the last call that used them must be done
+            if (p->cache[hit].used_valid && cudaEventSynchronize(p->cache[hit].used) != cudaSuccess) return VORTA_ERR_CUDA;
         }
-    if (n_core &&
-        (cudaMemcpy(p->d_core_slice, core_slice.data(), sizeof(int32_t) * g.B * n_core, cudaMemcpyHostToDevice) != cudaSuccess ||
-         cudaMemcpy(p->d_core_xslice, core_x.data(), sizeof(int32_t) * g.B * n_core, cudaMemcpyHostToDevice) != cudaSuccess))
-        return VORTA_ERR_CUDA;
+        vorta_plan::RouteEntry &e = p->cache[hit];
+        e.routes.clear();  // not a valid entry until everything below has succeeded
+        e.used_valid = false;
+        std::vector<uint8_t> branches(g.heads);
+        for (int32_t h = 0; h < g.heads; ++h) branches[h] = (uint8_t)(1u << p->routes[h]);
+        int rc = build_list(p, e.wl, branches, false);
+        if (rc != VORTA_OK) return rc;
+        const int32_t n_core = (int32_t)core_heads.size();
+        std::vector<int32_t> core_slice((size_t)g.B * std::max(n_core, 1)), core_x(core_slice.size());
+        for (int32_t b = 0; b < g.B; ++b)
+            for (int32_t k = 0; k < n_core; ++k) {
+                core_slice[(size_t)b * n_core + k] = b * g.heads + core_heads[k];
+                core_x[(size_t)b * n_core + k] = b;
+            }
+        if (n_core &&
+            (upload(p, e.d_core_slice, core_slice.data(), sizeof(int32_t) * g.B * n_core) != cudaSuccess ||
+             upload(p, e.d_core_xslice, core_x.data(), sizeof(int32_t) * g.B * n_core) != cudaSuccess ||
+             cudaStreamSynchronize(p->s_in) != cudaSuccess))
+            return VORTA_ERR_CUDA;
+        e.core_heads = core_heads;
+        e.routes = p->routes;
+    }
+    vorta_plan::RouteEntry &e = p->cache[hit];
+    e.stamp = ++p->activations;
+    p->cur = hit;
+    p->routed = e.wl;
+    p->core_heads = e.core_heads;
+    p->d_core_slice = e.d_core_slice;
+    p->d_core_xslice = e.d_core_xslice;
     p->chunks_stale = true;
     return VORTA_OK;
+}
+
+// Order between the two kinds of persistent attention kernel on one device.  A cluster kernel (CTA
+// pairs) and the single-CTA kernel must not share the GPU: side by side, the single-CTA kernel's
+// bounded waits have expired.  Calls from different plans or streams could still mix them, so every
+// launch of one kind first makes its stream wait for the last launch of the other kind on that
+// device, and records itself afterwards.  Kernels of the same kind may overlap freely.
+struct KernelOrder {
+    std::mutex m;
+    cudaEvent_t last[2] = {nullptr, nullptr};  // 0: pair kernel, 1: single-CTA kernel
+    bool recorded[2] = {false, false};
+};
+KernelOrder *kernel_order(int device)
+{
+    static KernelOrder table[64];
+    return device >= 0 && device < 64 ? &table[device] : nullptr;
+}
+// before a launch of `kind` on stream s
+cudaError_t order_before(int device, int kind, cudaStream_t s)
+{
+    KernelOrder *o = kernel_order(device);
+    if (!o) return cudaSuccess;
+    std::lock_guard<std::mutex> lock(o->m);
+    const int other = kind ^ 1;
+    return o->recorded[other] ? cudaStreamWaitEvent(s, o->last[other], 0) : cudaSuccess;
+}
+// after it
+cudaError_t order_after(int device, int kind, cudaStream_t s)
+{
+    KernelOrder *o = kernel_order(device);
+    if (!o) return cudaSuccess;
+    std::lock_guard<std::mutex> lock(o->m);
+    if (!o->last[kind]) {
+        cudaError_t e = cudaEventCreateWithFlags(&o->last[kind], cudaEventDisableTiming);
+        if (e != cudaSuccess) return e;
+    }
+    cudaError_t e = cudaEventRecord(o->last[kind], s);
+    if (e == cudaSuccess) o->recorded[kind] = true;
+    return e;
 }
 
 struct DeviceGuard {
@@ -646,6 +915,19 @@ int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
                 valid[a] = std::min(std::max(extent - b[a] * g.box[a], 0), g.box[a]);
             }
             const int32_t id = 1 + code * g.boxes_per_tile + bx;
+            // the shape of the part inside the grid: which axes cut THIS box (a box of a cut tile may
+            // still be whole, or lie outside altogether: such boxes are never listed)
+            int32_t shape = 0;
+            for (int a = 0; a < 3; ++a)
+                if (valid[a] > 0 && valid[a] < g.box[a]) shape |= 4 >> a;
+#ifdef VORTA_NO_SHORT_BOXES
+            shape = 0;
+#endif
+            if (valid[0] > 0 && valid[1] > 0 && valid[2] > 0 && shape) {
+                p->cls_shape[id] = (uint8_t)shape;
+                p->shape_rows[shape] = (int16_t)(valid[0] * valid[1] * valid[2]);
+                for (int a = 0; a < 3; ++a) p->shape_ext[shape][a] = valid[a];
+            }
             for (int32_t r = 0; r < g.box_rows; ++r) {
                 int32_t lw = r % g.box[2], lh = (r / g.box[2]) % g.box[1], lt = r / (g.box[2] * g.box[1]);
                 if (lw < valid[2] && lh < valid[1] && lt < valid[0]) masks[(size_t)id * 4 + r / 32] |= 1u << (r % 32);
@@ -683,8 +965,6 @@ int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
     ok = ok && cudaMalloc(&p->d_seg_start, sizeof(int32_t) * g.n_buckets) == cudaSuccess;
     ok = ok && cudaMalloc(&p->d_bucket_tab, sizeof(int32_t) * btab.size()) == cudaSuccess;
     ok = ok && cudaMemcpy(p->d_bucket_tab, btab.data(), sizeof(int32_t) * btab.size(), cudaMemcpyHostToDevice) == cudaSuccess;
-    ok = ok && cudaMalloc(&p->d_core_slice, sizeof(int32_t) * (size_t)g.B * g.heads) == cudaSuccess;
-    ok = ok && cudaMalloc(&p->d_core_xslice, sizeof(int32_t) * (size_t)g.B * g.heads) == cudaSuccess;
     ok = ok && cudaMalloc(&p->d_status, sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMemset(p->d_status, 0, sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMemcpy(p->d_colmasks, masks.data(), sizeof(uint32_t) * masks.size(), cudaMemcpyHostToDevice) == cudaSuccess;
@@ -706,7 +986,8 @@ int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
     // self-check: the lists must hold exactly the blocks the window arithmetic predicts
     for (int32_t qt = 0; qt < g.n_tiles; ++qt)
         if (p->kv_count[qt] < 1 || p->kv_count[qt] > g.max_kv_per_tile) { free_device(p); delete p; return VORTA_ERR_INTERNAL; }
-    int rc = build_work(p);
+    int rc = build_pair_lists(p);
+    if (rc == VORTA_OK) rc = build_work(p);
     if (rc != VORTA_OK) { free_device(p); delete p; return rc; }
     *out = p;
     return VORTA_OK;
@@ -720,8 +1001,11 @@ int vorta_plan_set_routes(vorta_plan *p, const uint8_t *routes, int32_t n)
     p->routes.assign(routes, routes + n);
     if (p->host_only) return build_work(p);
     DeviceGuard guard(p->device);
-    if (!guard.ok || cudaDeviceSynchronize() != cudaSuccess) return VORTA_ERR_CUDA;
-    return build_work(p);
+    p->broken = true;
+    if (!guard.ok) return VORTA_ERR_CUDA;
+    int rc = build_work(p);  // no device-wide wait: see RouteEntry
+    p->broken = rc != VORTA_OK;
+    return rc;
 }
 
 int vorta_plan_destroy(vorta_plan *p)
@@ -920,7 +1204,9 @@ static int run_layer(const vorta_plan *p, const vorta_plan::WorkList &wl, int32_
     prm.g = g;
     prm.scale_log2 = p->scale * 1.4426950408889634f;
     prm.items = wl.d_items; prm.cta_begin = wl.d_cta_begin; prm.cta_count = wl.d_cta_count;
-    prm.kv_list = p->d_kv_list; prm.colmasks = p->d_colmasks;
+    prm.kv_list = p->d_kv_list; prm.kv_pairs = p->d_kv_pairs; prm.colmasks = p->d_colmasks;
+    std::memcpy(prm.cls_shape, p->cls_shape, sizeof(prm.cls_shape));
+    std::memcpy(prm.shape_rows, p->shape_rows, sizeof(prm.shape_rows));
     prm.O = o_attn; prm.Oc = Oc; prm.Q = q; prm.K = k; prm.V = v; prm.Qc = Qc; prm.Kc = Kc; prm.Vc = Vc;
     prm.status = p->d_status;
 #ifdef VORTA_TRACE
@@ -959,6 +1245,17 @@ static int run_layer(const vorta_plan *p, const vorta_plan::WorkList &wl, int32_
             // the video rows of a head as a T x H x W grid; heads are L + Lt rows apart
             ok = ok && make_map(&dst[t][MODE_TILES], src[t], g.d, g.W, g.H, g.T, BH, g.box[2], g.box[1], g.box[0],
                                 g.Ltot);
+        }
+        // the short boxes of the KV tiles the grid cuts (shapes that do not occur alias the whole box)
+        for (int sh = 0; sh < kBoxShapes && ok; ++sh) {
+            if (p->shape_rows[sh] > 0) {
+                const int32_t *e = p->shape_ext[sh];
+                ok = ok && make_map(&maps.k_cut[sh], k, g.d, g.W, g.H, g.T, BH, e[2], e[1], e[0], g.Ltot);
+                ok = ok && make_map(&maps.v_cut[sh], v, g.d, g.W, g.H, g.T, BH, e[2], e[1], e[0], g.Ltot);
+            } else {
+                maps.k_cut[sh] = maps.k[MODE_TILES];
+                maps.v_cut[sh] = maps.v[MODE_TILES];
+            }
         }
         if (g.Lt > 0) {
             // the text rows of K and V: Lt rows starting L rows into every head, in boxes of bn_tile rows
@@ -1022,19 +1319,25 @@ static int run_layer(const vorta_plan *p, const vorta_plan::WorkList &wl, int32_
             // bounded waits expired at hunyuan-720p: CTAs of a cluster kernel and of a plain kernel
             // are not mixed on the GPU here.)
             if (wl.n_linear > 0) {
+                if (order_before(p->device, 0, s) != cudaSuccess) return VORTA_ERR_CUDA;
                 e = launch_attention_sm100_pair(prm_pair, maps, p->sm_count, s);
-                if (e != cudaSuccess) return VORTA_ERR_CUDA;
+                if (e != cudaSuccess || order_after(p->device, 0, s) != cudaSuccess) return VORTA_ERR_CUDA;
                 ++launches;
             }
             if (wl.n_linear > 0 && wl.n_items - wl.n_linear > 0) mark(5);
             if (wl.n_items - wl.n_linear > 0) {
+                if (order_before(p->device, 1, s) != cudaSuccess) return VORTA_ERR_CUDA;
                 e = launch_attention_sm100(prm_tiles, maps, p->sm_count, s);
-                if (e != cudaSuccess) return VORTA_ERR_CUDA;
+                if (e != cudaSuccess || order_after(p->device, 1, s) != cudaSuccess) return VORTA_ERR_CUDA;
                 ++launches;
             }
+        } else if (kernel == VORTA_KERNEL_TCGEN05) {
+            if (order_before(p->device, 1, s) != cudaSuccess) return VORTA_ERR_CUDA;
+            e = launch_attention_sm100(prm, maps, p->sm_count, s);
+            if (e != cudaSuccess || order_after(p->device, 1, s) != cudaSuccess) return VORTA_ERR_CUDA;
+            ++launches;
         } else {
-            e = kernel == VORTA_KERNEL_TCGEN05 ? launch_attention_sm100(prm, maps, p->sm_count, s)
-                                                  : launch_attention_simt(prm, wl.n_items, s);
+            e = launch_attention_simt(prm, wl.n_items, s);
             if (e != cudaSuccess) return VORTA_ERR_CUDA;
             ++launches;
         }
@@ -1055,6 +1358,7 @@ int vorta_routed_attention(const vorta_plan *p, const void *Q, const void *K, co
 {
     if (!p || !Q || !K || !V || !O) return VORTA_ERR_INVALID_ARG;
     if (p->host_only) return VORTA_ERR_UNSUPPORTED;
+    if (p->broken) return VORTA_ERR_INTERNAL;
     const Geometry &g = p->g;
     if (X && Hx != 1 && Hx != g.heads) return VORTA_ERR_INVALID_ARG;
     if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) || (X && !aligned(X, 16)))
@@ -1068,9 +1372,16 @@ int vorta_routed_attention(const vorta_plan *p, const void *Q, const void *K, co
     DeviceGuard guard(p->device);
     if (!guard.ok) return VORTA_ERR_CUDA;
     __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(O);
-    return run_layer(p, p->routed, n_core, p->d_core_slice, p->d_core_xslice, static_cast<const __nv_bfloat16 *>(Q),
-                     static_cast<const __nv_bfloat16 *>(K), static_cast<const __nv_bfloat16 *>(V), o, o, X, Hx,
-                     workspace, static_cast<cudaStream_t>(stream), true);
+    int rc = run_layer(p, p->routed, n_core, p->d_core_slice, p->d_core_xslice, static_cast<const __nv_bfloat16 *>(Q),
+                       static_cast<const __nv_bfloat16 *>(K), static_cast<const __nv_bfloat16 *>(V), o, o, X, Hx,
+                       workspace, static_cast<cudaStream_t>(stream), true);
+    // this route vector's lists are in use until here on the stream
+    if (p->cur >= 0) {
+        vorta_plan::RouteEntry &e = p->cache[p->cur];
+        if (cudaEventRecord(e.used, static_cast<cudaStream_t>(stream)) == cudaSuccess) e.used_valid = true;
+        else if (rc == VORTA_OK) rc = VORTA_ERR_CUDA;
+    }
+    return rc;
 }
 
 int vorta_soft_mixture(vorta_plan *p, const void *Q, const void *K, const void *V, const float *gates, void *O,
@@ -1120,6 +1431,7 @@ int vorta_routed_attention_host(const vorta_plan *p, const void *Qh, const void 
 {
     if (!p || !Qh || !Kh || !Vh || !Oh || !scratch) return VORTA_ERR_INVALID_ARG;
     if (p->host_only) return VORTA_ERR_UNSUPPORTED;
+    if (p->broken) return VORTA_ERR_INTERNAL;
     vorta_plan_info_t info;
     vorta_plan_info(p, &info);
     if ((int64_t)scratch_bytes < info.host_call_scratch_bytes) return VORTA_ERR_WORKSPACE;
@@ -1132,7 +1444,10 @@ int vorta_routed_attention_host(const vorta_plan *p, const void *Qh, const void 
         // first call since the routes were set: build the groups' work lists (small device
         // allocations and synchronous copies; later calls only enqueue)
         int rc = build_host_chunks(const_cast<vorta_plan *>(p));
-        if (rc != VORTA_OK) return rc;
+        if (rc != VORTA_OK) {
+            const_cast<vorta_plan *>(p)->broken = true;  // the groups' lists are half built
+            return rc;
+        }
         p->chunks_stale = false;
     }
     const int64_t tb = tensor_bytes(g), tba = align_up(tb, 256);
@@ -1203,6 +1518,7 @@ int vorta_routed_attention_host(const vorta_plan *p, const void *Qh, const void 
     }
     if (cudaEventRecord(p->ev_out, p->s_out) != cudaSuccess || cudaStreamWaitEvent(s, p->ev_out, 0) != cudaSuccess)
         return VORTA_ERR_CUDA;
+    const_cast<vorta_plan *>(p)->host_call_made = true;
     return VORTA_OK;
 }
 

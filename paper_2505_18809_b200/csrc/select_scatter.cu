@@ -318,8 +318,12 @@ coreset_select_d128_kernel(Geometry g, const __nv_bfloat16 *__restrict__ X, cons
                 dot += __shfl_xor_sync(0xffffffffu, dot, m);
                 njsq += __shfl_xor_sync(0xffffffffu, njsq, m);
             }
-            if (pass * 4 + sub < n && !(njsq > 1e-30f && njsq < 1e30f)) doubtful = true;
-            const float score = dot * rsqrtf(csq * njsq);
+            // the product of the two squared norms must itself be an ordinary fp32 number: two small
+            // norms (or two large ones) each pass the range test and still underflow (overflow) together,
+            // and the infinite or zero score that follows would slip through the guard band
+            const float nsq = csq * njsq;
+            if (pass * 4 + sub < n && !(njsq > 1e-30f && njsq < 1e30f && nsq > 1e-30f && nsq < 1e30f)) doubtful = true;
+            const float score = dot * rsqrtf(nsq);
             const float got = __shfl_sync(0xffffffffu, score, (lane & 3) * 8);
             if ((lane >> 2) == pass) my32 = got;
         }

@@ -23,6 +23,7 @@ constexpr int kBlockM = 128;       // query rows per M-block (one MMA M)
 constexpr int kMaxBoxes = 8;       // a sliding tile is cut into at most this many TMA boxes of <= 128 tokens
 constexpr int kMaxMasks = 1 + 8 * kMaxBoxes;  // column-mask classes of the sliding branch (0 = none):
                                               // which axes the grid cuts the tile on x which box of the tile
+constexpr int kBoxShapes = 8;      // KV box shapes of the sliding branch: bit 2 / 1 / 0 = cut by the grid on T / H / W
 constexpr int kAttnThreads = 320;  // tcgen05 kernel: 2 control warps + 2 x 4 softmax warps
 constexpr int kBucketTabStride = 34;  // per bucket shape class: token count, centre, 32 token offsets
 
@@ -43,11 +44,16 @@ struct Geometry {
     int32_t box[3], nbox[3], box_rows, bn_tile, boxes_per_tile, max_kv_per_tile;
 };
 
-// One KV block of a sliding-tile query: origin of its box and its column-mask class.
+// One KV block of a sliding-tile query: origin of its box and its column-mask class.  In the lists of
+// packed items (two query tiles in one 128-row block, see WorkItem::flags) the two top bits of mask_id
+// say which of the two tiles has the block in its window: 0 both, 1 only the first, 2 only the second.
 struct KvEntry {
     int16_t w0, h0, t0;
     uint16_t mask_id;
 };
+constexpr uint32_t kMaskIdBits = 0x3fffu;
+constexpr int kVisShift = 14;
+constexpr int32_t kItemPacked = 1;  // WorkItem::flags
 
 // One unit of work of the attention kernel: up to two 128-row query blocks that
 // walk the same sequence of KV blocks.
@@ -62,7 +68,10 @@ struct WorkItem {
     int32_t out_slice;    // slice of the output tensor the rows are written to (non-compact modes)
     int32_t kv_fast;      // the first kv_fast blocks are 128 real keys each: no column needs masking
     int32_t kv_text;      // MODE_TILES: blocks [kv_count - kv_text, kv_count) are bn_tile-key blocks of text tokens
-    int32_t pad[1];
+    // kItemPacked (MODE_TILES, tiles of at most 64 tokens, n_mblk = 1): the one query block holds TWO tiles
+    // that are neighbours along W, q_org[0] in rows [0, 64) and q_org[1] in rows [64, 128); the KV blocks are
+    // the union of the two windows, listed in AttnParams::kv_pairs from kv_begin on.
+    int32_t flags;
 };
 static_assert(sizeof(WorkItem) == 64, "WorkItem must stay 64 bytes");
 
@@ -71,6 +80,10 @@ struct AttnMaps {
     CUtensorMap q[3], k[3], v[3];  // indexed by mode
     CUtensorMap kt, vt;            // text rows [L, L + Lt) of K and V in boxes of bn_tile rows (sliding items)
     CUtensorMap k_half[3];         // pair kernel: K of the linear modes in boxes of 64 rows
+    // Sliding branch, KV boxes the grid cuts: one map per shape whose box is just the part inside the
+    // grid (index = which axes are cut; 0 is unused, the whole box goes through k/v[MODE_TILES]), so a
+    // cut box arrives as a short run of real keys instead of a 128-row box with holes.
+    CUtensorMap k_cut[kBoxShapes], v_cut[kBoxShapes];
 };
 
 struct AttnParams {
@@ -80,7 +93,10 @@ struct AttnParams {
     const int32_t *cta_begin;      // [grid] first item of each CTA
     const int32_t *cta_count;      // [grid]
     const KvEntry *kv_list;
+    const KvEntry *kv_pairs;       // KV lists of the packed items
     const uint32_t *colmasks;      // [kMaxMasks][4]
+    uint8_t cls_shape[kMaxMasks + 7];  // column-mask class -> box shape (0: whole box, or no short map for it)
+    int16_t shape_rows[kBoxShapes];    // keys in a box of each shape (all of them real)
     __nv_bfloat16 *O;              // [B*heads, L + Lt, d]
     __nv_bfloat16 *Oc;             // [n_compact, Lc + Lt, d]
     const __nv_bfloat16 *Q, *K, *V;     // originals (SIMT kernel)

@@ -266,6 +266,51 @@ def test_routes_can_change_between_steps_and_shared_selection_features():
     p.close()
 
 
+def test_routes_alternate_between_steps_without_waiting_for_the_device():
+    """The router decides per timestep (Section 3.3, Eq. 4): two route vectors taken in turn over six
+    steps, each step enqueued while the one before may still be running (no synchronisation between
+    set_routes and the calls), then a third, fourth, fifth and sixth vector so that kept lists are
+    replaced.  Every step's output must be the oracle's for the routes it ran with, and switching back
+    to a known vector must not cost a rebuild."""
+    import time
+    wl = Workload("alt", (6, 16, 16), 4, 128, (2, 8, 8), (3, 3, 3), 0.5, (0, 1, 2, 1), 66, False)
+    Q, K, V = workloads.make_qkv(wl, DEV)
+    p = vb.Plan.from_workload(wl)
+    ws = p.workspace(DEV) if p.info.workspace_bytes_max else None
+    ws = torch.empty(int(p.info.workspace_bytes_max) + 256, dtype=torch.uint8, device=DEV)
+    vectors = [(0, 1, 2, 1), (2, 2, 1, 0)]
+    outs = []
+    for step in range(6):
+        routes = vectors[step % 2]
+        p.set_routes(routes)
+        O = torch.full_like(Q, float("nan"))
+        p.routed_attention(Q, K, V, O, workspace=ws)
+        outs.append((routes, O))
+    for routes in [(1, 1, 1, 1), (0, 0, 2, 2), (2, 1, 0, 0), (1, 2, 2, 2), vectors[0]]:
+        p.set_routes(routes)
+        O = torch.full_like(Q, float("nan"))
+        p.routed_attention(Q, K, V, O, workspace=ws)
+        outs.append((routes, O))
+    assert p.device_status() == 0
+    want = {}
+    for routes, O in outs:
+        for h in range(wl.heads):
+            key = (h, routes[h])
+            if key not in want:
+                want[key] = oracle_head_rows(wl, Q, K, V, 0, h, None, route=routes[h])
+            assert_close(O[0, h], want[key], f"routes {routes} h{h}")
+    # a vector whose lists are kept: no rebuild, no copy, no wait
+    p.set_routes(vectors[1])
+    p.set_routes(vectors[0])
+    t0 = time.perf_counter()
+    for _ in range(20):
+        p.set_routes(vectors[1])
+        p.set_routes(vectors[0])
+    per_call = (time.perf_counter() - t0) / 40
+    assert per_call < 0.5e-3, per_call      # measured: a few microseconds
+    p.close()
+
+
 def test_default_kernel_choice_follows_the_routes():
     """VORTA_KERNEL_AUTO: the pair kernel where full and core-set heads hold at least 60 % of the
     work, the single-CTA kernel otherwise; the choice is remade when the routes change."""

@@ -14,6 +14,8 @@ device may make the driver set the array aside, so it is not held to that.
 It is collected last on purpose: a run that stops at the first failure has then already run
 every other test.  It also passes on its own in a fresh process.
 """
+import gc
+
 import pytest
 import torch
 
@@ -47,6 +49,7 @@ def test_static_workspace_entry_point_matches_the_workspace_one_twice():
         want = plan.routed_attention(Q, K, V)
         assert plan.device_status() == 0
         got = torch.full_like(Q, float("nan"))
+        gc.collect()                     # tensors of the previous round must not be released under the call
         torch.cuda.synchronize()
         before, free_before = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
         vb.vorta_routed_attention_static(plan.handle, Q.data_ptr(), K.data_ptr(), V.data_ptr(),
