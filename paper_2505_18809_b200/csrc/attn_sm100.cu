@@ -431,10 +431,11 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
             if (!mbar_wait(bars + 8 * (BAR_S_FULL + 2 * m + b), (s_par >> b) & 1, ctl, p.status, 301 + m)) return false;
             s_par ^= 1u << b;
             tc_fence_after();
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                uint32_t(&chunk)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[32 * c]);
-                if (decltype(full)::value || c * 32 < width) ptx::tcgen05_ld_32x32b(chunk, t_s + b * 64 + c * 32);
+            if (decltype(full)::value || width > 32) {
+                ptx::tcgen05_ld_32x32b(s, t_s + b * 64);  // one 64-column load
+            } else {
+                uint32_t(&chunk)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[0]);
+                ptx::tcgen05_ld_32x32b(chunk, t_s + b * 64);
             }
             tc_wait_ld();
             return true;

@@ -409,11 +409,7 @@ __device__ __forceinline__ bool softmax_block(const AttnParams &p, Ctl *ctl, con
     // this thread's row of S, 64 columns at a time: half h is keys [64 h, 64 h + 64)
     uint32_t s[64];
     auto load_half = [&](int h) {
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-            uint32_t(&chunk)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[32 * c]);
-            ptx::tcgen05_ld_32x32b(chunk, t_s + h * 64 + c * 32);
-        }
+        ptx::tcgen05_ld_32x32b(s, t_s + h * 64);  // one 64-column load (two 32-column ones: 1.2 % slower)
         tc_wait_ld();
         if (!kFull && (m[2 * h] & m[2 * h + 1]) != 0xffffffffu) {
 #pragma unroll
