@@ -1,6 +1,8 @@
 // Memory-bound kernels of the routed-attention layer: the block-sparse sliding-tile
 // mask builder, bucketed core-set selection, the gather (pool) of the kept rows
 // and the scatter (unpool) of the attention output.
+#include <algorithm>
+
 #include "vorta_internal.h"
 
 namespace vorta {
@@ -211,18 +213,6 @@ coreset_select_kernel(Geometry g, const __nv_bfloat16 *__restrict__ X, int32_t d
     src_slot[(int64_t)p * g.L + tok] = slot;
 }
 
-// The same selection for the common case dx = 128 and buckets of at most 12 tokens
-// (the paper's (2, 3, 2)).  Every lane first issues the loads of all its chunks -- its
-// share of the centre row and of the three token rows it helps to score -- so that a
-// warp has the whole bucket in flight before any arithmetic.
-//
-// Scores are first taken in fp32 (products of bf16 values are exact there; the sums of
-// 128 terms are not): each cosine is then within 2.5e-5 of its true value.  Only the SET
-// of pruned tokens matters, i.e. the order of the k-th and (k+1)-th largest scores, so
-// the fp32 ranking is accepted when those two are at least 2^-13 apart.  Otherwise --
-// near-ties, exact ties, rows with a vanishing or non-finite squared norm in fp32 -- the
-// bucket is scored again in fp64 with the formula of the general kernel, from the same
-// registers, and ranked on those scores.  The results are those of the general kernel.
 __device__ __forceinline__ void bf16x8_to_f32(const uint4 &u, float out[8])
 {
     const uint32_t w[4] = {u.x, u.y, u.z, u.w};
@@ -233,176 +223,199 @@ __device__ __forceinline__ void bf16x8_to_f32(const uint4 &u, float out[8])
     }
 }
 
-__global__ void __launch_bounds__(256, 4)
-coreset_select_d128_kernel(Geometry g, const __nv_bfloat16 *__restrict__ X, const int32_t *__restrict__ prob_slice,
+// ---------------------------------------------------------------------------------
+// The same selection for the common case dx = 128 and buckets of at most 12 tokens (the
+// paper's (2, 3, 2)), with ONE THREAD PER TOKEN.  A block of 256 threads takes 21 buckets
+// (12 slots per bucket): thread 12 b + l is local token l of the block's bucket b.
+//
+// The block first brings the rows of its 252 tokens into shared memory with coalesced
+// 16-byte asynchronous copies, sixteen consecutive threads per row.  (A thread reading
+// its own row straight from global memory makes every load instruction touch 32 cache
+// lines, and the L1 pipeline, not HBM, sets the pace: measured 0.103 ms per layer at 7 heads
+// of 118 800 tokens; staged: 0.078 ms.)  Every thread then reads its own row and its
+// bucket's centre row from shared memory (rows 272 bytes apart: conflict-free 16-byte
+// reads) and keeps fp32 sums of <centre, row> and <row, row>, taken with the
+// mixed-precision fma on the bf16 halves as they are; the centre's own <row, row> is the
+// centre norm, shared through shared memory.  A warp per bucket with eight lanes per row
+// (the first version of this kernel) needed about 850 warp instructions per bucket and
+// was bound by instruction issue at 0.088 ms.
+//
+// Scores are first taken in fp32 (products of bf16 values are exact there; the sums of 128
+// terms are not): each cosine is then within 2.5e-5 of its true value.  Only the SET of
+// pruned tokens matters, i.e. the order of the k-th and (k+1)-th largest scores, so the
+// fp32 ranking is accepted when those two are at least 2^-13 apart.  Otherwise -- near-ties,
+// exact ties, rows whose squared norm, or whose product of squared norms with the centre's,
+// leaves the range fp32 handles -- the bucket is scored again in fp64 with the formula of
+// the general kernel, the sums running over the channels in ascending order like the plain
+// definition of the cosine, and ranked on those scores.
+// ---------------------------------------------------------------------------------
+#ifndef VORTA_SELECT_THREADS
+#define VORTA_SELECT_THREADS 256
+#endif
+constexpr int kRowsThreads = VORTA_SELECT_THREADS, kRowsSlots = 12, kRowsBuckets = kRowsThreads / kRowsSlots;
+constexpr int kRowsPitch = 272;  // bytes between staged rows: 256 of data, 16 of padding
+
+__global__ void __launch_bounds__(kRowsThreads)
+coreset_select_rows_kernel(Geometry g, const __nv_bfloat16 *__restrict__ X, const int32_t *__restrict__ prob_slice,
                            const int32_t *__restrict__ seg_start, const int32_t *__restrict__ bucket_tab,
                            int32_t *__restrict__ core_idx, int32_t *__restrict__ src_slot)
 {
-    constexpr int32_t dx = 128, kPasses = 3;
+    constexpr int32_t dx = 128;
     constexpr float kGuard = 1.220703125e-4f;  // 2^-13
-    // bucket shape classes (which axes the grid cuts): token count, centre, token offsets
     __shared__ int32_t tab[8 * kBucketTabStride];
+    __shared__ int32_t keep_tab[8];
+    __shared__ float sc32[kRowsThreads], csq_s[kRowsBuckets], lo_s[kRowsBuckets], hi_s[kRowsBuckets];
+    __shared__ double sc64[kRowsThreads], csq64_s[kRowsBuckets];
+    __shared__ int32_t doubt_s[kRowsBuckets];
+    __shared__ uint8_t kept_s[kRowsThreads];
+    __shared__ int32_t tok_s[kRowsThreads];
+    extern __shared__ __align__(16) unsigned char rows_smem[];  // [252][kRowsPitch]
     for (int i = threadIdx.x; i < 8 * kBucketTabStride; i += blockDim.x) tab[i] = bucket_tab[i];
+    if (threadIdx.x < kRowsBuckets) doubt_s[threadIdx.x] = 0;
     __syncthreads();
+    if (threadIdx.x < 8) {
+        const int32_t n = tab[threadIdx.x * kBucketTabStride];
+        keep_tab[threadIdx.x] = max((int32_t)floor(g.ratio * (double)n + 0.5), 1);
+    }
 
-    const int lane = threadIdx.x & 31;
-    const int32_t bkt = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (bkt >= g.n_buckets) return;
+    const int32_t t = threadIdx.x, b = t / kRowsSlots, l = t - b * kRowsSlots;
+    const int32_t bkt = blockIdx.x * kRowsBuckets + b;
+    const bool has_bucket = b < kRowsBuckets && bkt < g.n_buckets;
     const int32_t p = blockIdx.y;
     const int32_t slice = prob_slice ? prob_slice[p] : p;
     const __nv_bfloat16 *Xs = X + (int64_t)slice * g.Ltot * dx;  // video rows of the slice
-
-    const int32_t bt = bkt / (g.nb[2] * g.nb[1]), bhw = bkt - bt * (g.nb[2] * g.nb[1]);
-    const int32_t bh = bhw / g.nb[2], bw = bhw - bh * g.nb[2];
-    const int32_t cls = ((g.T - bt * g.bucket[0] < g.bucket[0]) ? 4 : 0) | ((g.H - bh * g.bucket[1] < g.bucket[1]) ? 2 : 0) |
-                        ((g.W - bw * g.bucket[2] < g.bucket[2]) ? 1 : 0);
-    const int32_t *t = tab + cls * kBucketTabStride;
-    const int32_t n = t[0], centre = t[1];
-    const int32_t origin = (bt * g.bucket[0] * g.H + bh * g.bucket[1]) * g.W + bw * g.bucket[2];
-    auto token_of = [&](int32_t l) -> int32_t { return origin + t[2 + l]; };
-
-    const int sub = lane >> 3, sl = lane & 7;
-    const uint4 zero = make_uint4(0, 0, 0, 0);
-    const uint4 *xc = reinterpret_cast<const uint4 *>(Xs + (int64_t)token_of(centre) * dx);
-    const uint4 c0 = __ldg(xc + sl), c1 = __ldg(xc + sl + 8);
-    uint4 r[kPasses][2];
-#pragma unroll
-    for (int pass = 0; pass < kPasses; ++pass) {
-        const int32_t l = pass * 4 + sub;
-        r[pass][0] = zero;
-        r[pass][1] = zero;
-        if (l < n) {
-            const uint4 *xj = reinterpret_cast<const uint4 *>(Xs + (int64_t)token_of(l) * dx);
-            r[pass][0] = __ldg(xj + sl);
-            r[pass][1] = __ldg(xj + sl + 8);
-        }
+    int32_t n = 0, centre = 0, cls = 0, origin = 0, seg = 0;
+    if (has_bucket) {
+        const int32_t bt = bkt / (g.nb[2] * g.nb[1]), bhw = bkt - bt * (g.nb[2] * g.nb[1]);
+        const int32_t bh = bhw / g.nb[2], bw = bhw - bh * g.nb[2];
+        cls = ((g.T - bt * g.bucket[0] < g.bucket[0]) ? 4 : 0) | ((g.H - bh * g.bucket[1] < g.bucket[1]) ? 2 : 0) |
+              ((g.W - bw * g.bucket[2] < g.bucket[2]) ? 1 : 0);
+        origin = (bt * g.bucket[0] * g.H + bh * g.bucket[1]) * g.W + bw * g.bucket[2];
+        n = tab[cls * kBucketTabStride];
+        centre = tab[cls * kBucketTabStride + 1];
+        seg = seg_start[bkt];  // needed at the end: in flight under the scoring
     }
-
-    int32_t keep = (int32_t)floor(g.ratio * (double)n + 0.5);
-    keep = max(keep, 1);
-    const int32_t k = n - keep;
-    const bool is_tok = lane < n, is_centre = lane == centre;
-
-    // ---- fp32 scores and ranks
-    float my32 = 0.f;
-    bool doubtful = false;
+    const bool is_tok = has_bucket && l < n, is_centre = is_tok && l == centre;
+    const int32_t tok = is_tok ? origin + tab[cls * kBucketTabStride + 2 + l] : 0;
+    // stage the rows: slot s of the block (= thread s's token) at rows_smem + s * kRowsPitch
+    tok_s[t] = is_tok ? tok : -1;
+    __syncthreads();
     {
-        float csq = 0.f;
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            float a[8];
-            bf16x8_to_f32(h ? c1 : c0, a);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) csq = fmaf(a[i], a[i], csq);
+        const uint32_t base = static_cast<uint32_t>(__cvta_generic_to_shared(rows_smem));
+#pragma unroll 4
+        for (int32_t idx = t; idx < kRowsBuckets * kRowsSlots * 16; idx += kRowsThreads) {
+            const int32_t slot = idx >> 4, chunk = idx & 15, tk = tok_s[slot];
+            if (tk >= 0)
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(base + slot * kRowsPitch + chunk * 16),
+                             "l"(reinterpret_cast<const unsigned char *>(Xs + (int64_t)tk * dx) + chunk * 16)
+                             : "memory");
         }
-#pragma unroll
-        for (int m = 4; m >= 1; m >>= 1) csq += __shfl_xor_sync(0xffffffffu, csq, m);
-        doubtful = !(csq > 1e-30f && csq < 1e30f);
-#pragma unroll
-        for (int pass = 0; pass < kPasses; ++pass) {
-            if (pass * 4 >= n) break;  // warp-uniform
-            float dot = 0.f, njsq = 0.f;
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                float a[8], b[8];
-                bf16x8_to_f32(h ? c1 : c0, a);
-                bf16x8_to_f32(r[pass][h], b);
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    dot = fmaf(a[i], b[i], dot);
-                    njsq = fmaf(b[i], b[i], njsq);
-                }
-            }
-#pragma unroll
-            for (int m = 4; m >= 1; m >>= 1) {
-                dot += __shfl_xor_sync(0xffffffffu, dot, m);
-                njsq += __shfl_xor_sync(0xffffffffu, njsq, m);
-            }
-            // the product of the two squared norms must itself be an ordinary fp32 number: two small
-            // norms (or two large ones) each pass the range test and still underflow (overflow) together,
-            // and the infinite or zero score that follows would slip through the guard band
-            const float nsq = csq * njsq;
-            if (pass * 4 + sub < n && !(njsq > 1e-30f && njsq < 1e30f && nsq > 1e-30f && nsq < 1e30f)) doubtful = true;
-            const float score = dot * rsqrtf(nsq);
-            const float got = __shfl_sync(0xffffffffu, score, (lane & 3) * 8);
-            if ((lane >> 2) == pass) my32 = got;
-        }
+        asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
     }
+    __syncthreads();
+    const uint4 *row = reinterpret_cast<const uint4 *>(rows_smem + (size_t)t * kRowsPitch);
+    const uint4 *cen = reinterpret_cast<const uint4 *>(rows_smem + (size_t)(b < kRowsBuckets ? b * kRowsSlots + centre : 0) * kRowsPitch);
+
+    // ---- fp32 sums over the 128 channels
+    float dot = 0.f, nsq = 0.f;
+    if (is_tok) {
+        // four partial sums each (independent chains; the order of an fp32 sum is free here: what the
+        // ranking may rest on is decided by the guard band)
+        float d4[4] = {0.f, 0.f, 0.f, 0.f}, n4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 4
+        for (int i = 0; i < 16; ++i) {
+            // the mixed-precision fma takes the bf16 halves of the words as they are (exact products,
+            // fp32 sums): no unpacking
+            const uint4 cu = cen[i], ru = row[i];
+            const uint32_t cw[4] = {cu.x, cu.y, cu.z, cu.w}, rw[4] = {ru.x, ru.y, ru.z, ru.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                unsigned short a0, a1, r0, r1;
+                asm("mov.b32 {%0, %1}, %2;" : "=h"(a0), "=h"(a1) : "r"(cw[e]));
+                asm("mov.b32 {%0, %1}, %2;" : "=h"(r0), "=h"(r1) : "r"(rw[e]));
+                asm("fma.rn.f32.bf16 %0, %1, %2, %0;" : "+f"(d4[e]) : "h"(a0), "h"(r0));
+                asm("fma.rn.f32.bf16 %0, %1, %2, %0;" : "+f"(n4[e]) : "h"(r0), "h"(r0));
+                asm("fma.rn.f32.bf16 %0, %1, %2, %0;" : "+f"(d4[e]) : "h"(a1), "h"(r1));
+                asm("fma.rn.f32.bf16 %0, %1, %2, %0;" : "+f"(n4[e]) : "h"(r1), "h"(r1));
+            }
+        }
+        dot = (d4[0] + d4[1]) + (d4[2] + d4[3]);
+        nsq = (n4[0] + n4[1]) + (n4[2] + n4[3]);
+    }
+    if (is_centre) csq_s[b] = nsq;
+    __syncthreads();
+
+    // fp32 score; a bucket with a norm (or a product of norms) outside the range fp32 handles is doubtful
+    float my32 = 0.f;
+    if (is_tok && !is_centre) {
+        const float csq = csq_s[b], prod = csq * nsq;
+        if (!(csq > 1e-30f && csq < 1e30f && nsq > 1e-30f && nsq < 1e30f && prod > 1e-30f && prod < 1e30f)) doubt_s[b] = 1;
+        my32 = dot * rsqrtf(prod);
+    }
+    sc32[t] = my32;
+    const int32_t keep = keep_tab[cls], k = n - keep;
+    __syncthreads();
+    // rank among the bucket's other tokens: most similar first, equal scores by ascending index
     int32_t rank = 0;
-    for (int32_t m = 0; m < n; ++m) {
-        const float sm = __shfl_sync(0xffffffffu, my32, m);
-        if (m != centre && (sm > my32 || (sm == my32 && m < lane))) ++rank;
+    if (is_tok && !is_centre) {
+        for (int32_t m = 0; m < n; ++m) {
+            const float sm = sc32[b * kRowsSlots + m];
+            if (m != centre && (sm > my32 || (sm == my32 && m < l))) ++rank;
+        }
+        // last pruned (rank k-1) and first surviving (rank k) token of the bucket
+        if (k > 0 && k < n - 1) {
+            if (rank == k - 1) lo_s[b] = my32;
+            if (rank == k) hi_s[b] = my32;
+        }
     }
-    bool need64 = __any_sync(0xffffffffu, doubtful);
-    if (!need64 && k > 0 && k < n - 1) {
-        // last pruned (rank k-1) against first surviving (rank k) token
-        const uint32_t b_lo = __ballot_sync(0xffffffffu, is_tok && !is_centre && rank == k - 1);
-        const uint32_t b_hi = __ballot_sync(0xffffffffu, is_tok && !is_centre && rank == k);
-        const float s_lo = __shfl_sync(0xffffffffu, my32, __ffs(b_lo) - 1);
-        const float s_hi = __shfl_sync(0xffffffffu, my32, __ffs(b_hi) - 1);
-        need64 = !(s_lo - s_hi >= kGuard);
-    }
+    __syncthreads();
+    const bool need64 = has_bucket && (doubt_s[b] != 0 || (k > 0 && k < n - 1 && !(lo_s[b] - hi_s[b] >= kGuard)));
 
     // ---- fp64 scores and ranks for the buckets the guard band does not clear
-    if (need64) {
-        // (the summation order differs from the general kernel's only in grouping by chunk)
-        double csq = 0.0;
+    double ddot = 0.0, dnsq = 0.0;
+    if (is_tok && need64) {
+        for (int i = 0; i < 16; ++i) {
+            double a[8], r[8];
+            bf16x8_to_f64(cen[i], a);
+            bf16x8_to_f64(row[i], r);
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            double a[8];
-            bf16x8_to_f64(h ? c1 : c0, a);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) csq = fma(a[i], a[i], csq);
-        }
-#pragma unroll
-        for (int m = 4; m >= 1; m >>= 1) csq += shfl_xor_f64(csq, m);
-        const double nc = sqrt(csq);
-        double my64 = 0.0;
-#pragma unroll 1
-        for (int pass = 0; pass < kPasses; ++pass) {
-            if (pass * 4 >= n) break;
-            double dot = 0.0, njsq = 0.0;
-            const uint4 rp0 = pass == 0 ? r[0][0] : (pass == 1 ? r[1][0] : r[2][0]);
-            const uint4 rp1 = pass == 0 ? r[0][1] : (pass == 1 ? r[1][1] : r[2][1]);
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                double a[8], b[8];
-                bf16x8_to_f64(h ? c1 : c0, a);
-                bf16x8_to_f64(h ? rp1 : rp0, b);
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    dot = fma(a[i], b[i], dot);
-                    njsq = fma(b[i], b[i], njsq);
-                }
+            for (int e = 0; e < 8; ++e) {
+                ddot = fma(a[e], r[e], ddot);
+                dnsq = fma(r[e], r[e], dnsq);
             }
-#pragma unroll
-            for (int m = 4; m >= 1; m >>= 1) {
-                dot += shfl_xor_f64(dot, m);
-                njsq += shfl_xor_f64(njsq, m);
-            }
-            const double nj = sqrt(njsq);
-            const double score = (nc == 0.0 || nj == 0.0) ? 0.0 : dot / (nc * nj);
-            const double got = shfl_f64(score, (lane & 3) * 8);
-            if ((lane >> 2) == pass) my64 = got;
         }
+        if (is_centre) csq64_s[b] = dnsq;
+    }
+    __syncthreads();
+    double my64 = 0.0;
+    if (is_tok && need64 && !is_centre) {
+        const double nc = sqrt(csq64_s[b]), nj = sqrt(dnsq);
+        my64 = (nc == 0.0 || nj == 0.0) ? 0.0 : ddot / (nc * nj);
+    }
+    sc64[t] = my64;
+    __syncthreads();
+    if (is_tok && need64 && !is_centre) {
         rank = 0;
         for (int32_t m = 0; m < n; ++m) {
-            const double sm = shfl_f64(my64, m);
-            if (m != centre && (sm > my64 || (sm == my64 && m < lane))) ++rank;
+            const double sm = sc64[b * kRowsSlots + m];
+            if (m != centre && (sm > my64 || (sm == my64 && m < l))) ++rank;
         }
     }
 
+    // ---- the bucket's segment of the index list: centre first, then the other kept tokens ascending
     const bool kept = is_tok && (is_centre || rank >= k);
-    const uint32_t kept_others = __ballot_sync(0xffffffffu, kept && !is_centre);
+    kept_s[t] = kept && !is_centre;
+    __syncthreads();
     if (!is_tok) return;
-    const int32_t seg = seg_start[bkt];
-    const int32_t tok = token_of(lane);
-    int32_t slot = seg;
-    if (kept && !is_centre) slot = seg + 1 + __popc(kept_others & ((1u << lane) - 1u));
+    int32_t slot = seg;  // the centre's slot: pruned tokens receive its output
+    if (kept && !is_centre) {
+        int32_t before = 0;
+        for (int32_t m = 0; m < l; ++m) before += kept_s[b * kRowsSlots + m];
+        slot = seg + 1 + before;
+    }
     if (kept) core_idx[(int64_t)p * g.Lc + slot] = tok;
     src_slot[(int64_t)p * g.L + tok] = slot;
 }
-
 cudaError_t launch_select(const Geometry &g, const __nv_bfloat16 *X, int32_t dx, int32_t n_prob,
                           const int32_t *prob_slice, const int32_t *seg_start, const int32_t *bucket_tab,
                           int32_t *core_idx, int32_t *src_slot, cudaStream_t s)
@@ -410,8 +423,18 @@ cudaError_t launch_select(const Geometry &g, const __nv_bfloat16 *X, int32_t dx,
     int64_t warps = (int64_t)n_prob * g.n_buckets;
     if (warps == 0) return cudaSuccess;
     if (dx == 128 && g.bucket[0] * g.bucket[1] * g.bucket[2] <= 12 && n_prob <= 65535) {
-        dim3 grid((unsigned)((g.n_buckets + 7) / 8), (unsigned)n_prob);
-        coreset_select_d128_kernel<<<grid, 256, 0, s>>>(g, X, prob_slice, seg_start, bucket_tab, core_idx, src_slot);
+        constexpr int kSmem = kRowsBuckets * kRowsSlots * kRowsPitch;
+        // more than 48 KB of dynamic shared memory has to be asked for, once per device
+        static bool attr_set[64] = {};
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return cudaGetLastError();
+        if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+            cudaError_t ea = cudaFuncSetAttribute(coreset_select_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+            if (ea != cudaSuccess) return ea;
+            if (dev >= 0 && dev < 64) attr_set[dev] = true;
+        }
+        dim3 grid((unsigned)((g.n_buckets + kRowsBuckets - 1) / kRowsBuckets), (unsigned)n_prob);
+        coreset_select_rows_kernel<<<grid, kRowsThreads, kSmem, s>>>(g, X, prob_slice, seg_start, bucket_tab, core_idx, src_slot);
     } else {
         int64_t blocks = (warps + 7) / 8;
         coreset_select_kernel<<<(unsigned)blocks, 256, 0, s>>>(g, X, dx, n_prob, prob_slice, seg_start,
@@ -424,27 +447,49 @@ cudaError_t launch_select(const Geometry &g, const __nv_bfloat16 *X, int32_t dx,
 // pool: gather the kept rows of Q, K, V into compact [n_prob, Lc, d] tensors.
 // 16 bytes per thread; blockIdx.y picks the tensor.
 // ---------------------------------------------------------------------------------
+// One problem per blockIdx.y, the tensor per blockIdx.z.  A thread owns one 16-byte chunk of a row and
+// walks the rows in steps of the grid, four rows at a time (four index loads, then four row loads in
+// flight); rows and chunks come from shifts (d / 8 chunks per row is 8 or 16), never from a division.
+constexpr int kCopyUnroll = 4;
+
 __global__ void __launch_bounds__(256)
-gather_rows_kernel(Geometry g, int32_t n_prob, const int32_t *__restrict__ prob_slice,
-                   const int32_t *__restrict__ core_idx, const uint4 *__restrict__ Q,
-                   const uint4 *__restrict__ K, const uint4 *__restrict__ V, uint4 *__restrict__ Qc,
-                   uint4 *__restrict__ Kc, uint4 *__restrict__ Vc)
+gather_rows_kernel(Geometry g, const int32_t *__restrict__ prob_slice, const int32_t *__restrict__ core_idx,
+                   const uint4 *__restrict__ Q, const uint4 *__restrict__ K, const uint4 *__restrict__ V,
+                   uint4 *__restrict__ Qc, uint4 *__restrict__ Kc, uint4 *__restrict__ Vc)
 {
-    const int32_t cpr = g.d >> 3;  // 16-byte chunks per row
+    const int32_t cpr = g.d >> 3, sh = g.d == 128 ? 4 : 3;  // 16-byte chunks per row
+    const int32_t c = (int32_t)threadIdx.x & (cpr - 1), rows_per_block = 256 >> sh;
+    const int32_t p = blockIdx.y;
+    const int32_t slice = prob_slice ? prob_slice[p] : p;
+    const uint4 *src = (blockIdx.z == 0 ? Q : (blockIdx.z == 1 ? K : V)) + (int64_t)slice * g.Ltot * cpr;
+    uint4 *dst = (blockIdx.z == 0 ? Qc : (blockIdx.z == 1 ? Kc : Vc)) + (int64_t)p * g.Lct * cpr;
+    const int32_t *idx = core_idx + (int64_t)p * g.Lc;
+    const int32_t step = (int32_t)gridDim.x * rows_per_block;
     // compact row r of a problem: kept video token core_idx[r] for r < Lc, text token r - Lc after that
-    const int64_t total = (int64_t)n_prob * g.Lct * cpr;
-    const uint4 *src = blockIdx.y == 0 ? Q : (blockIdx.y == 1 ? K : V);
-    uint4 *dst = blockIdx.y == 0 ? Qc : (blockIdx.y == 1 ? Kc : Vc);
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
-         i += (int64_t)gridDim.x * blockDim.x) {
-        int64_t row = i / cpr;
-        int32_t c = (int32_t)(i % cpr);
-        int32_t p = (int32_t)(row / g.Lct);
-        int32_t r = (int32_t)(row % g.Lct);
-        int32_t tok = r < g.Lc ? __ldg(core_idx + (int64_t)p * g.Lc + r) : g.L + (r - g.Lc);
-        const int32_t slice = prob_slice ? prob_slice[p] : p;
-        dst[i] = __ldg(src + ((int64_t)slice * g.Ltot + tok) * cpr + c);
+    for (int32_t r0 = (int32_t)blockIdx.x * rows_per_block + ((int32_t)threadIdx.x >> sh); r0 < g.Lct; r0 += kCopyUnroll * step) {
+        int32_t tok[kCopyUnroll];
+        uint4 v[kCopyUnroll];
+#pragma unroll
+        for (int u = 0; u < kCopyUnroll; ++u) {
+            const int32_t r = r0 + u * step;
+            tok[u] = r < g.Lc ? __ldg(idx + r) : g.L + (r - g.Lc);
+        }
+#pragma unroll
+        for (int u = 0; u < kCopyUnroll; ++u)
+            if (r0 + u * step < g.Lct) v[u] = __ldg(src + (int64_t)tok[u] * cpr + c);
+#pragma unroll
+        for (int u = 0; u < kCopyUnroll; ++u)
+            if (r0 + u * step < g.Lct) dst[(int64_t)(r0 + u * step) * cpr + c] = v[u];
     }
+}
+
+// blocks along x for `rows` rows of one problem: enough to fill the GPU a few times over, no more
+static unsigned copy_blocks(int64_t rows, int32_t d, int64_t n_launch_y)
+{
+    const int64_t rows_per_block = 256 / (d >> 3);
+    int64_t want = (rows + rows_per_block * kCopyUnroll - 1) / (rows_per_block * kCopyUnroll);
+    const int64_t cap = std::max<int64_t>(1, (148 * 16 + n_launch_y - 1) / n_launch_y);
+    return (unsigned)std::max<int64_t>(1, std::min(want, cap));
 }
 
 cudaError_t launch_gather(const Geometry &g, int32_t n_prob, const int32_t *prob_slice,
@@ -453,10 +498,8 @@ cudaError_t launch_gather(const Geometry &g, int32_t n_prob, const int32_t *prob
                           __nv_bfloat16 *Vc, cudaStream_t s)
 {
     if (n_prob == 0) return cudaSuccess;
-    int64_t total = (int64_t)n_prob * g.Lct * (g.d >> 3);
-    unsigned blocks = (unsigned)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
-    gather_rows_kernel<<<dim3(blocks, 3), 256, 0, s>>>(
-        g, n_prob, prob_slice, core_idx, reinterpret_cast<const uint4 *>(Q),
+    gather_rows_kernel<<<dim3(copy_blocks(g.Lct, g.d, (int64_t)n_prob * 3), (unsigned)n_prob, 3), 256, 0, s>>>(
+        g, prob_slice, core_idx, reinterpret_cast<const uint4 *>(Q),
         reinterpret_cast<const uint4 *>(K), reinterpret_cast<const uint4 *>(V),
         reinterpret_cast<uint4 *>(Qc), reinterpret_cast<uint4 *>(Kc), reinterpret_cast<uint4 *>(Vc));
     return cudaGetLastError();
@@ -543,22 +586,32 @@ cudaError_t launch_merge(const Geometry &g, int32_t n_prob, const int32_t *prob_
 // (its own row if kept, its bucket centre's row if pruned).
 // ---------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
-scatter_rows_kernel(Geometry g, int32_t n_prob, const int32_t *__restrict__ prob_slice,
-                    const int32_t *__restrict__ src_slot, const uint4 *__restrict__ Oc,
-                    uint4 *__restrict__ O)
+scatter_rows_kernel(Geometry g, const int32_t *__restrict__ prob_slice, const int32_t *__restrict__ src_slot,
+                    const uint4 *__restrict__ Oc, uint4 *__restrict__ O)
 {
-    const int32_t cpr = g.d >> 3;
+    const int32_t cpr = g.d >> 3, sh = g.d == 128 ? 4 : 3;
+    const int32_t c = (int32_t)threadIdx.x & (cpr - 1), rows_per_block = 256 >> sh;
+    const int32_t p = blockIdx.y;
+    const int32_t slice = prob_slice ? prob_slice[p] : p;
+    const uint4 *src = Oc + (int64_t)p * g.Lct * cpr;
+    uint4 *dst = O + (int64_t)slice * g.Ltot * cpr;
+    const int32_t *slots = src_slot + (int64_t)p * g.L;
+    const int32_t step = (int32_t)gridDim.x * rows_per_block;
     // a video token takes the row of its slot, a text token its own compact row
-    const int64_t total = (int64_t)n_prob * g.Ltot * cpr;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
-         i += (int64_t)gridDim.x * blockDim.x) {
-        int64_t row = i / cpr;
-        int32_t c = (int32_t)(i % cpr);
-        int32_t p = (int32_t)(row / g.Ltot);
-        int32_t tok = (int32_t)(row % g.Ltot);
-        int32_t slot = tok < g.L ? __ldg(src_slot + (int64_t)p * g.L + tok) : g.Lc + (tok - g.L);
-        const int32_t slice = prob_slice ? prob_slice[p] : p;
-        O[((int64_t)slice * g.Ltot + tok) * cpr + c] = __ldg(Oc + ((int64_t)p * g.Lct + slot) * cpr + c);
+    for (int32_t t0 = (int32_t)blockIdx.x * rows_per_block + ((int32_t)threadIdx.x >> sh); t0 < g.Ltot; t0 += kCopyUnroll * step) {
+        int32_t slot[kCopyUnroll];
+        uint4 v[kCopyUnroll];
+#pragma unroll
+        for (int u = 0; u < kCopyUnroll; ++u) {
+            const int32_t tok = t0 + u * step;
+            slot[u] = tok < g.L ? __ldg(slots + tok) : g.Lc + (tok - g.L);
+        }
+#pragma unroll
+        for (int u = 0; u < kCopyUnroll; ++u)
+            if (t0 + u * step < g.Ltot) v[u] = __ldg(src + (int64_t)slot[u] * cpr + c);
+#pragma unroll
+        for (int u = 0; u < kCopyUnroll; ++u)
+            if (t0 + u * step < g.Ltot) dst[(int64_t)(t0 + u * step) * cpr + c] = v[u];
     }
 }
 
@@ -567,11 +620,8 @@ cudaError_t launch_scatter(const Geometry &g, int32_t n_prob, const int32_t *pro
                            cudaStream_t s)
 {
     if (n_prob == 0) return cudaSuccess;
-    int64_t total = (int64_t)n_prob * g.Ltot * (g.d >> 3);
-    unsigned blocks = (unsigned)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
-    scatter_rows_kernel<<<blocks, 256, 0, s>>>(g, n_prob, prob_slice, src_slot,
-                                               reinterpret_cast<const uint4 *>(Oc),
-                                               reinterpret_cast<uint4 *>(O));
+    scatter_rows_kernel<<<dim3(copy_blocks(g.Ltot, g.d, n_prob), (unsigned)n_prob), 256, 0, s>>>(
+        g, prob_slice, src_slot, reinterpret_cast<const uint4 *>(Oc), reinterpret_cast<uint4 *>(O));
     return cudaGetLastError();
 }
 
