@@ -7,6 +7,7 @@
 #include <mutex>
 #include <new>
 #include <queue>
+#include <unordered_map>
 
 #include "vorta_internal.h"
 
@@ -426,6 +427,7 @@ int build_list(vorta_plan *p, vorta_plan::WorkList &wl, const std::vector<uint8_
             if (branches[h] & (1u << VORTA_ROUTE_FULL))
                 linear_items(MODE_LINEAR, slice, by_branch ? VORTA_ROUTE_FULL * BH + slice : slice, g.Ltot, 0, g.Ltot);
             if (branches[h] & (1u << VORTA_ROUTE_SLIDING)) {
+                std::unordered_map<int64_t, size_t> lone;  // window centre -> item holding one lone box so far
                 for (int32_t qt = 0; qt < g.n_tiles; ++qt) {
                     int32_t q[3] = {qt / (g.nt[2] * g.nt[1]), (qt / g.nt[2]) % g.nt[1], qt % g.nt[2]};
                     const int32_t pi = (q[0] * g.nt[1] + q[1]) * (g.nt[2] / 2) + q[2] / 2;
@@ -474,6 +476,27 @@ int build_list(vorta_plan *p, vorta_plan::WorkList &wl, const std::vector<uint8_
                         w.n_mblk = std::min(2, nb - b0);
                         for (int m = 0; m < w.n_mblk; ++m)
                             for (int a = 0; a < 3; ++a) w.q_org[m][a] = org[b0 + m][a];
+                        if (w.n_mblk == 1) {
+                            // A lone box (the one box of a tile the grid cuts down to one, e.g. the last, one-frame
+                            // T tile of the 720p grids) would run with one of the two softmax groups idle.  Tiles
+                            // whose windows have the same centre tile on every axis (neighbours at a border of the
+                            // tile grid) have the SAME key list: two lone boxes of such tiles share an item.
+                            int64_t key = 0;
+                            for (int a = 0; a < 3; ++a) {
+                                const int32_t c = g.restricted[a] ? std::min(std::max(q[a], g.half[a]), g.nt[a] - 1 - g.half[a]) : 0;
+                                key = key * 65536 + c;
+                            }
+                            auto it = lone.find(key);
+                            if (it != lone.end()) {
+                                WorkItem &first = items[it->second];
+                                for (int a = 0; a < 3; ++a) first.q_org[1][a] = w.q_org[0][a];
+                                first.n_mblk = 2;
+                                cost[it->second] = 2.0 * (double)item_keys[it->second] / 128.0 + 2.0;
+                                lone.erase(it);
+                                continue;
+                            }
+                            lone[key] = items.size();
+                        }
                         items.push_back(w);
                         item_keys.push_back(issued_keys[qt] + (int64_t)w.kv_text * g.bn_tile);
                         cost.push_back((double)w.n_mblk * (double)item_keys.back() / 128.0 + 2.0);
