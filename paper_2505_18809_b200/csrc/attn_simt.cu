@@ -57,7 +57,7 @@ attention_simt_kernel(AttnParams p)
             kv_len = g.Ltot;
             org[0] = g.L + (j - (w.kv_count - w.kv_text)) * g.bn_tile; org[1] = 0; org[2] = 0;
         } else if (w.mode == MODE_TILES) {
-            KvEntry e = (packed ? p.kv_pairs : p.kv_list)[w.kv_begin + j];
+            KvEntry e = (item_uses_pair_list(w.flags) ? p.kv_pairs : p.kv_list)[w.kv_begin + j];
             org[0] = e.w0; org[1] = e.h0; org[2] = e.t0;
             vis = e.mask_id >> kVisShift;
             const uint32_t id = e.mask_id & kMaskIdBits;

@@ -150,7 +150,7 @@ __device__ __forceinline__ void kv_block_coords(const AttnParams &p, const WorkI
     if (text) {
         c1 = (j - (w.kv_count - w.kv_text)) * p.g.bn_tile; c2 = 0; c3 = 0; mask_id = 0;
     } else if (w.mode == MODE_TILES) {
-        const KvEntry e = ((w.flags & kItemPacked) ? p.kv_pairs : p.kv_list)[w.kv_begin + j];
+        const KvEntry e = (item_uses_pair_list(w.flags) ? p.kv_pairs : p.kv_list)[w.kv_begin + j];
         c1 = e.w0; c2 = e.h0; c3 = e.t0; mask_id = e.mask_id & kMaskIdBits;
     } else {
         c1 = j * kBlockM; c2 = 0; c3 = 0; mask_id = 0;
@@ -200,10 +200,13 @@ __device__ __forceinline__ void producer_role(const AttnParams &p, const AttnMap
         if (lane == 0) {
             if (w.flags & kItemPacked) {
                 // two tiles of at most 64 tokens in one query block: the second one 64 rows further down
-                mbar_expect_tx(bars + 8 * BAR_Q_FULL, half_bytes * kHalves * 2);
+                // (lone short boxes of larger tiles come through a map whose box is 64 rows at most)
+                const bool lone = (w.flags & kItemSameWindow) != 0;
+                const CUtensorMap *qmap = lone ? &maps.q_lone : &maps.q[w.mode];
+                mbar_expect_tx(bars + 8 * BAR_Q_FULL, (lone ? (uint32_t)p.lone_rows * 128u : half_bytes) * kHalves * 2);
                 for (int t = 0; t < 2; ++t)
                     for (int h = 0; h < kHalves; ++h)
-                        tma_load_5d(smem_base + kSmemQ + h * kHalfBytes + t * (kHalfBytes / 2), &maps.q[w.mode],
+                        tma_load_5d(smem_base + kSmemQ + h * kHalfBytes + t * (kHalfBytes / 2), qmap,
                                     bars + 8 * BAR_Q_FULL, h * 64, w.q_org[t][0], w.q_org[t][1], w.q_org[t][2], w.slice);
             } else {
                 mbar_expect_tx(bars + 8 * BAR_Q_FULL, half_bytes * kHalves * w.n_mblk);
@@ -302,7 +305,7 @@ __device__ __forceinline__ void mma_role(const AttnParams &p, Ctl *ctl, uint32_t
         const bool tiles = uniform_u32((uint32_t)w->mode) == MODE_TILES;
         const int32_t first_cut = tiles ? (int32_t)uniform_u32((uint32_t)w->kv_fast) : n;
         const int32_t n_boxes = n - (tiles ? (int32_t)uniform_u32((uint32_t)w->kv_text) : 0);
-        const KvEntry *entries = (uniform_u32((uint32_t)w->flags) & kItemPacked ? p.kv_pairs : p.kv_list) +
+        const KvEntry *entries = (item_uses_pair_list((int32_t)uniform_u32((uint32_t)w->flags)) ? p.kv_pairs : p.kv_list) +
                                  (tiles ? (int32_t)uniform_u32((uint32_t)w->kv_begin) : 0);
         // The classes of 32 consecutive blocks are fetched with one load (lane l holds block tab_first + l)
         // and handed round by shuffle: a load per block would put a trip to global memory on this warp's
@@ -408,7 +411,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams &p, Ctl *ctl, uint
         if (m >= wp->n_mblk) continue;
         const int32_t w_mode = wp->mode, w_kv_len = wp->kv_len, w_kv_count = wp->kv_count;
         const bool packed = (wp->flags & kItemPacked) != 0;
-        const KvEntry *kv_entries = (packed ? p.kv_pairs : p.kv_list) + wp->kv_begin;
+        const KvEntry *kv_entries = (item_uses_pair_list(wp->flags) ? p.kv_pairs : p.kv_list) + wp->kv_begin;
         // packed item: this row belongs to the first (rows 0-63) or the second tile; a block that only the
         // other tile has in its window holds no key for it (visibility code in the entry's top bits)
         const uint32_t my_vis = packed ? 1u + (uint32_t)(row >> 6) : 0u;

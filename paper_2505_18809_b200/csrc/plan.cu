@@ -36,6 +36,7 @@ struct vorta_plan {
     std::vector<int32_t> pair_begin, pair_count;
     std::vector<int64_t> pair_keys;
     bool pack_tiles = false;
+    int32_t lone_t = 0;  // frames of the lone short box of the last T tile (0: that tile has no such box); see build_list
     // KV boxes the grid cuts (sliding branch): column-mask class -> box shape, and per shape the extents
     // (T, H, W) and the number of keys of the part of the box that lies inside the grid
     uint8_t cls_shape[kMaxMasks + 7] = {};
@@ -486,12 +487,21 @@ int build_list(vorta_plan *p, vorta_plan::WorkList &wl, const std::vector<uint8_
                                 const int32_t c = g.restricted[a] ? std::min(std::max(q[a], g.half[a]), g.nt[a] - 1 - g.half[a]) : 0;
                                 key = key * 65536 + c;
                             }
+                            // (a lone box of at most 64 rows: two of those even fit ONE query block, rows 0-63 and
+                            // 64-127; short boxes only pair with short boxes)
+                            const bool shorty = p->lone_t > 0 && nb == 1 && q[0] == g.nt[0] - 1;
+                            key = key * 2 + (shorty ? 1 : 0);
                             auto it = lone.find(key);
                             if (it != lone.end()) {
                                 WorkItem &first = items[it->second];
                                 for (int a = 0; a < 3; ++a) first.q_org[1][a] = w.q_org[0][a];
-                                first.n_mblk = 2;
-                                cost[it->second] = 2.0 * (double)item_keys[it->second] / 128.0 + 2.0;
+                                if (shorty) {
+                                    first.flags = kItemPacked | kItemSameWindow;
+                                    cost[it->second] = 1.3 * (double)item_keys[it->second] / 128.0 + 2.0;
+                                } else {
+                                    first.n_mblk = 2;
+                                    cost[it->second] = 2.0 * (double)item_keys[it->second] / 128.0 + 2.0;
+                                }
                                 lone.erase(it);
                                 continue;
                             }
@@ -907,6 +917,12 @@ int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
     g.max_kv_per_tile = kv_tiles * g.boxes_per_tile;
     g.text_blocks = (g.Lt + g.bn_tile - 1) / g.bn_tile;
     p->sliding_pairs = sliding_valid_pairs(g);
+    {
+        // The last T tile may hold a single box with fewer frames than a box has: if those frames are at most 64 rows,
+        // two such boxes (of tiles with the same window) fit one 128-row query block.
+        const int32_t rem = g.T - (g.nt[0] - 1) * g.tile[0];
+        if (g.boxes_per_tile > 1 && rem < g.box[0] && rem * g.box[1] * g.box[2] <= 64) p->lone_t = rem;
+    }
 
     if (p->host_only) {
         int rc = build_work(p);
@@ -1230,6 +1246,7 @@ static int run_layer(const vorta_plan *p, const vorta_plan::WorkList &wl, int32_
     prm.kv_list = p->d_kv_list; prm.kv_pairs = p->d_kv_pairs; prm.colmasks = p->d_colmasks;
     std::memcpy(prm.cls_shape, p->cls_shape, sizeof(prm.cls_shape));
     std::memcpy(prm.shape_rows, p->shape_rows, sizeof(prm.shape_rows));
+    prm.lone_rows = p->lone_t * g.box[1] * g.box[2];
     prm.O = o_attn; prm.Oc = Oc; prm.Q = q; prm.K = k; prm.V = v; prm.Qc = Qc; prm.Kc = Kc; prm.Vc = Vc;
     prm.status = p->d_status;
 #ifdef VORTA_TRACE
@@ -1280,6 +1297,10 @@ static int run_layer(const vorta_plan *p, const vorta_plan::WorkList &wl, int32_
                 maps.v_cut[sh] = maps.v[MODE_TILES];
             }
         }
+        if (p->lone_t > 0)
+            ok = ok && make_map(&maps.q_lone, q, g.d, g.W, g.H, g.T, BH, g.box[2], g.box[1], p->lone_t, g.Ltot);
+        else
+            maps.q_lone = maps.q[MODE_TILES];
         if (g.Lt > 0) {
             // the text rows of K and V: Lt rows starting L rows into every head, in boxes of bn_tile rows
             const __nv_bfloat16 *kt = k + (int64_t)g.L * g.d, *vt = v + (int64_t)g.L * g.d;

@@ -53,7 +53,8 @@ struct KvEntry {
 };
 constexpr uint32_t kMaskIdBits = 0x3fffu;
 constexpr int kVisShift = 14;
-constexpr int32_t kItemPacked = 1;  // WorkItem::flags
+constexpr int32_t kItemPacked = 1;      // WorkItem::flags
+constexpr int32_t kItemSameWindow = 2;  // with kItemPacked: both tiles have the item's own window (see WorkItem)
 
 // One unit of work of the attention kernel: up to two 128-row query blocks that
 // walk the same sequence of KV blocks.
@@ -71,9 +72,18 @@ struct WorkItem {
     // kItemPacked (MODE_TILES, tiles of at most 64 tokens, n_mblk = 1): the one query block holds TWO tiles
     // that are neighbours along W, q_org[0] in rows [0, 64) and q_org[1] in rows [64, 128); the KV blocks are
     // the union of the two windows, listed in AttnParams::kv_pairs from kv_begin on.
+    // kItemPacked | kItemSameWindow: the two tiles are lone, short boxes (at most 64 rows, e.g. the one valid frame of
+    // the last T tile) of tiles with the SAME window: the keys are the first tile's list in AttnParams::kv_list, every
+    // block is seen by both, and each box is fetched through AttnMaps::q_lone (a 64-row box).
     int32_t flags;
 };
 static_assert(sizeof(WorkItem) == 64, "WorkItem must stay 64 bytes");
+
+// the KV list an item's kv_begin counts in
+__host__ __device__ inline bool item_uses_pair_list(int32_t flags)
+{
+    return (flags & kItemPacked) && !(flags & kItemSameWindow);
+}
 
 // Tensor maps of one attention launch (all 5-D: d, W|rows, H, T, slice).
 struct AttnMaps {
@@ -84,6 +94,7 @@ struct AttnMaps {
     // grid (index = which axes are cut; 0 is unused, the whole box goes through k/v[MODE_TILES]), so a
     // cut box arrives as a short run of real keys instead of a 128-row box with holes.
     CUtensorMap k_cut[kBoxShapes], v_cut[kBoxShapes];
+    CUtensorMap q_lone;            // Q of the sliding branch in boxes of the lone short box (kItemSameWindow)
 };
 
 struct AttnParams {
@@ -97,6 +108,7 @@ struct AttnParams {
     const uint32_t *colmasks;      // [kMaxMasks][4]
     uint8_t cls_shape[kMaxMasks + 7];  // column-mask class -> box shape (0: whole box, or no short map for it)
     int16_t shape_rows[kBoxShapes];    // keys in a box of each shape (all of them real)
+    int32_t lone_rows;                 // rows of a q_lone box (kItemSameWindow items)
     __nv_bfloat16 *O;              // [B*heads, L + Lt, d]
     __nv_bfloat16 *Oc;             // [n_compact, Lc + Lt, d]
     const __nv_bfloat16 *Q, *K, *V;     // originals (SIMT kernel)
