@@ -39,10 +39,10 @@ DEFAULT_WORKLOAD = "hunyuan-720p"
 FALLBACK_PEAK_TFLOPS = 1590.0   # used only if MEASURED_PEAKS.json is absent
 # DRAM traffic of the attention kernels per algorithmic byte, from ncu captures of the three-head
 # profiling case (profiles/): the single-CTA kernel over all three heads read 441.5 MB and wrote 62.6 MB
-# for 304.1 MB of algorithmic bytes; the pair kernel over the full and the core-set head read 481.5 MB
-# and wrote 84.2 MB for 182.5 MB.  A launch of another workload is estimated by the same ratio.
+# for 304.1 MB of algorithmic bytes; the pair kernel over the full and the core-set head read 445.8 MB
+# and wrote 68.5 MB for 182.5 MB.  A launch of another workload is estimated by the same ratio.
 ATTENTION_TRAFFIC_PER_ALGORITHMIC_BYTE = 504.1 / 304.1
-PAIR_KERNEL_TRAFFIC_PER_ALGORITHMIC_BYTE = 565.7 / 182.5
+PAIR_KERNEL_TRAFFIC_PER_ALGORITHMIC_BYTE = 514.3 / 182.5
 # VORTA_KERNEL_* id -> what the attention stage launches
 ATTENTION_KERNEL_NAMES = {
     0: "attention_sm100_kernel",
