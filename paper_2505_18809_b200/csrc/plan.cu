@@ -959,9 +959,6 @@ int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
             int32_t shape = 0;
             for (int a = 0; a < 3; ++a)
                 if (valid[a] > 0 && valid[a] < g.box[a]) shape |= 4 >> a;
-#ifdef VORTA_NO_SHORT_BOXES
-            shape = 0;
-#endif
             if (valid[0] > 0 && valid[1] > 0 && valid[2] > 0 && shape) {
                 p->cls_shape[id] = (uint8_t)shape;
                 p->shape_rows[shape] = (int16_t)(valid[0] * valid[1] * valid[2]);

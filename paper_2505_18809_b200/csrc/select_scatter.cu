@@ -249,10 +249,7 @@ __device__ __forceinline__ void bf16x8_to_f32(const uint4 &u, float out[8])
 // the general kernel, the sums running over the channels in ascending order like the plain
 // definition of the cosine, and ranked on those scores.
 // ---------------------------------------------------------------------------------
-#ifndef VORTA_SELECT_THREADS
-#define VORTA_SELECT_THREADS 256
-#endif
-constexpr int kRowsThreads = VORTA_SELECT_THREADS, kRowsSlots = 12, kRowsBuckets = kRowsThreads / kRowsSlots;
+constexpr int kRowsThreads = 256, kRowsSlots = 12, kRowsBuckets = kRowsThreads / kRowsSlots;
 constexpr int kRowsPitch = 272;  // bytes between staged rows: 256 of data, 16 of padding
 
 __global__ void __launch_bounds__(kRowsThreads)
