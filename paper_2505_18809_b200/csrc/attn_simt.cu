@@ -52,6 +52,7 @@ attention_simt_kernel(AttnParams p)
         const bool text = w.mode == MODE_TILES && j >= w.kv_count - w.kv_text;
         int32_t kv_mode = w.mode, kv_len = w.kv_len;
         uint32_t vis = 0;  // packed items: which of the two tiles sees the block (0: both)
+        bool paired = false;  // the block is two 64-row boxes: this one and the same box one tile further along W
         if (text) {
             kv_mode = MODE_LINEAR;
             kv_len = g.Ltot;
@@ -60,6 +61,7 @@ attention_simt_kernel(AttnParams p)
             KvEntry e = (item_uses_pair_list(w.flags) ? p.kv_pairs : p.kv_list)[w.kv_begin + j];
             org[0] = e.w0; org[1] = e.h0; org[2] = e.t0;
             vis = e.mask_id >> kVisShift;
+            paired = (e.mask_id & kEntryPaired) != 0;
             const uint32_t id = e.mask_id & kMaskIdBits;
             if (id)
                 for (int i = 0; i < 4; ++i) mask[i] = p.colmasks[id * 4 + i];
@@ -70,8 +72,13 @@ attention_simt_kernel(AttnParams p)
             __syncthreads();
             if (threadIdx.x < kKvChunk) {
                 int32_t n = c0 + threadIdx.x, tok = -1, t;
-                if (n < bn && ((mask[n >> 5] >> (n & 31)) & 1u) &&
-                    block_row_token(g, kv_mode, org, kv_len, n, &t))
+                int32_t o2[3] = {org[0], org[1], org[2]}, nn = n;
+                if (paired && n >= 64) {
+                    o2[0] += g.tile[2];
+                    nn = n - 64;
+                }
+                if (n < bn && (!paired || nn < 64) && ((mask[n >> 5] >> (n & 31)) & 1u) &&
+                    block_row_token(g, kv_mode, o2, kv_len, nn, &t))
                     tok = t;
                 sTok[threadIdx.x] = tok;
             }

@@ -144,14 +144,16 @@ __device__ __forceinline__ uint32_t instr_desc(uint32_t n, uint32_t b_mn_major)
 // block is a run of bn_tile text tokens (the last kv_text blocks of a sliding item), fetched
 // through the text-row tensor maps.
 __device__ __forceinline__ void kv_block_coords(const AttnParams &p, const WorkItem &w, int32_t j, int32_t &c1,
-                                                int32_t &c2, int32_t &c3, uint32_t &mask_id, bool &text)
+                                                int32_t &c2, int32_t &c3, uint32_t &mask_id, bool &text, bool &paired)
 {
+    paired = false;
     text = w.mode == MODE_TILES && j >= w.kv_count - w.kv_text;
     if (text) {
         c1 = (j - (w.kv_count - w.kv_text)) * p.g.bn_tile; c2 = 0; c3 = 0; mask_id = 0;
     } else if (w.mode == MODE_TILES) {
         const KvEntry e = (item_uses_pair_list(w.flags) ? p.kv_pairs : p.kv_list)[w.kv_begin + j];
         c1 = e.w0; c2 = e.h0; c3 = e.t0; mask_id = e.mask_id & kMaskIdBits;
+        paired = (e.mask_id & kEntryPaired) != 0;
     } else {
         c1 = j * kBlockM; c2 = 0; c3 = 0; mask_id = 0;
     }
@@ -219,8 +221,8 @@ __device__ __forceinline__ void producer_role(const AttnParams &p, const AttnMap
         for (int32_t j = 0; j < w.kv_count; ++j) {
             int32_t c1, c2, c3;
             uint32_t mask_id;
-            bool text;
-            kv_block_coords(p, w, j, c1, c2, c3, mask_id, text);
+            bool text, paired;
+            kv_block_coords(p, w, j, c1, c2, c3, mask_id, text, paired);
             // a box the grid cuts is fetched as its part inside the grid: a short run of real keys
             const uint32_t shape = (!text && w.mode == MODE_TILES) ? p.cls_shape[mask_id] : 0u;
             const uint32_t kv_bytes = (text ? (uint32_t)p.g.bn_tile * 128u
@@ -235,9 +237,18 @@ __device__ __forceinline__ void producer_role(const AttnParams &p, const AttnMap
                     const CUtensorMap *map = text ? (kv == 0 ? &maps.kt : &maps.vt)
                                              : shape ? (kv == 0 ? &maps.k_cut[shape] : &maps.v_cut[shape])
                                                      : (kv == 0 ? &maps.k[w.mode] : &maps.v[w.mode]);
-                    for (int h = 0; h < kHalves; ++h)
-                        tma_load_5d(smem_base + kSmemKV + slot * kTileBytes + h * kHalfBytes, map, full, h * 64, c1,
-                                    c2, c3, w.slice);
+                    if (paired) {
+                        // two 64-row boxes (the short T box of this tile and of the next one along W) fill the slot
+                        const CUtensorMap *cut = kv == 0 ? &maps.k_cut[4] : &maps.v_cut[4];
+                        for (int t = 0; t < 2; ++t)
+                            for (int h = 0; h < kHalves; ++h)
+                                tma_load_5d(smem_base + kSmemKV + slot * kTileBytes + h * kHalfBytes + t * (kHalfBytes / 2), cut,
+                                            full, h * 64, c1 + t * p.g.tile[2], c2, c3, w.slice);
+                    } else {
+                        for (int h = 0; h < kHalves; ++h)
+                            tma_load_5d(smem_base + kSmemKV + slot * kTileBytes + h * kHalfBytes, map, full, h * 64, c1,
+                                        c2, c3, w.slice);
+                    }
                 }
                 ++kv_it;
             }

@@ -1013,7 +1013,9 @@ int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out)
     ok = ok && cudaEventCreateWithFlags(&p->ev_start, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&p->ev_out, cudaEventDisableTiming) == cudaSuccess;
     // the mask builder runs once per shape; its per-tile counts come back for the work list
-    ok = ok && launch_block_mask(g, p->d_bm, p->d_kv_list, p->d_kv_count, nullptr) == cudaSuccess;
+    // short T boxes of exactly 64 keys pair up into whole 128-key blocks (see kv_list_kernel)
+    const int32_t pair_t = (g.bn_tile == kBlockM && p->shape_rows[4] == 64 && g.nbox[1] == 1 && g.nbox[2] == 1) ? 1 : 0;
+    ok = ok && launch_block_mask(g, p->d_bm, p->d_kv_list, p->d_kv_count, pair_t, nullptr) == cudaSuccess;
     p->kv_count.resize(2 * (size_t)g.n_tiles);
     ok = ok && cudaMemcpy(p->kv_count.data(), p->d_kv_count, sizeof(int32_t) * 2 * g.n_tiles, cudaMemcpyDeviceToHost) == cudaSuccess;
     ok = ok && attention_sm100_prepare() == cudaSuccess;

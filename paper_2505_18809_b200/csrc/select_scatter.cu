@@ -41,15 +41,28 @@ __global__ void block_mask_kernel(Geometry g, uint8_t *__restrict__ bm)
 // One thread per query tile: turn its mask row into the list of KV blocks the
 // attention kernel walks (key tiles ascending; a tile of more than 128 tokens
 // gives several boxes; boxes that lie wholly outside the grid are dropped).
+// pair_t: a box the grid cuts on T only down to exactly 64 rows (the one valid frame of the last
+// T tile of the 720p grids) is listed together with the same box of the next window tile along W
+// as ONE block of 64 + 64 real keys (kEntryPaired): a whole block as far as the MMAs and the
+// softmax are concerned.
 __global__ void kv_list_kernel(Geometry g, const uint8_t *__restrict__ bm, KvEntry *__restrict__ list,
-                               int32_t *__restrict__ count)
+                               int32_t *__restrict__ count, int32_t pair_t)
 {
     int32_t qt = blockIdx.x * blockDim.x + threadIdx.x;
     if (qt >= g.n_tiles) return;
     KvEntry *out = list + (int64_t)qt * g.max_kv_per_tile;
-    // Two passes: the boxes that lie wholly inside the grid (mask class 0) first, the cut
-    // ones after them, so that the attention kernel can run the leading blocks without
-    // any masking.  count[n_tiles + qt] is the number of leading whole boxes.
+    // the query tile's window along W: tiles [lo_w, hi_w]
+    int32_t lo_w = 0, hi_w = g.nt[2] - 1;
+    if (g.restricted[2]) {
+        const int32_t c = min(max(qt % g.nt[2], g.half[2]), g.nt[2] - 1 - g.half[2]);
+        lo_w = c - g.half[2];
+        hi_w = c + g.half[2];
+    }
+    // the last tile along W does not pair if the grid cuts it
+    const int32_t hi_pair = (g.W - hi_w * g.tile[2] < g.tile[2]) ? hi_w - 1 : hi_w;
+    // Two passes: the boxes that lie wholly inside the grid (mask class 0) and the paired short boxes
+    // first, the other cut ones after them, so that the attention kernel can run the leading blocks
+    // without any masking.  count[n_tiles + qt] is the number of those leading blocks.
     int32_t n = 0, n_whole = 0;
     for (int pass = 0; pass < 2; ++pass) {
         for (int32_t kt = 0; kt < g.n_tiles; ++kt) {
@@ -59,19 +72,30 @@ __global__ void kv_list_kernel(Geometry g, const uint8_t *__restrict__ bm, KvEnt
             int32_t t0 = k[0] * g.tile[0], h0 = k[1] * g.tile[1], w0 = k[2] * g.tile[2];
             int32_t pt = (g.T - t0 < g.tile[0]), ph = (g.H - h0 < g.tile[1]), pw = (g.W - w0 < g.tile[2]);
             bool whole = !pt && !ph && !pw && g.box_rows == g.bn_tile;
-            if (whole != (pass == 0)) continue;
             for (int32_t bx = 0; bx < g.boxes_per_tile; ++bx) {
                 // box bx of the tile; boxes that start outside the grid are dropped
                 int32_t tb = t0 + (bx / (g.nbox[1] * g.nbox[2])) * g.box[0];
                 int32_t hb = h0 + ((bx / g.nbox[2]) % g.nbox[1]) * g.box[1];
                 int32_t wb = w0 + (bx % g.nbox[2]) * g.box[2];
                 if (tb >= g.T || hb >= g.H || wb >= g.W) continue;
+                // a short T box that pairs with its neighbour in the window: position r in the run of
+                // pairable tiles [lo_w, hi_pair] of this row of tiles
+                const int32_t vt = min(g.box[0], g.T - tb);
+                const bool shorty = pair_t && pt && !ph && !pw && vt < g.box[0] && vt * g.box[1] * g.box[2] == 64 &&
+                                    g.nbox[1] == 1 && g.nbox[2] == 1 && k[2] <= hi_pair;
+                const int32_t r = k[2] - lo_w;
+                const bool first_of_pair = shorty && (r % 2 == 0) && k[2] + 1 <= hi_pair;
+                const bool second_of_pair = shorty && (r % 2 == 1);
+                if (second_of_pair) continue;  // listed with the tile before it
+                const bool lead = whole || first_of_pair;
+                if (lead != (pass == 0)) continue;
                 if (n < g.max_kv_per_tile) {
                     KvEntry e;
                     e.w0 = (int16_t)wb;
                     e.h0 = (int16_t)hb;
                     e.t0 = (int16_t)tb;
-                    e.mask_id = whole ? 0 : (uint16_t)(1 + ((pt * 2 + ph) * 2 + pw) * g.boxes_per_tile + bx);
+                    e.mask_id = whole ? 0 : (first_of_pair ? (uint16_t)kEntryPaired
+                                                           : (uint16_t)(1 + ((pt * 2 + ph) * 2 + pw) * g.boxes_per_tile + bx));
                     out[n] = e;
                 }
                 ++n;
@@ -84,13 +108,13 @@ __global__ void kv_list_kernel(Geometry g, const uint8_t *__restrict__ bm, KvEnt
 }
 
 cudaError_t launch_block_mask(const Geometry &g, uint8_t *bm, KvEntry *kv_list, int32_t *kv_count,
-                              cudaStream_t s)
+                              int32_t pair_t, cudaStream_t s)
 {
     int64_t total = (int64_t)g.n_tiles * g.n_tiles;
     block_mask_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(g, bm);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    kv_list_kernel<<<(g.n_tiles + 127) / 128, 128, 0, s>>>(g, bm, kv_list, kv_count);
+    kv_list_kernel<<<(g.n_tiles + 127) / 128, 128, 0, s>>>(g, bm, kv_list, kv_count, pair_t);
     return cudaGetLastError();
 }
 

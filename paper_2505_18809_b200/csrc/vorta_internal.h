@@ -51,7 +51,11 @@ struct KvEntry {
     int16_t w0, h0, t0;
     uint16_t mask_id;
 };
-constexpr uint32_t kMaskIdBits = 0x3fffu;
+constexpr uint32_t kMaskIdBits = 0x1fffu;
+// kEntryPaired (per-tile lists only): the block is TWO boxes, this one and the same box of the next tile along W, each
+// the 64-row part inside the grid of a box the grid cuts on T only (the last, short T tile): 64 + 64 real keys that
+// fill a whole 128-key block, fetched by two loads into the halves of one ring slot.  Its class is 0 (a whole block).
+constexpr uint32_t kEntryPaired = 0x2000u;
 constexpr int kVisShift = 14;
 constexpr int32_t kItemPacked = 1;      // WorkItem::flags
 constexpr int32_t kItemSameWindow = 2;  // with kItemPacked: both tiles have the item's own window (see WorkItem)
@@ -121,7 +125,7 @@ struct AttnParams {
 
 // ---- launchers (each returns cudaGetLastError of its launch) ----------------------
 cudaError_t launch_block_mask(const Geometry &g, uint8_t *bm, KvEntry *kv_list, int32_t *kv_count,
-                              cudaStream_t s);
+                              int32_t pair_t, cudaStream_t s);
 cudaError_t launch_select(const Geometry &g, const __nv_bfloat16 *X, int32_t dx, int32_t n_prob,
                           const int32_t *prob_slice, const int32_t *seg_start, const int32_t *bucket_tab,
                           int32_t *core_idx, int32_t *src_slot, cudaStream_t s);
