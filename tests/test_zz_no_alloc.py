@@ -57,7 +57,7 @@ def test_static_workspace_entry_point_matches_the_workspace_one_twice():
         assert plan.device_status() == 0
         assert torch.cuda.memory_allocated() == before
         if call == 1:
-            assert torch.cuda.mem_get_info()[0] == free_before   # no allocation by anyone, the library included
+            assert torch.cuda.mem_get_info()[0] >= free_before   # nothing was allocated, by the library or anyone
         # same kernels, same inputs: the tolerance of the parity tests, and in fact the same bits
         err = (got.float() - want.float()).abs()
         assert float(err.max()) <= 2e-2 and float(err.mean()) <= 2e-3
