@@ -143,8 +143,15 @@ typedef struct {
 VORTA_API int vorta_plan_create(const vorta_plan_desc *desc, vorta_plan **out);
 
 /* Replace the per-head routes (Section 3.3: the router decides per diffusion
- * timestep) and rebuild the work list; geometry tables are kept.  routes_host is
- * [n] with n == heads.  Synchronises with the plan's device. */
+ * timestep); geometry tables are kept.  routes_host is [n] with n == heads.
+ * Does not wait for the device: the plan keeps the work lists of the last four route
+ * vectors, each in device buffers of its own.  A vector it still holds becomes current
+ * at once (microseconds, nothing touches the device); a new one is built on the host
+ * (about a millisecond for ten thousand work items) into the entry used least recently,
+ * after a wait for the last call that ran THAT entry only, and copied up on a stream of
+ * the plan.  Calls already enqueued keep the lists they were enqueued with.  If a rebuild
+ * fails (VORTA_ERR_CUDA) the plan launches nothing (VORTA_ERR_INTERNAL) until a later
+ * vorta_plan_set_routes succeeds. */
 VORTA_API int vorta_plan_set_routes(vorta_plan *plan, const uint8_t *routes_host, int32_t n);
 
 VORTA_API int vorta_plan_destroy(vorta_plan *plan);
@@ -244,8 +251,8 @@ VORTA_API int vorta_routed_attention(const vorta_plan *plan, const void *Q, cons
  * vorta_plan_info().host_call_scratch_bytes, 256-byte aligned.  Two calls on the
  * same plan must not be in flight on different streams at once (they share the
  * plan's copy streams and events).  The first call after plan creation or a route
- * change builds the groups' work lists (small device allocations, synchronous
- * copies) before it enqueues.
+ * change builds the groups' work lists before it enqueues (small device allocations and
+ * copies, after a wait for the previous host-buffer call of the plan).
  */
 VORTA_API int vorta_routed_attention_host(const vorta_plan *plan, const void *Q_host,
                                           const void *K_host, const void *V_host, void *O_host,
